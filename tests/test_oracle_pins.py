@@ -1,0 +1,411 @@
+"""Pins of the CPU oracle against things other than itself: hand-computed codes (Eq. 1),
+closed forms of the momentum update (Eq. 7-8), brute force in Python integers, cases where
+the quantized forward (Eq. 9) must equal the exact product, the rounding error bound,
+numpy float64 products for the LoRA branch and finite differences for the backward."""
+import os
+
+import numpy as np
+import pytest
+
+import oracle
+from paper_2505_14742_b200 import synth
+
+GOLD = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def bf(x):
+    return synth.f32_to_bf16_bits(np.asarray(x, dtype=np.float32))
+
+
+def f32(b):
+    return synth.bf16_bits_to_f32(b)
+
+
+def half_ulp_bf16(t):
+    """Half a unit in the last place of bf16 (8 significant bits) at the magnitude of t."""
+    return 2.0 ** (np.floor(np.log2(np.maximum(np.abs(t), 1e-300))) - 8)
+
+
+def rand_bf(rng, shape, scale=1.0):
+    return bf(rng.standard_normal(shape).astype(np.float32) * scale)
+
+
+# ----------------------------------------------------------------------------- Eq. 1
+def _golden_rows():
+    rows = []
+    for line in open(os.path.join(GOLD, "quant_examples.txt")):
+        if line.startswith("#") or not line.strip():
+            continue
+        a, b, c = line.split("|")
+        rows.append(([float(v) for v in a.split()], [int(v) for v in b.split()], float(c)))
+    return rows
+
+
+@pytest.mark.parametrize("xs,codes,num", _golden_rows())
+def test_quant_hand_examples_per_token(xs, codes, num):
+    X = bf([xs])
+    assert np.array_equal(f32(X)[0], np.float32(xs)), "example must be exact in bf16"
+    Xq, xqo, dx = oracle.quant_act(X, np.zeros(0, np.int32), np.zeros(0, np.float32), 0)
+    assert Xq[0].tolist() == codes
+    assert dx[0] == np.float32(num) / np.float32(127.0)
+
+
+@pytest.mark.parametrize("xs,codes,num", _golden_rows())
+def test_quant_hand_examples_per_output_channel(xs, codes, num):
+    # the same rows as a weight: row n of Wt is quantized with its own step size
+    Wt = bf([xs, [0.0] * len(xs)])
+    Wq, dW, W_O, wmax = oracle.prepare_weight(Wt, np.zeros(0, np.int32))
+    assert Wq[0].tolist() == codes and Wq[1].tolist() == [0] * len(xs)
+    assert dW[0] == np.float32(num) / np.float32(127.0) and dW[1] == 0.0
+
+
+def test_quant_outlier_column_is_divided_by_s():
+    # x = 100 on the outlier channel, s = 50 -> xhat = 2; the row maximum becomes 4 (channel 0)
+    X = bf([[4.0, 100.0, 1.0, -2.0]])
+    Xq, xqo, dx = oracle.quant_act(X, np.array([1], np.int32), np.array([50.0], np.float32), 4)
+    # r = 127/4 = 31.75: 4 -> 127, 2 -> 63.5 -> 64 (tie to even), 1 -> 31.75 -> 32, -2 -> -63.5 -> -64
+    assert Xq[0].tolist() == [127, 64, 32, -64]
+    assert xqo[0].tolist() == [64, 0, 0, 0]
+    assert dx[0] == np.float32(4.0) / np.float32(127.0)
+
+
+def test_quant_invariants_random():
+    rng = np.random.default_rng(1)
+    X = rand_bf(rng, (37, 129))
+    X[5] = 0
+    O = np.array([3, 77, 128], np.int32)
+    s = np.array([1.5, 7.0, 1.0], np.float32)
+    Xq, xqo, dx, nd = oracle.quant_act(X, O, s, 8, count_literal=True)
+    assert Xq.min() >= -127 and Xq.max() <= 127
+    amax = np.abs(Xq.astype(np.int32)).max(axis=1)
+    assert (amax[np.arange(37) != 5] == 127).all() and amax[5] == 0 and dx[5] == 0
+    assert np.array_equal(xqo[:, :3], Xq[:, O]) and (xqo[:, 3:] == 0).all()
+    # Eq. 1 literally divides by Delta; multiplying by 127/amax may flip a rare tie only
+    assert nd <= 2
+    # step size: the largest |xhat| of the row over 127
+    xh = f32(X).astype(np.float64)
+    xh[:, O] = (f32(X)[:, O] / s[None, :]).astype(np.float64)
+    assert np.allclose(dx, np.abs(xh).max(axis=1) / 127.0, rtol=1e-6)
+    # codes are the nearest integers of xhat / Delta
+    nz = dx > 0
+    assert np.abs(Xq[nz] - xh[nz] / dx[nz, None].astype(np.float64)).max() <= 0.5 + 1e-4
+
+
+def test_requant_rows_hand_example():
+    # W_O (2 outlier rows, 3 output channels), s = (3, 1.5): what = (2*W_O[0], 0.5*W_O[1])
+    W_O = bf([[1.0, -0.5, 0.0], [2.0, 4.0, 0.0]])
+    s = np.array([3.0, 1.5], np.float32)
+    wq, dw = oracle.requant_weight_rows(W_O, s, 4)
+    # column 0: what = (2, 1) -> amax 2 -> codes (127, 63.5 -> 64); column 1: (-1, 2) -> (-63.5 -> -64, 127); column 2: zeros
+    assert wq.tolist() == [[127, 64, 0, 0], [-64, 127, 0, 0], [0, 0, 0, 0]]
+    assert dw.tolist() == [np.float32(2.0) / np.float32(127.0), np.float32(2.0) / np.float32(127.0), 0.0]
+
+
+def test_requant_s_equal_one_gives_zero():
+    rng = np.random.default_rng(2)
+    W_O = rand_bf(rng, (5, 33), 0.02)
+    wq, dw = oracle.requant_weight_rows(W_O, np.ones(5, np.float32), 8)
+    assert not wq.any() and not dw.any()
+
+
+# ----------------------------------------------------------------------------- Eq. 7-8
+def test_beta_exact_values_and_clamp():
+    # colmax = 4 * wmax -> beta = 2 exactly; colmax < wmax -> beta = 1; zero weight row -> beta = 1
+    X = bf([[8.0, 0.25, 3.0], [-2.0, 0.125, 1.0]])
+    O = np.array([0, 1, 2], np.int32)
+    wmax = np.array([2.0, 0.5, 0.0], np.float32)
+    s, cm, be = oracle.momentum_update(X, O, wmax, 0.0, np.ones(3, np.float32))
+    assert cm.tolist() == [8.0, 0.25, 3.0]
+    assert be.tolist() == [2.0, 1.0, 1.0]
+    assert s.tolist() == [2.0, 1.0, 1.0]          # gamma = 0: s_t = beta ("without momentum")
+
+
+def test_momentum_gamma_one_is_static():
+    rng = np.random.default_rng(3)
+    X = rand_bf(rng, (16, 8), 50.0)
+    s0 = np.array([1.0, 3.5, 17.25], np.float32)
+    s, _, _ = oracle.momentum_update(X, np.array([1, 4, 6], np.int32), np.full(3, 0.05, np.float32), 1.0, s0)
+    assert np.array_equal(s, s0)
+
+
+@pytest.mark.parametrize("gamma", [0.2, 0.9])
+def test_momentum_closed_form_constant_input(gamma):
+    # constant X -> constant beta -> s_t = beta + gamma^t (s_0 - beta)
+    X = bf([[9.0, 1.0], [-36.0, 2.0]])
+    O = np.array([0], np.int32)
+    wmax = np.array([0.25], np.float32)           # beta = sqrt(36 / 0.25) = 12
+    s = np.array([1.0], np.float32)
+    for t in range(1, 30):
+        s, _, be = oracle.momentum_update(X, O, wmax, gamma, s)
+        assert be[0] == 12.0
+        expect = 12.0 + (gamma ** t) * (1.0 - 12.0)
+        assert abs(float(s[0]) - expect) <= 2e-6 * expect
+        assert 1.0 <= s[0] <= 12.0
+
+
+def test_momentum_touches_only_outlier_columns():
+    rng = np.random.default_rng(4)
+    X = rand_bf(rng, (20, 10))
+    O = np.array([2, 7], np.int32)
+    wmax = np.array([0.01, 0.02], np.float32)
+    _, cm, _ = oracle.momentum_update(X, O, wmax, 0.5, np.ones(2, np.float32))
+    assert np.array_equal(cm, np.abs(f32(X))[:, O].max(axis=0))
+    X2 = X.copy()
+    X2[:, [0, 1, 3, 4, 5, 6, 8, 9]] = bf(np.float32(1e4))
+    _, cm2, _ = oracle.momentum_update(X2, O, wmax, 0.5, np.ones(2, np.float32))
+    assert np.array_equal(cm, cm2)
+
+
+# ----------------------------------------------------------------------------- integer GEMM
+def test_int_gemm_brute_force_python_ints():
+    rng = np.random.default_rng(5)
+    for (M, N, K) in [(1, 1, 1), (3, 5, 7), (8, 8, 8), (2, 9, 33)]:
+        A = rng.integers(-127, 128, (M, K)).astype(np.int8)
+        B = rng.integers(-127, 128, (N, K)).astype(np.int8)
+        C = oracle.int_gemm(A, B)
+        for m in range(M):
+            for n in range(N):
+                assert int(C[m, n]) == sum(int(A[m, k]) * int(B[n, k]) for k in range(K))
+
+
+def test_int_gemm_extremes():
+    K = 16384
+    A = np.full((2, K), 127, np.int8)
+    B = np.stack([np.full(K, 127, np.int8), np.full(K, -127, np.int8), np.ones(K, np.int8)])
+    C = oracle.int_gemm(A, B)
+    assert C.tolist() == [[16129 * K, -16129 * K, 127 * K]] * 2
+
+
+# ----------------------------------------------------------------------------- Eq. 9 as a whole
+def _setup(rng, M, K, N, nO, r, s_val=None, b_std=0.02, x_scale=1.0):
+    O = np.sort(rng.permutation(K)[:nO]).astype(np.int32)
+    x = rng.standard_normal((M, K)).astype(np.float32) * x_scale
+    x[:, O] *= rng.uniform(20, 100, nO).astype(np.float32)
+    X = bf(x)
+    Wt = rand_bf(rng, (N, K), 0.02)
+    A = rand_bf(rng, (K, r), 0.02) if r else None
+    B = rand_bf(rng, (r, N), b_std) if r else None
+    Wq, dW, W_O, wmax = oracle.prepare_weight(Wt, O)
+    if s_val is None:
+        s, _, _ = oracle.momentum_update(X, O, wmax, 0.0, np.ones(nO, np.float32))
+    else:
+        s = np.full(nO, s_val, np.float32)
+    return O, X, Wt, A, B, Wq, dW, W_O, wmax, s
+
+
+def _forward(O, X, Wq, dW, W_O, s, A, B, lora_scale, nOp):
+    Xq, xqo, dx = oracle.quant_act(X, O, s, nOp)
+    wq, dw = oracle.requant_weight_rows(W_O, s, nOp)
+    Y, T, a1, a2 = oracle.qlinear_fwd(Xq, xqo, dx, Wq, dW, wq, dw, X, A, B, lora_scale)
+    return Y, T, a1, a2, (Xq, xqo, dx, wq, dw)
+
+
+def test_forward_exact_when_quantization_is_lossless():
+    """Integer-valued X and W with every row/column maximum equal to 127 (254 on the outlier
+    channels, s = 2) quantize without error, so Eq. 9 must return X W exactly (Eq. 3-5)."""
+    rng = np.random.default_rng(6)
+    M, K, N = 9, 24, 7
+    O = np.array([2, 11, 23], np.int32)
+    x = rng.integers(-127, 128, (M, K)).astype(np.float32)
+    x[:, 0] = 127                                   # every token row reaches 127 off the outliers
+    x[:, O] = 2 * rng.integers(-127, 128, (M, 3))   # even, up to 254 -> /2 is an integer <= 127
+    w = rng.integers(-127, 128, (N, K)).astype(np.float32)
+    w[:, 1] = 127                                   # every output channel reaches 127
+    w[:, O] = rng.choice([-127.0, 0.0, 127.0], (N, 3))
+    w[:, O[0]] = 127                                # every column of what reaches 127
+    X, Wt = bf(x), bf(w)
+    assert np.array_equal(f32(X), x) and np.array_equal(f32(Wt), w)
+    Wq, dW, W_O, wmax = oracle.prepare_weight(Wt, O)
+    s = np.full(3, 2.0, np.float32)
+    Y, T, a1, a2, _ = _forward(O, X, Wq, dW, W_O, s, None, None, 0.0, 4)
+    exact = x.astype(np.float64) @ w.astype(np.float64).T
+    assert np.array_equal(Y, exact)
+    # brute force of both integer accumulators in Python integers
+    xi = x.astype(np.int64)
+    xi[:, O] //= 2
+    for m in range(M):
+        for n in range(N):
+            assert int(a1[m, n]) == sum(int(xi[m, k]) * int(w[n, k]) for k in range(K))
+            assert int(a2[m, n]) == sum(int(xi[m, O[i]]) * int(w[n, O[i]]) for i in range(3))
+
+
+def test_forward_s_one_equals_naive_waq():
+    """s = 1 makes what = 0, so Eq. 9 must be bit-identical to Eq. 2 (no outlier set at all)."""
+    rng = np.random.default_rng(7)
+    O, X, Wt, A, B, Wq, dW, W_O, wmax, s = _setup(rng, 12, 64, 20, 4, 0, s_val=1.0)
+    Y, _, a1, a2, _ = _forward(O, X, Wq, dW, W_O, s, None, None, 0.0, 8)
+    none = np.zeros(0, np.int32)
+    Wq0, dW0, W_O0, _ = oracle.prepare_weight(Wt, none)
+    Y0, _, b1, b2, _ = _forward(none, X, Wq0, dW0, W_O0, np.zeros(0, np.float32), None, None, 0.0, 0)
+    assert np.array_equal(Y, Y0) and np.array_equal(a1, b1) and not a2.any()
+    # and Eq. 2 written out with numpy on the oracle's codes
+    Xq, _, dx = oracle.quant_act(X, none, np.zeros(0, np.float32), 0)
+    ref = dx.astype(np.float64)[:, None] * (Xq.astype(np.int64) @ Wq0.astype(np.int64).T) * dW0.astype(np.float64)[None, :]
+    assert np.allclose(Y0, ref, rtol=1e-14, atol=0)
+
+
+def test_forward_error_bound_and_outlier_suppression():
+    rng = np.random.default_rng(8)
+    M, K, N, nO = 32, 256, 48, 6
+    O, X, Wt, A, B, Wq, dW, W_O, wmax, s = _setup(rng, M, K, N, nO, 0)
+    assert (s > 1).all()
+    Y, _, _, _, (Xq, xqo, dx, wq, dw) = _forward(O, X, Wq, dW, W_O, s, None, None, 0.0, 8)
+    x = f32(X).astype(np.float64)
+    w = f32(Wt).astype(np.float64)                  # [N,K]
+    exact = x @ w.T
+    # rounding bound of Eq. 1 applied to both GEMMs of Eq. 9: |x - D q| <= D/2 for each factor
+    xh = x.copy()
+    xh[:, O] /= s.astype(np.float64)[None, :]
+    Dx = dx.astype(np.float64)[:, None]
+    DW = dW.astype(np.float64)[None, :]
+    Dw = dw.astype(np.float64)[None, :]
+    what = (s.astype(np.float64) - 1.0)[None, :] * w[:, O]          # [N,nO]
+    slack = 1.0 + 1e-5                                              # fp32 evaluation of the step sizes
+    bound = (np.abs(xh) @ np.ones((K, 1))) * (DW / 2) + (Dx / 2) * (np.ones((M, 1)) @ np.abs(w).sum(axis=1)[None, :]) + K * Dx * DW / 4
+    bound += (np.abs(xh[:, O]).sum(axis=1)[:, None]) * (Dw / 2) + (Dx / 2) * np.abs(what).sum(axis=1)[None, :] + nO * Dx * Dw / 4
+    assert (np.abs(Y - exact) <= bound * slack + 1e-12).all()
+    # outlier suppression must reduce the error of naive W8A8 on outlier-bearing data
+    none = np.zeros(0, np.int32)
+    Wq0, dW0, W_O0, _ = oracle.prepare_weight(Wt, none)
+    Y0 = _forward(none, X, Wq0, dW0, W_O0, np.zeros(0, np.float32), None, None, 0.0, 0)[0]
+    e_quaff = np.linalg.norm(Y - exact)
+    e_naive = np.linalg.norm(Y0 - exact)
+    assert e_quaff < 0.5 * e_naive
+
+
+def test_scaling_identity_on_dequantized_operands():
+    """Eq. 4-5: Xhat W + Xhat_O (s_O - 1) W_O = X W; checked through the oracle's codes: the
+    dequantized operands must reproduce X W within the rounding bound, and the two terms must
+    carry the right channels (a wrong index or a dropped term breaks the agreement)."""
+    rng = np.random.default_rng(9)
+    O, X, Wt, A, B, Wq, dW, W_O, wmax, s = _setup(rng, 16, 128, 24, 5, 0)
+    Y = _forward(O, X, Wq, dW, W_O, s, None, None, 0.0, 8)[0]
+    exact = f32(X).astype(np.float64) @ f32(Wt).astype(np.float64).T
+    rel = np.linalg.norm(Y - exact) / np.linalg.norm(exact)
+    assert rel < 2e-2
+    # dropping the outlier term must be far worse
+    s1 = np.ones_like(s)
+    wq0, dw0 = oracle.requant_weight_rows(W_O, s1, 8)
+    Xq, xqo, dx = oracle.quant_act(X, O, s, 8)
+    Ybad = oracle.qlinear_fwd(Xq, xqo, dx, Wq, dW, wq0, dw0, X, None, None, 0.0)[0]
+    assert np.linalg.norm(Ybad - exact) / np.linalg.norm(exact) > 10 * rel
+
+
+# ----------------------------------------------------------------------------- LoRA
+def test_lora_branch_against_numpy_float64():
+    rng = np.random.default_rng(10)
+    O, X, Wt, A, B, Wq, dW, W_O, wmax, s = _setup(rng, 10, 96, 18, 3, 8)
+    Y1, T, _, _, _ = _forward(O, X, Wq, dW, W_O, s, A, B, 2.0, 4)
+    Y0 = _forward(O, X, Wq, dW, W_O, s, None, None, 0.0, 4)[0]
+    t = f32(X).astype(np.float64) @ f32(A).astype(np.float64)
+    # T is X A rounded once to bf16: within half a bf16 ulp
+    assert (np.abs(f32(T) - t) <= half_ulp_bf16(t)).all()
+    lora = 2.0 * (f32(T).astype(np.float64) @ f32(B).astype(np.float64))
+    assert np.allclose(Y1 - Y0, lora, rtol=1e-9, atol=1e-12)
+    # B = 0 (the usual initialisation): the branch vanishes
+    Yz = _forward(O, X, Wq, dW, W_O, s, A, np.zeros_like(B), 2.0, 4)[0]
+    assert np.array_equal(Yz, Y0)
+
+
+# ----------------------------------------------------------------------------- backward
+def _dequantized_map(O, Wq, dW, wq, dw, s, K):
+    """The linear map of Eq. 9 with the codes held fixed: Y = X @ Weff, Weff[k,n]."""
+    Wd = f32(bf(Wq.astype(np.float32) * dW[:, None])).astype(np.float64)          # [N,K]
+    wd = f32(bf(wq.astype(np.float32) * dw[:, None])).astype(np.float64)          # [N,nOp]
+    Weff = Wd.T.copy()                                                            # [K,N]
+    for i, k in enumerate(O):
+        Weff[k] = (Weff[k] + wd[:, i]) / float(s[i])
+    return Weff
+
+
+def test_backward_dx_by_finite_differences():
+    rng = np.random.default_rng(11)
+    M, K, N, nO, r = 6, 40, 14, 3, 4
+    O, X, Wt, A, B, Wq, dW, W_O, wmax, s = _setup(rng, M, K, N, nO, r, b_std=0.0)   # B = 0: G = 0, map is linear
+    wq, dw = oracle.requant_weight_rows(W_O, s, 8)
+    dY = rand_bf(rng, (M, N), 1e-2)
+    T = bf(np.zeros((M, r), np.float32))
+    dX, dA, dB, G = oracle.qlinear_bwd(dY, Wq, dW, wq, dw, O, s, X, T, A, B, 1.0)
+    assert not G.any()
+    Weff = _dequantized_map(O, Wq, dW, wq, dw, s, K)
+    g = f32(dY).astype(np.float64)
+
+    def loss(x):
+        return float(np.sum(g * (x @ Weff)))
+
+    x0 = f32(X).astype(np.float64)
+    h = 1.0
+    for (m, k) in [(0, 0), (1, int(O[0])), (2, int(O[2])), (5, 39), (3, 17)]:
+        e = np.zeros_like(x0)
+        e[m, k] = h
+        fd = (loss(x0 + e) - loss(x0 - e)) / (2 * h)
+        assert abs(fd - dX[m, k]) <= 1e-9 * max(1.0, abs(fd))
+
+
+def test_backward_matches_full_precision_gradient_statistically():
+    rng = np.random.default_rng(12)
+    M, K, N, nO = 24, 192, 40, 4
+    O, X, Wt, A, B, Wq, dW, W_O, wmax, s = _setup(rng, M, K, N, nO, 0)
+    wq, dw = oracle.requant_weight_rows(W_O, s, 8)
+    dY = rand_bf(rng, (M, N), 1e-2)
+    dX = oracle.qlinear_bwd(dY, Wq, dW, wq, dw, O, s, X, None, None, None, 0.0)[0]
+    full = f32(dY).astype(np.float64) @ f32(Wt).astype(np.float64)
+    assert np.linalg.norm(dX - full) / np.linalg.norm(full) < 3e-2
+    # per-channel: the outlier columns must carry s_i W_i / s_i = W_i as well
+    colerr = np.linalg.norm((dX - full)[:, O], axis=0) / np.linalg.norm(full[:, O], axis=0)
+    assert (colerr < 5e-2).all()
+
+
+def test_backward_lora_grads_against_numpy_float64():
+    rng = np.random.default_rng(13)
+    M, K, N, nO, r = 12, 48, 20, 2, 4
+    O, X, Wt, A, B, Wq, dW, W_O, wmax, s = _setup(rng, M, K, N, nO, r)
+    wq, dw = oracle.requant_weight_rows(W_O, s, 4)
+    Y, T, _, _, _ = _forward(O, X, Wq, dW, W_O, s, A, B, 0.5, 4)
+    dY = rand_bf(rng, (M, N), 1e-2)
+    dX, dA, dB, G = oracle.qlinear_bwd(dY, Wq, dW, wq, dw, O, s, X, T, A, B, 0.5)
+    g = f32(dY).astype(np.float64)
+    gexact = 0.5 * (g @ f32(B).astype(np.float64).T)
+    assert (np.abs(f32(G) - gexact) <= half_ulp_bf16(gexact)).all()
+    Gd = f32(G).astype(np.float64)
+    assert np.allclose(dA, f32(X).astype(np.float64).T @ Gd, rtol=1e-12, atol=1e-15)
+    assert np.allclose(dB, 0.5 * (f32(T).astype(np.float64).T @ g), rtol=1e-12, atol=1e-15)
+    # dX = (codes-fixed linear map)^T dY + G A^T
+    Weff = _dequantized_map(O, Wq, dW, wq, dw, s, K)
+    assert np.allclose(dX, g @ Weff.T + Gd @ f32(A).astype(np.float64).T, rtol=1e-10, atol=1e-14)
+
+
+def test_lora_gradients_by_finite_differences_of_the_forward():
+    """dA and dB are the derivatives of sum(dY * Y) w.r.t. A and B of the oracle's own forward,
+    up to the bf16 roundings of T and G (2^-9 each)."""
+    rng = np.random.default_rng(14)
+    M, K, N, nO, r = 8, 32, 12, 2, 4
+    O, X, Wt, A, B, Wq, dW, W_O, wmax, s = _setup(rng, M, K, N, nO, r, b_std=0.05)
+    wq, dw = oracle.requant_weight_rows(W_O, s, 4)
+    Y, T, _, _, _ = _forward(O, X, Wq, dW, W_O, s, A, B, 1.0, 4)
+    dY = rand_bf(rng, (M, N), 1.0)
+    _, dA, dB, _ = oracle.qlinear_bwd(dY, Wq, dW, wq, dw, O, s, X, T, A, B, 1.0)
+    x = f32(X).astype(np.float64)
+    a = f32(A).astype(np.float64)
+    b = f32(B).astype(np.float64)
+    g = f32(dY).astype(np.float64)
+    dA_true = x.T @ (g @ b.T)
+    dB_true = (x @ a).T @ g
+    assert np.linalg.norm(dA - dA_true) / np.linalg.norm(dA_true) < 4e-3
+    assert np.linalg.norm(dB - dB_true) / np.linalg.norm(dB_true) < 4e-3
+
+
+# ----------------------------------------------------------------------------- generator sanity
+def test_synthetic_workload_shapes_and_outliers():
+    wl = synth.WORKLOADS["tiny"]
+    lin = synth.layer_inputs(wl, 0)
+    X, dY = synth.step_inputs(wl, 0, 0, lin)
+    assert X.shape == (256, 512) and dY.shape == (256, 512) and lin.W.shape == (512, 512)
+    assert len(np.unique(lin.O_idx)) == 8 and (np.diff(lin.O_idx) > 0).all()
+    colmax = np.abs(f32(X)).max(axis=0)
+    rest = np.delete(colmax, lin.O_idx)
+    assert colmax[lin.O_idx].min() > 5 * rest.max()
+    X2, _ = synth.step_inputs(wl, 0, 0, lin)
+    assert np.array_equal(X, X2)
+    X3, _ = synth.step_inputs(wl, 0, 1, lin)
+    assert not np.array_equal(X, X3)
