@@ -1,0 +1,175 @@
+/*
+ * quaff.h — C ABI of the B200 (sm_100a) library for the Quaff quantized linear layer:
+ * INT8 weight-activation quantization with targeted momentum scaling on a fixed set of
+ * outlier input channels, plus the adjacent LoRA branch, forward and backward.
+ *
+ * Notation follows the paper (Sec. 2.2): t -> M tokens, c_in -> K, c_out -> N, Y = X W with
+ * W in R^{c_in x c_out}.  The frozen weight is stored in the nn.Linear layout [N][K]
+ * (Wt[n][k] = W[k][n]), so both INT8 GEMM operands are contiguous along the contraction.
+ * O is the fixed, sorted, duplicate-free set of outlier input channels, nO = |O|; nOp is nO
+ * padded up to a multiple of 32 (the padding columns hold zero codes).
+ *
+ * Conventions
+ *  - Every pointer is a DEVICE pointer unless its comment says "host".  The caller owns every
+ *    buffer; the library allocates nothing and keeps no state between calls.
+ *  - All work is enqueued on the given stream; no call synchronises the device.
+ *  - Matrices are row-major with leading dimensions given in ELEMENTS.
+ *  - bf16 data are raw 16-bit patterns (quaff_bf16); INT8 codes are symmetric in [-127, 127].
+ *  - Scratch memory comes from the caller (`ws`, `ws_bytes`); quaff_workspace_bytes() gives
+ *    the size each entry point needs.  A workspace may be shared by calls on one stream.
+ *  - Return value: QUAFF_OK or an error code; on error nothing has been launched.
+ *    A device-side wait that gave up is reported through the optional `status` word
+ *    (QUAFF_ERR_TIMEOUT) after the stream has been synchronised; outputs are then undefined.
+ *  - Inputs must be finite.  Results are deterministic (no floating-point atomics).
+ */
+#ifndef QUAFF_H_
+#define QUAFF_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef uint16_t quaff_bf16;
+typedef void* quaff_stream_t; /* a cudaStream_t */
+
+typedef enum {
+    QUAFF_OK = 0,
+    QUAFF_ERR_INVALID_ARG = 1,       /* null pointer, negative size, nO > K, gamma outside [0,1], ... */
+    QUAFF_ERR_UNSUPPORTED_SHAPE = 2, /* a size outside what the kernels are built for */
+    QUAFF_ERR_ALIGNMENT = 3,         /* base pointer or leading dimension not 16-byte aligned */
+    QUAFF_ERR_WORKSPACE_TOO_SMALL = 4,
+    QUAFF_ERR_CUDA = 5,              /* a CUDA runtime / driver call failed (launch, tensor map) */
+    QUAFF_ERR_TIMEOUT = 6            /* only ever written to the device `status` word */
+} quaff_status_t;
+
+enum { QUAFF_BF16 = 0, QUAFF_F32 = 1 }; /* y_dtype of quaff_qlinear_fwd */
+
+enum { /* `which` of quaff_workspace_bytes */
+    QUAFF_WS_PREPARE = 0,
+    QUAFF_WS_MOMENTUM = 1,
+    QUAFF_WS_FWD = 2,
+    QUAFF_WS_BWD = 3
+};
+
+const char* quaff_status_string(quaff_status_t s);
+
+/* Bytes of scratch that entry point `which` needs for these sizes (a multiple of 256; may be 0). */
+size_t quaff_workspace_bytes(int which, int M, int K, int N, int nOp, int r);
+
+/*
+ * One-time weight preprocessing (Sec. 3.3, "weights preprocessing"; Eq. 1 per output channel).
+ *   Wt   [N][K] bf16, ldw      frozen weight (in)
+ *   Wq   [N][K] int8, ldwq     codes, Wq[n][k] = [Wt[n][k] / dW[n]]   (out)
+ *   dW   [N] f32               step sizes max_k|Wt[n][k]| / 127       (out)
+ *   W_O  [nO][N] bf16, ldwo    W_O[i][n] = Wt[n][O_i], the only full-precision rows kept (out)
+ *   wmax_O [nO] f32            max_n |W_O[i][n]|, the max|W_i| of Eq. 8 (out)
+ * nO may be 0 (W_O, wmax_O, O_idx may then be null).
+ */
+quaff_status_t quaff_prepare_weight(const quaff_bf16* Wt, int64_t ldw, int N, int K,
+                                    const int32_t* O_idx, int nO,
+                                    int8_t* Wq, int64_t ldwq, float* dW,
+                                    quaff_bf16* W_O, int64_t ldwo, float* wmax_O,
+                                    quaff_stream_t stream);
+
+/*
+ * Targeted momentum scaling (Eq. 8 then Eq. 7), only on the channels of O:
+ *   colmax_i = max_m |X[m][O_i]| ;  beta_i = max(1, sqrt(colmax_i / wmax_O[i]))  (1 if wmax_O[i] = 0)
+ *   s_O[i]  <- gamma * s_O[i] + (1 - gamma) * beta_i
+ *   X [M][K] bf16, ldx (in);  O_idx [nO] int32 (in);  wmax_O [nO] f32 (in);  gamma in [0,1]
+ *   s_O [nO] f32 (in: s_{t-1}, out: s_t; the caller initialises it, 1 = no scaling)
+ *   colmax_O_opt, beta_O_opt [nO] f32: optional diagnostics, may be null
+ *   ws: QUAFF_WS_MOMENTUM bytes.  nO = 0 is a no-op.  fp32, one rounding per operation.
+ */
+quaff_status_t quaff_momentum_update(const quaff_bf16* X, int64_t ldx, int M, int K,
+                                     const int32_t* O_idx, int nO, const float* wmax_O, float gamma,
+                                     float* s_O, float* colmax_O_opt, float* beta_O_opt,
+                                     void* ws, size_t ws_bytes, quaff_stream_t stream);
+
+/*
+ * Scale and quantize the activations (Eq. 5: Xhat = X s^-1, s_i = 1 off O; Eq. 1 per token).
+ *   Xhat[m][O_i] = X[m][O_i] / s_O[i];  dx[m] = max_k|Xhat[m][k]| / 127;
+ *   Xq[m][k] = round_to_nearest_even(Xhat[m][k] * (127 / max_k|Xhat[m][k]|)), clamped to +-127
+ *   xq_O[m][i] = Xq[m][O_i] for i < nO, 0 for nO <= i < nOp      (Eq. 9: xhat_int = [Xhat_int]_{:,O})
+ *   X [M][K] bf16, ldx (in; ldx % 8 == 0);  Xq [M][K] int8, ldxq (out; ldxq % 16 == 0)
+ *   xq_O [M][nOp] int8, ldxo (out; may be null when nOp == 0);  dx [M] f32 (out)
+ * An all-zero row gives dx = 0 and zero codes.  One pass over X.
+ */
+quaff_status_t quaff_quant_act(const quaff_bf16* X, int64_t ldx, int M, int K,
+                               const int32_t* O_idx, int nO, const float* s_O,
+                               int8_t* Xq, int64_t ldxq,
+                               int8_t* xq_O, int64_t ldxo, int nOp,
+                               float* dx, quaff_stream_t stream);
+
+/*
+ * Re-quantize the scaled outlier rows of the weight (Eq. 5: what = (s_O - 1) W_O; Eq. 1 per
+ * output channel; Sec. 3.1 "computing what in real time"):
+ *   what[i][n] = (s_O[i] - 1) * W_O[i][n];  dw_O[n] = max_i|what[i][n]| / 127;
+ *   wq_O[n][i] = round_to_nearest_even(what[i][n] * (127 / max_i|what[i][n]|)), 0 for i >= nO
+ *   W_O [nO][N] bf16, ldwo (in);  s_O [nO] f32 (in)
+ *   wq_O [N][nOp] int8, ldwq (out; same orientation as Wq; ldwq % 16 == 0);  dw_O [N] f32 (out)
+ */
+quaff_status_t quaff_requant_weight_rows(const quaff_bf16* W_O, int64_t ldwo, int nO, int N,
+                                         const float* s_O,
+                                         int8_t* wq_O, int64_t ldwq, int nOp,
+                                         float* dw_O, quaff_stream_t stream);
+
+/*
+ * Forward (Eq. 9) with the LoRA branch fused into the epilogue:
+ *   acc1 = Xq Wq^T  (INT8 x INT8 -> INT32 over K),  acc2 = xq_O wq_O^T  (over nOp)
+ *   T    = bf16(X A)                                                     [M][r], LoRA down-projection
+ *   Y[m][n] = dx[m] * (acc1[m][n] * dW[n] + acc2[m][n] * dw_O[n]) + lora_scale * (T B)[m][n]
+ *   Xq [M][K], ldxq;  xq_O [M][nOp], ldxo;  dx [M]           from quaff_quant_act
+ *   Wq [N][K], ldwq_main;  dW [N]                             frozen (quaff_prepare_weight)
+ *   wq_O [N][nOp], ldwq;  dw_O [N]                            from quaff_requant_weight_rows
+ *   X [M][K] bf16, ldx;  A [K][r] bf16;  B [r][N] bf16        LoRA (dense, ld = r and N); r == 0 disables
+ *   T_out [M][r] bf16 (out, dense; kept for the backward)
+ *   Y [M][N], ldy, y_dtype QUAFF_BF16 or QUAFF_F32 (out)
+ *   dbg_acc_main, dbg_acc_out: optional dense [M][N] int32 dumps of acc1 / acc2 (parity checks)
+ *   status_opt: optional int32[4] device word, must be zero on entry; see QUAFF_ERR_TIMEOUT
+ *   ws: QUAFF_WS_FWD bytes
+ * Alignment: all matrix bases 16-byte aligned; ldxq, ldxo, ldwq_main, ldwq multiples of 16;
+ * ldx multiple of 8; r multiple of 8, r <= 256; nOp multiple of 32 (0 allowed).
+ */
+quaff_status_t quaff_qlinear_fwd(int M, int K, int N,
+                                 const int8_t* Xq, int64_t ldxq, const int8_t* xq_O, int64_t ldxo, int nOp,
+                                 const float* dx,
+                                 const int8_t* Wq, int64_t ldwq_main, const float* dW,
+                                 const int8_t* wq_O, int64_t ldwq, const float* dw_O,
+                                 const quaff_bf16* X, int64_t ldx, const quaff_bf16* A, const quaff_bf16* B,
+                                 int r, float lora_scale,
+                                 quaff_bf16* T_out,
+                                 void* Y, int y_dtype, int64_t ldy,
+                                 int32_t* dbg_acc_main, int32_t* dbg_acc_out,
+                                 int32_t* status_opt, void* ws, size_t ws_bytes, quaff_stream_t stream);
+
+/*
+ * Backward.  The paper states no backward; this is the straight-through derivative of Eq. 9
+ * with s and every step size held constant.  Gradients are not quantized (the paper keeps the
+ * model in floating point and applies INT8 to the linear layers' forward operands only); the
+ * frozen weight is used through its INT8 codes, dequantized to bf16 on the fly:
+ *   Wd[n][k] = bf16(Wq[n][k] * dW[n]),  wd[n][i] = bf16(wq_O[n][i] * dw_O[n])
+ *   dXhat = dY Wd ;  dXhat[:,O_i] += dY wd[:,i] ;  dXhat[:,O_i] /= s_O[i]
+ *   G  = bf16(lora_scale * dY B^T)                                   [M][r]
+ *   dX = dXhat + G A^T                                               [M][K] bf16, lddx (nullable: skipped)
+ *   dA = X^T G  [K][r] f32 ;  dB = lora_scale * T^T dY  [r][N] f32   (nullable pair; accumulate != 0 adds)
+ *   dY [M][N] bf16, lddy (lddy % 8 == 0);  T [M][r] bf16 from the forward
+ *   ws: QUAFF_WS_BWD bytes;  status_opt as in the forward.
+ */
+quaff_status_t quaff_qlinear_bwd(int M, int K, int N,
+                                 const quaff_bf16* dY, int64_t lddy,
+                                 const int8_t* Wq, int64_t ldwq_main, const float* dW,
+                                 const int8_t* wq_O, int64_t ldwq, const float* dw_O, int nOp,
+                                 const int32_t* O_idx, int nO, const float* s_O,
+                                 const quaff_bf16* X, int64_t ldx, const quaff_bf16* T,
+                                 const quaff_bf16* A, const quaff_bf16* B, int r, float lora_scale,
+                                 quaff_bf16* dX, int64_t lddx,
+                                 float* dA, float* dB, int accumulate,
+                                 int32_t* status_opt, void* ws, size_t ws_bytes, quaff_stream_t stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* QUAFF_H_ */

@@ -1,0 +1,380 @@
+// HBM-bound kernels of the Quaff linear layer: momentum scale update (Eq. 7-8), activation
+// scaling + per-token INT8 quantization (Eq. 5, Eq. 1), outlier weight-row re-quantization
+// (Eq. 5, Eq. 1 per output channel) and the one-time weight preprocessing.
+//
+// Bit-exactness contract: every value that decides an INT8 code, a step size or a scale factor is
+// computed in fp32 with explicit round-to-nearest intrinsics (__fmul_rn, __fdiv_rn, __fsqrt_rn,
+// __fadd_rn, __fsub_rn), which the compiler never contracts into FMAs.
+#include "common.cuh"
+
+namespace quaff {
+
+int sm_count() {
+    static int cached[64] = {0};
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (dev < 0 || dev >= 64) dev = 0;
+    if (cached[dev] == 0) {
+        int n = 0;
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
+        cached[dev] = n;
+    }
+    return cached[dev];
+}
+
+// =====================================================================================
+// Activation scaling + per-token quantization (one pass over X)
+// =====================================================================================
+// One CTA owns one token row at a time and keeps it in registers as packed bf16 between the
+// absmax reduction and the quantization, so X is read from HBM exactly once.  A thread owns up to
+// J "units" of 16 consecutive channels (two 128-bit loads, one 128-bit store of codes).  Which of
+// a thread's units contain outlier channels is the same for every row, so it is found once per
+// CTA (binary search in the sorted O) and kept in registers; those units divide the outlier
+// elements by s before both the absmax and the rounding.
+
+__device__ __forceinline__ void unit_decode(const uint4& a, const uint4& b, float (&v)[16]) {
+    const uint32_t w[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        v[2 * i] = bf16_lo(w[i]);
+        v[2 * i + 1] = bf16_hi(w[i]);
+    }
+}
+
+__device__ __forceinline__ void unit_apply_scale(float (&v)[16], int ustart, int obeg, int ocnt,
+                                                 const int* O_s, const float* s_s) {
+    for (int t = 0; t < ocnt; ++t) {
+        const int e = O_s[obeg + t] - ustart;
+        const float sv = s_s[obeg + t];
+#pragma unroll
+        for (int i = 0; i < 16; ++i)
+            if (i == e) v[i] = __fdiv_rn(v[i], sv);
+    }
+}
+
+template <int J>
+__global__ void __launch_bounds__(256) quant_act_kernel(const uint16_t* __restrict__ X, int64_t ldx, int M, int K,
+                                                        const int32_t* __restrict__ O_idx, int nO,
+                                                        const float* __restrict__ s_O,
+                                                        int8_t* __restrict__ Xq, int64_t ldxq,
+                                                        int8_t* __restrict__ xq_O, int64_t ldxo, int nOp,
+                                                        float* __restrict__ dx) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    float* red = reinterpret_cast<float*>(smem_raw);            // [2][8]
+    int* O_s = reinterpret_cast<int*>(smem_raw + 64);           // [nO]
+    float* s_s = reinterpret_cast<float*>(smem_raw + 64) + nO;  // [nO]
+
+    const int tid = threadIdx.x, T = blockDim.x;
+    const int lane = tid & 31, warp = tid >> 5, nwarps = T >> 5;
+    const int nunits = (K + 15) >> 4;
+
+    for (int i = tid; i < nO; i += T) {
+        O_s[i] = O_idx[i];
+        s_s[i] = s_O[i];
+    }
+    __syncthreads();
+
+    int obeg[J], ocnt[J];
+#pragma unroll
+    for (int j = 0; j < J; ++j) {
+        const int u = tid + j * T;
+        obeg[j] = 0;
+        ocnt[j] = 0;
+        if (u < nunits && nO > 0) {
+            const int lo_key = u << 4, hi_key = lo_key + 16;
+            int lo = 0, hi = nO;
+            while (lo < hi) {  // first index with O >= lo_key
+                const int mid = (lo + hi) >> 1;
+                if (O_s[mid] < lo_key) lo = mid + 1; else hi = mid;
+            }
+            const int b = lo;
+            hi = nO;
+            while (lo < hi) {  // first index with O >= hi_key
+                const int mid = (lo + hi) >> 1;
+                if (O_s[mid] < hi_key) lo = mid + 1; else hi = mid;
+            }
+            obeg[j] = b;
+            ocnt[j] = lo - b;
+        }
+    }
+
+    int parity = 0;
+    for (int m = blockIdx.x; m < M; m += gridDim.x, parity ^= 1) {
+        const uint16_t* xrow = X + (int64_t)m * ldx;
+        uint4 raw[J][2];
+#pragma unroll
+        for (int j = 0; j < J; ++j) {
+            const int u = tid + j * T;
+            const int k0 = u << 4;
+            if (k0 + 16 <= K) {
+                const uint4* p = reinterpret_cast<const uint4*>(xrow + k0);
+                raw[j][0] = __ldg(p);
+                raw[j][1] = __ldg(p + 1);
+            } else {
+                uint32_t w[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+                for (int e = 0; e < 16; ++e)
+                    if (k0 + e < K) w[e >> 1] |= (uint32_t)xrow[k0 + e] << ((e & 1) * 16);
+                raw[j][0] = make_uint4(w[0], w[1], w[2], w[3]);
+                raw[j][1] = make_uint4(w[4], w[5], w[6], w[7]);
+            }
+        }
+        float amax = 0.0f;
+#pragma unroll
+        for (int j = 0; j < J; ++j) {
+            float v[16];
+            unit_decode(raw[j][0], raw[j][1], v);
+            if (ocnt[j]) unit_apply_scale(v, (tid + j * T) << 4, obeg[j], ocnt[j], O_s, s_s);
+#pragma unroll
+            for (int i = 0; i < 16; ++i) amax = fmaxf(amax, fabsf(v[i]));
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+        if (nwarps > 1) {
+            if (lane == 0) red[parity * 8 + warp] = amax;
+            __syncthreads();
+            amax = red[parity * 8];
+            for (int w = 1; w < nwarps; ++w) amax = fmaxf(amax, red[parity * 8 + w]);
+        }
+        const float rinv = amax > 0.0f ? __fdiv_rn(127.0f, amax) : 0.0f;
+        if (tid == 0) dx[m] = __fdiv_rn(amax, 127.0f);
+
+        int8_t* qrow = Xq + (int64_t)m * ldxq;
+#pragma unroll
+        for (int j = 0; j < J; ++j) {
+            const int u = tid + j * T;
+            const int k0 = u << 4;
+            if (k0 >= K) continue;
+            float v[16];
+            unit_decode(raw[j][0], raw[j][1], v);
+            if (ocnt[j]) unit_apply_scale(v, k0, obeg[j], ocnt[j], O_s, s_s);
+            uint32_t c[4] = {0, 0, 0, 0};
+#pragma unroll
+            for (int i = 0; i < 16; ++i) c[i >> 2] |= ((uint32_t)quant_code(v[i], rinv) & 0xFFu) << ((i & 3) * 8);
+            if (k0 + 16 <= K) {
+                *reinterpret_cast<uint4*>(qrow + k0) = make_uint4(c[0], c[1], c[2], c[3]);
+            } else {
+                for (int e = 0; e < 16 && k0 + e < K; ++e) qrow[k0 + e] = (int8_t)((c[e >> 2] >> ((e & 3) * 8)) & 0xFFu);
+            }
+            for (int t = 0; t < ocnt[j]; ++t) {  // Eq. 9: the outlier operand is a column gather of the codes
+                const int e = O_s[obeg[j] + t] - k0;
+                xq_O[(int64_t)m * ldxo + obeg[j] + t] = (int8_t)((c[e >> 2] >> ((e & 3) * 8)) & 0xFFu);
+            }
+        }
+        for (int i = nO + tid; i < nOp; i += T) xq_O[(int64_t)m * ldxo + i] = 0;
+    }
+}
+
+template <int J>
+static quaff_status_t launch_quant_act(int T, const uint16_t* X, int64_t ldx, int M, int K, const int32_t* O_idx, int nO,
+                                       const float* s_O, int8_t* Xq, int64_t ldxq, int8_t* xq_O, int64_t ldxo, int nOp,
+                                       float* dx, cudaStream_t st) {
+    const size_t smem = 64 + (size_t)nO * 8;
+    int per_sm = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, quant_act_kernel<J>, T, smem) != cudaSuccess || per_sm < 1)
+        per_sm = 1;
+    const int grid = min(M, sm_count() * per_sm);
+    quant_act_kernel<J><<<grid, T, smem, st>>>(X, ldx, M, K, O_idx, nO, s_O, Xq, ldxq, xq_O, ldxo, nOp, dx);
+    return launch_status();
+}
+
+static quaff_status_t quant_act_dispatch(const uint16_t* X, int64_t ldx, int M, int K, const int32_t* O_idx, int nO,
+                                         const float* s_O, int8_t* Xq, int64_t ldxq, int8_t* xq_O, int64_t ldxo,
+                                         int nOp, float* dx, cudaStream_t st) {
+    const int nunits = (K + 15) / 16;
+    int J = ceil_div(nunits, 256);
+    if (J > 8) return QUAFF_ERR_UNSUPPORTED_SHAPE;  // K > 32768
+    const int T = min(256, ceil_div(ceil_div(nunits, J), 32) * 32);
+#define QA(JJ) return launch_quant_act<JJ>(T, X, ldx, M, K, O_idx, nO, s_O, Xq, ldxq, xq_O, ldxo, nOp, dx, st)
+    switch (J) {
+        case 1: QA(1);
+        case 2: QA(2);
+        case 3: QA(3);
+        case 4: QA(4);
+        case 5:
+        case 6: QA(6);
+        default: QA(8);
+    }
+#undef QA
+}
+
+// =====================================================================================
+// Momentum scale update (Eq. 8 then Eq. 7), only over the channels of O
+// =====================================================================================
+// Column maxima of |X| over the nO outlier columns: each block scans a slice of rows (lane =
+// channel, warp = row), reduces in shared memory and merges with an integer atomicMax on the
+// fp32 bit pattern (non-negative floats order like integers, so the result is exact and
+// order-free).  The last block to finish derives beta and updates s.
+__global__ void __launch_bounds__(256) momentum_kernel(const uint16_t* __restrict__ X, int64_t ldx, int M,
+                                                       const int32_t* __restrict__ O_idx, int nO,
+                                                       const float* __restrict__ wmax_O, float gamma,
+                                                       float* __restrict__ s_O, float* __restrict__ colmax_opt,
+                                                       float* __restrict__ beta_opt, unsigned int* __restrict__ ws) {
+    __shared__ unsigned int red[8][32];
+    __shared__ int is_last;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int rows_per_block = (M + gridDim.x - 1) / gridDim.x;
+    const int r0 = blockIdx.x * rows_per_block;
+    const int r1 = min(M, r0 + rows_per_block);
+
+    for (int c0 = 0; c0 < nO; c0 += 32) {
+        const int i = c0 + lane;
+        unsigned int best = 0;
+        if (i < nO) {
+            const int col = O_idx[i];
+            for (int m = r0 + warp; m < r1; m += 8) {
+                const unsigned int mag = ((unsigned int)X[(int64_t)m * ldx + col] & 0x7FFFu) << 16;  // |x| as fp32 bits
+                best = max(best, mag);
+            }
+        }
+        red[warp][lane] = best;
+        __syncthreads();
+        if (warp == 0) {
+#pragma unroll
+            for (int w = 1; w < 8; ++w) best = max(best, red[w][lane]);
+            if (i < nO && best) atomicMax(&ws[i], best);
+        }
+        __syncthreads();
+    }
+    __threadfence();
+    if (tid == 0) is_last = (atomicAdd(&ws[nO], 1u) == gridDim.x - 1);
+    __syncthreads();
+    if (!is_last) return;
+    __threadfence();
+    const float one_minus_gamma = __fsub_rn(1.0f, gamma);
+    for (int i = tid; i < nO; i += blockDim.x) {
+        const float cmax = __uint_as_float(*reinterpret_cast<volatile unsigned int*>(&ws[i]));
+        const float wmax = wmax_O[i];
+        float beta = 1.0f;
+        if (wmax > 0.0f) beta = fmaxf(1.0f, __fsqrt_rn(__fdiv_rn(cmax, wmax)));   // Eq. 8
+        s_O[i] = __fadd_rn(__fmul_rn(gamma, s_O[i]), __fmul_rn(one_minus_gamma, beta));  // Eq. 7
+        if (colmax_opt) colmax_opt[i] = cmax;
+        if (beta_opt) beta_opt[i] = beta;
+    }
+}
+
+// =====================================================================================
+// Outlier weight rows: what = (s_O - 1) W_O, per-output-channel quantization
+// =====================================================================================
+// One thread per output channel n: reads down column n of W_O (coalesced across n), twice (the
+// second pass comes from L2), and writes its own row of codes wq_O[n][0..nOp).
+__global__ void __launch_bounds__(64) requant_rows_kernel(const uint16_t* __restrict__ W_O, int64_t ldwo, int nO, int N,
+                                                          const float* __restrict__ s_O, int8_t* __restrict__ wq_O,
+                                                          int64_t ldwq, int nOp, float* __restrict__ dw_O) {
+    const int n = blockIdx.x * blockDim.x + threadIdx.x;
+    if (n >= N) return;
+    float amax = 0.0f;
+    for (int i = 0; i < nO; ++i) {
+        const float sm1 = __fsub_rn(__ldg(s_O + i), 1.0f);
+        const float w = __fmul_rn(sm1, bf16_bits_to_f32(__ldg(W_O + (int64_t)i * ldwo + n)));
+        amax = fmaxf(amax, fabsf(w));
+    }
+    dw_O[n] = __fdiv_rn(amax, 127.0f);
+    const float rinv = amax > 0.0f ? __fdiv_rn(127.0f, amax) : 0.0f;
+    int8_t* out = wq_O + (int64_t)n * ldwq;
+    for (int i0 = 0; i0 < nOp; i0 += 16) {
+        uint32_t c[4] = {0, 0, 0, 0};
+#pragma unroll
+        for (int e = 0; e < 16; ++e) {
+            const int i = i0 + e;
+            if (i < nO) {
+                const float sm1 = __fsub_rn(__ldg(s_O + i), 1.0f);
+                const float w = __fmul_rn(sm1, bf16_bits_to_f32(__ldg(W_O + (int64_t)i * ldwo + n)));
+                c[e >> 2] |= ((uint32_t)quant_code(w, rinv) & 0xFFu) << ((e & 3) * 8);
+            }
+        }
+        *reinterpret_cast<uint4*>(out + i0) = make_uint4(c[0], c[1], c[2], c[3]);
+    }
+}
+
+// =====================================================================================
+// Weight preprocessing helpers: gather the outlier rows W_O and their maxima
+// =====================================================================================
+__global__ void __launch_bounds__(256) gather_outlier_rows_kernel(const uint16_t* __restrict__ Wt, int64_t ldw, int N,
+                                                                 const int32_t* __restrict__ O_idx,
+                                                                 uint16_t* __restrict__ W_O, int64_t ldwo,
+                                                                 float* __restrict__ wmax_O) {
+    __shared__ unsigned int red[8];
+    const int i = blockIdx.x;
+    const int col = O_idx[i];
+    unsigned int best = 0;
+    for (int n = threadIdx.x; n < N; n += blockDim.x) {
+        const uint16_t w = Wt[(int64_t)n * ldw + col];
+        W_O[(int64_t)i * ldwo + n] = w;
+        best = max(best, ((unsigned int)w & 0x7FFFu) << 16);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) best = max(best, __shfl_xor_sync(0xffffffffu, best, o));
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = best;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        for (int w = 1; w < 8; ++w) best = max(best, red[w]);
+        wmax_O[i] = __uint_as_float(best);
+    }
+}
+
+static bool valid_outlier_args(const int32_t* O_idx, int nO, int K) {
+    return nO >= 0 && nO <= K && nO <= 4096 && (nO == 0 || O_idx != nullptr);
+}
+
+}  // namespace quaff
+
+using namespace quaff;
+
+extern "C" quaff_status_t quaff_quant_act(const quaff_bf16* X, int64_t ldx, int M, int K, const int32_t* O_idx, int nO,
+                                          const float* s_O, int8_t* Xq, int64_t ldxq, int8_t* xq_O, int64_t ldxo,
+                                          int nOp, float* dx, quaff_stream_t stream) {
+    QUAFF_RETURN_IF(!X || !Xq || !dx || M < 0 || K <= 0, QUAFF_ERR_INVALID_ARG);
+    QUAFF_RETURN_IF(!valid_outlier_args(O_idx, nO, K) || (nO > 0 && !s_O), QUAFF_ERR_INVALID_ARG);
+    QUAFF_RETURN_IF(nOp < nO || (nOp > 0 && !xq_O) || ldx < K || ldxq < K || (nOp > 0 && ldxo < nOp), QUAFF_ERR_INVALID_ARG);
+    QUAFF_RETURN_IF(!aligned16(X) || !aligned16(Xq) || (ldx % 8) || (ldxq % 16), QUAFF_ERR_ALIGNMENT);
+    if (M == 0) return QUAFF_OK;
+    return quant_act_dispatch(X, ldx, M, K, O_idx, nO, s_O, Xq, ldxq, xq_O, ldxo, nOp, dx, (cudaStream_t)stream);
+}
+
+extern "C" quaff_status_t quaff_momentum_update(const quaff_bf16* X, int64_t ldx, int M, int K, const int32_t* O_idx,
+                                                int nO, const float* wmax_O, float gamma, float* s_O,
+                                                float* colmax_O_opt, float* beta_O_opt, void* ws, size_t ws_bytes,
+                                                quaff_stream_t stream) {
+    QUAFF_RETURN_IF(!X || M < 0 || K <= 0 || ldx < K, QUAFF_ERR_INVALID_ARG);
+    QUAFF_RETURN_IF(!valid_outlier_args(O_idx, nO, K), QUAFF_ERR_INVALID_ARG);
+    QUAFF_RETURN_IF(!(gamma >= 0.0f && gamma <= 1.0f), QUAFF_ERR_INVALID_ARG);
+    if (nO == 0) return QUAFF_OK;
+    QUAFF_RETURN_IF(!wmax_O || !s_O, QUAFF_ERR_INVALID_ARG);
+    QUAFF_RETURN_IF(!ws || ws_bytes < quaff_workspace_bytes(QUAFF_WS_MOMENTUM, M, K, 0, nO, 0), QUAFF_ERR_WORKSPACE_TOO_SMALL);
+    cudaStream_t st = (cudaStream_t)stream;
+    if (cudaMemsetAsync(ws, 0, (size_t)(nO + 1) * 4, st) != cudaSuccess) return QUAFF_ERR_CUDA;
+    const int grid = max(1, min(ceil_div(M, 16), sm_count() * 2));
+    momentum_kernel<<<grid, 256, 0, st>>>(X, ldx, M, O_idx, nO, wmax_O, gamma, s_O, colmax_O_opt, beta_O_opt,
+                                          reinterpret_cast<unsigned int*>(ws));
+    return launch_status();
+}
+
+extern "C" quaff_status_t quaff_requant_weight_rows(const quaff_bf16* W_O, int64_t ldwo, int nO, int N, const float* s_O,
+                                                    int8_t* wq_O, int64_t ldwq, int nOp, float* dw_O,
+                                                    quaff_stream_t stream) {
+    QUAFF_RETURN_IF(nO < 0 || N <= 0 || nOp < nO || !dw_O, QUAFF_ERR_INVALID_ARG);
+    QUAFF_RETURN_IF(nO > 0 && (!W_O || !s_O || ldwo < N), QUAFF_ERR_INVALID_ARG);
+    QUAFF_RETURN_IF(nOp > 0 && (!wq_O || ldwq < nOp), QUAFF_ERR_INVALID_ARG);
+    QUAFF_RETURN_IF(nOp % 16, QUAFF_ERR_UNSUPPORTED_SHAPE);
+    QUAFF_RETURN_IF(nOp > 0 && (!aligned16(wq_O) || (ldwq % 16)), QUAFF_ERR_ALIGNMENT);
+    requant_rows_kernel<<<ceil_div(N, 64), 64, 0, (cudaStream_t)stream>>>(W_O, ldwo, nO, N, s_O, wq_O, ldwq, nOp, dw_O);
+    return launch_status();
+}
+
+extern "C" quaff_status_t quaff_prepare_weight(const quaff_bf16* Wt, int64_t ldw, int N, int K, const int32_t* O_idx,
+                                               int nO, int8_t* Wq, int64_t ldwq, float* dW, quaff_bf16* W_O,
+                                               int64_t ldwo, float* wmax_O, quaff_stream_t stream) {
+    QUAFF_RETURN_IF(!Wt || !Wq || !dW || N <= 0 || K <= 0 || ldw < K || ldwq < K, QUAFF_ERR_INVALID_ARG);
+    QUAFF_RETURN_IF(!valid_outlier_args(O_idx, nO, K), QUAFF_ERR_INVALID_ARG);
+    QUAFF_RETURN_IF(nO > 0 && (!W_O || !wmax_O || ldwo < N), QUAFF_ERR_INVALID_ARG);
+    QUAFF_RETURN_IF(!aligned16(Wt) || !aligned16(Wq) || (ldw % 8) || (ldwq % 16), QUAFF_ERR_ALIGNMENT);
+    cudaStream_t st = (cudaStream_t)stream;
+    // Eq. 1 per output channel of W = per row of the [N][K] layout: the per-token kernel without outliers
+    quaff_status_t rc = quant_act_dispatch(Wt, ldw, N, K, nullptr, 0, nullptr, Wq, ldwq, nullptr, 0, 0, dW, st);
+    if (rc != QUAFF_OK) return rc;
+    if (nO > 0) {
+        gather_outlier_rows_kernel<<<nO, 256, 0, st>>>(Wt, ldw, N, O_idx, W_O, ldwo, wmax_O);
+        rc = launch_status();
+    }
+    return rc;
+}

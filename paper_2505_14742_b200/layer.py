@@ -1,0 +1,87 @@
+"""One Quaff linear layer on the device: owns the buffers and chains the C-ABI calls of a step.
+
+No arithmetic happens here; every step of the path runs in the library's kernels:
+    forward : quaff_momentum_update -> quaff_requant_weight_rows -> quaff_quant_act -> quaff_qlinear_fwd
+    backward: quaff_qlinear_bwd
+"""
+from __future__ import annotations
+
+from typing import Optional
+
+import torch
+
+from . import binding as Q
+
+
+def pad32(n: int) -> int:
+    return (n + 31) // 32 * 32
+
+
+class QuaffLinear:
+    """Frozen INT8 weight + outlier rows + LoRA adapters + the momentum scale state s_O."""
+
+    def __init__(self, Wt: torch.Tensor, O_idx: Optional[torch.Tensor], A: Optional[torch.Tensor],
+                 B: Optional[torch.Tensor], lora_scale: float, gamma: float, max_tokens: int,
+                 y_dtype: torch.dtype = torch.bfloat16, debug_acc: bool = False):
+        dev = Wt.device
+        self.N, self.K = Wt.shape
+        self.nO = 0 if O_idx is None else int(O_idx.numel())
+        self.nOp = pad32(self.nO)
+        self.r = 0 if A is None else int(A.shape[1])
+        self.M = max_tokens
+        self.gamma = float(gamma)
+        self.lora_scale = float(lora_scale)
+        self.O_idx = O_idx
+        self.A, self.B = A, B
+        N, K, M, nO, nOp, r = self.N, self.K, self.M, self.nO, self.nOp, self.r
+        i8, f32, bf = torch.int8, torch.float32, torch.bfloat16
+        self.Wq = torch.empty((N, K), dtype=i8, device=dev)
+        self.dW = torch.empty(N, dtype=f32, device=dev)
+        self.W_O = torch.empty((nO, N), dtype=bf, device=dev) if nO else None
+        self.wmax_O = torch.empty(nO, dtype=f32, device=dev) if nO else None
+        self.s_O = torch.ones(nO, dtype=f32, device=dev) if nO else None
+        self.colmax_O = torch.empty(nO, dtype=f32, device=dev) if nO else None
+        self.beta_O = torch.empty(nO, dtype=f32, device=dev) if nO else None
+        self.wq_O = torch.empty((N, nOp), dtype=i8, device=dev) if nOp else None
+        self.dw_O = torch.empty(N, dtype=f32, device=dev)
+        self.Xq = torch.empty((M, K), dtype=i8, device=dev)
+        self.xq_O = torch.empty((M, nOp), dtype=i8, device=dev) if nOp else None
+        self.dx = torch.empty(M, dtype=f32, device=dev)
+        self.T = torch.empty((M, r), dtype=bf, device=dev) if r else None
+        self.Y = torch.empty((M, N), dtype=y_dtype, device=dev)
+        self.dX = torch.empty((M, K), dtype=bf, device=dev)
+        self.dA = torch.zeros((K, r), dtype=f32, device=dev) if r else None
+        self.dB = torch.zeros((r, N), dtype=f32, device=dev) if r else None
+        self.acc_main = torch.empty((M, N), dtype=torch.int32, device=dev) if debug_acc else None
+        self.acc_out = torch.empty((M, N), dtype=torch.int32, device=dev) if debug_acc else None
+        self.status = torch.zeros(4, dtype=torch.int32, device=dev)
+        ws_bytes = max(Q.workspace_bytes(Q.QUAFF_WS_MOMENTUM, M, K, N, nOp, r),
+                       Q.workspace_bytes(Q.QUAFF_WS_FWD, M, K, N, nOp, r),
+                       Q.workspace_bytes(Q.QUAFF_WS_BWD, M, K, N, nOp, r), 256)
+        self.ws = torch.empty(ws_bytes, dtype=torch.uint8, device=dev)
+        Q.quaff_prepare_weight(Wt, O_idx, self.Wq, self.dW, self.W_O, self.wmax_O)
+
+    def forward(self, X: torch.Tensor) -> torch.Tensor:
+        M = X.shape[0]
+        assert M <= self.M and X.shape[1] == self.K
+        Xq, dx, Y = self.Xq[:M], self.dx[:M], self.Y[:M]
+        xq_O = self.xq_O[:M] if self.nOp else None
+        T = self.T[:M] if self.r else None
+        if self.nO:
+            Q.quaff_momentum_update(X, self.O_idx, self.wmax_O, self.gamma, self.s_O, self.ws, self.colmax_O, self.beta_O)
+            Q.quaff_requant_weight_rows(self.W_O, self.s_O, self.wq_O, self.dw_O)
+        Q.quaff_quant_act(X, self.O_idx, self.s_O, Xq, xq_O, dx)
+        Q.quaff_qlinear_fwd(Xq, xq_O, dx, self.Wq, self.dW, self.wq_O, self.dw_O, X, self.A, self.B, self.lora_scale,
+                            T, Y, self.ws,
+                            self.acc_main[:M] if self.acc_main is not None else None,
+                            self.acc_out[:M] if self.acc_out is not None else None, self.status)
+        self._X = X
+        return Y
+
+    def backward(self, dY: torch.Tensor, accumulate: bool = False, need_dX: bool = True):
+        M = dY.shape[0]
+        dX = self.dX[:M] if need_dX else None
+        T = self.T[:M] if self.r else None
+        Q.quaff_qlinear_bwd(dY, self.Wq, self.dW, self.wq_O, self.dw_O, self.O_idx, self.s_O, self._X, T, self.A, self.B,
+                            self.lora_scale, dX, self.dA, self.dB, accumulate, self.ws, self.status)
+        return dX, self.dA, self.dB

@@ -1,0 +1,271 @@
+"""GPU parity: every C-ABI entry point against the CPU oracle on the same seeded inputs.
+INT8 codes, INT32 accumulators, step sizes and scale factors must be bit-exact; dequantized
+outputs and gradients within TOL_F32 (fp32 epilogue, no LoRA) or TOL_BF16 (bf16 / LoRA)."""
+import numpy as np
+import pytest
+
+import oracle
+from paper_2505_14742_b200 import synth
+from util import (TOL_BF16, TOL_F32, bf, bf16_ulp_diff, dev, dev_bf16, f32, host, host_bits, max_rel_err)
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def Q():
+    import torch
+    from paper_2505_14742_b200 import binding, build
+    build.build_library()
+    binding.lib()
+    assert torch.cuda.is_available()
+    return binding
+
+
+def _mk_inputs(seed, M, K, N, nO, r, b_std=0.02, zero_rows=()):
+    rng = np.random.default_rng(seed)
+    O = np.sort(rng.permutation(K)[:nO]).astype(np.int32)
+    x = rng.standard_normal((M, K)).astype(np.float32)
+    if nO:
+        x[:, O] *= rng.uniform(20, 100, nO).astype(np.float32)
+    for z in zero_rows:
+        x[z] = 0
+    X = bf(x)
+    Wt = bf(rng.standard_normal((N, K)).astype(np.float32) * 0.02)
+    A = bf(rng.standard_normal((K, r)).astype(np.float32) * 0.02) if r else None
+    B = bf(rng.standard_normal((r, N)).astype(np.float32) * b_std) if r else None
+    dY = bf(rng.standard_normal((M, N)).astype(np.float32) * 1e-2)
+    return O, X, Wt, A, B, dY
+
+
+def _pad32(n):
+    return (n + 31) // 32 * 32
+
+
+# ----------------------------------------------------------------------------- S2 quant_act
+@pytest.mark.parametrize("M,K,nO", [(1, 16, 0), (37, 136, 5), (64, 100, 3), (300, 3072, 32), (33, 11008, 55),
+                                    (5, 20000, 200), (256, 512, 8)])
+def test_quant_act_bit_exact(Q, M, K, nO):
+    import torch
+    O, X, _, _, _, _ = _mk_inputs(100 + M, M, K, 8, nO, 0, zero_rows=(0,) if M > 3 else ())
+    rng = np.random.default_rng(7)
+    s = (1.0 + 20.0 * rng.random(nO)).astype(np.float32)
+    nOp = _pad32(nO)
+    ldx = (K + 7) // 8 * 8 + 8
+    ldxq = (K + 15) // 16 * 16 + 16
+    Xd = torch.zeros((M, ldx), dtype=torch.bfloat16, device="cuda")
+    Xd[:, :K] = dev_bf16(X)
+    Xq = torch.full((M, ldxq), -128, dtype=torch.int8, device="cuda")
+    xqo = torch.full((M, nOp + 16), -128, dtype=torch.int8, device="cuda") if nOp else None
+    dx = torch.full((M,), -1.0, dtype=torch.float32, device="cuda")
+    Q.quaff_quant_act(Xd[:, :K], dev(O) if nO else None, dev(s) if nO else None, Xq[:, :K],
+                      xqo[:, :nOp] if nOp else None, dx)
+    torch.cuda.synchronize()
+    oXq, oxqo, odx = oracle.quant_act(X, O, s, nOp)
+    assert np.array_equal(host(Xq[:, :K]), oXq)
+    assert (host(Xq[:, K:]) == -128).all(), "wrote outside the row"
+    assert np.array_equal(host(dx), odx)
+    if nOp:
+        assert np.array_equal(host(xqo[:, :nOp]), oxqo)
+        assert (host(xqo[:, nOp:]) == -128).all()
+
+
+# ----------------------------------------------------------------------------- S1 momentum
+@pytest.mark.parametrize("M,K,nO,gamma", [(1, 64, 1, 0.5), (100, 256, 7, 0.9), (2048, 3072, 32, 0.2), (513, 1024, 100, 0.0)])
+def test_momentum_update_bit_exact(Q, M, K, nO, gamma):
+    import torch
+    O, X, Wt, _, _, _ = _mk_inputs(200 + M, M, K, 16, nO, 0)
+    _, _, _, wmax = oracle.prepare_weight(Wt, O)
+    wmax[0] = 0.0 if nO > 1 else wmax[0]      # a zero weight row must give beta = 1
+    s_host = np.ones(nO, np.float32)
+    s_dev = dev(s_host.copy())
+    cm = torch.empty(nO, dtype=torch.float32, device="cuda")
+    be = torch.empty(nO, dtype=torch.float32, device="cuda")
+    ws = torch.empty(Q.workspace_bytes(Q.QUAFF_WS_MOMENTUM, M, K, 16, _pad32(nO), 0), dtype=torch.uint8, device="cuda")
+    Xd = dev_bf16(X)
+    for step in range(3):
+        Q.quaff_momentum_update(Xd, dev(O), dev(wmax), gamma, s_dev, ws, cm, be)
+        torch.cuda.synchronize()
+        s_host, ocm, obe = oracle.momentum_update(X, O, wmax, gamma, s_host)
+        assert np.array_equal(host(cm), ocm)
+        assert np.array_equal(host(be), obe)
+        assert np.array_equal(host(s_dev), s_host)
+
+
+# ----------------------------------------------------------------------------- S3 requant + preprocessing
+@pytest.mark.parametrize("nO,N", [(1, 16), (5, 136), (32, 3072), (100, 1000)])
+def test_requant_weight_rows_bit_exact(Q, nO, N):
+    import torch
+    rng = np.random.default_rng(300 + nO)
+    W_O = bf(rng.standard_normal((nO, N)).astype(np.float32) * 0.02)
+    s = (1.0 + 10.0 * rng.random(nO)).astype(np.float32)
+    s[0] = 1.0
+    nOp = _pad32(nO)
+    wq = torch.full((N, nOp), -128, dtype=torch.int8, device="cuda")
+    dw = torch.empty(N, dtype=torch.float32, device="cuda")
+    Q.quaff_requant_weight_rows(dev_bf16(W_O), dev(s), wq, dw)
+    torch.cuda.synchronize()
+    owq, odw = oracle.requant_weight_rows(W_O, s, nOp)
+    assert np.array_equal(host(wq), owq)
+    assert np.array_equal(host(dw), odw)
+
+
+@pytest.mark.parametrize("N,K,nO", [(16, 32, 0), (136, 200, 5), (1000, 3072, 32)])
+def test_prepare_weight_bit_exact(Q, N, K, nO):
+    import torch
+    O, _, Wt, _, _, _ = _mk_inputs(400 + N, 1, K, N, nO, 0)
+    ldq = (K + 15) // 16 * 16
+    Wq = torch.empty((N, ldq), dtype=torch.int8, device="cuda")
+    dW = torch.empty(N, dtype=torch.float32, device="cuda")
+    W_O = torch.empty((nO, N), dtype=torch.bfloat16, device="cuda") if nO else None
+    wmax = torch.empty(nO, dtype=torch.float32, device="cuda") if nO else None
+    Q.quaff_prepare_weight(dev_bf16(Wt), dev(O) if nO else None, Wq[:, :K], dW, W_O, wmax)
+    torch.cuda.synchronize()
+    oWq, odW, oW_O, owmax = oracle.prepare_weight(Wt, O)
+    assert np.array_equal(host(Wq[:, :K]), oWq)
+    assert np.array_equal(host(dW), odW)
+    if nO:
+        assert np.array_equal(host_bits(W_O), oW_O)
+        assert np.array_equal(host(wmax), owmax)
+
+
+# ----------------------------------------------------------------------------- S4 + S5 forward
+def _oracle_state(O, X, Wt, gamma=0.0):
+    Wq, dW, W_O, wmax = oracle.prepare_weight(Wt, O)
+    nO = len(O)
+    s, _, _ = oracle.momentum_update(X, O, wmax, gamma, np.ones(nO, np.float32))
+    nOp = _pad32(nO)
+    Xq, xqo, dx = oracle.quant_act(X, O, s, nOp)
+    wq, dw = oracle.requant_weight_rows(W_O, s, nOp)
+    return Wq, dW, W_O, wmax, s, Xq, xqo, dx, wq, dw
+
+
+FWD_SHAPES = [(1, 128, 16, 0, 0), (128, 128, 128, 32, 16), (200, 320, 136, 5, 8), (256, 512, 512, 8, 8),
+              (384, 1024, 640, 40, 16), (130, 2048, 300, 33, 64), (257, 384, 129, 0, 32), (100, 256, 256, 3, 0)]
+
+
+@pytest.mark.parametrize("M,K,N,nO,r", FWD_SHAPES)
+@pytest.mark.parametrize("y_f32", [True, False])
+def test_qlinear_fwd(Q, M, K, N, nO, r, y_f32):
+    import torch
+    O, X, Wt, A, B, _ = _mk_inputs(500 + M + N, M, K, N, nO, r)
+    Wq, dW, W_O, wmax, s, Xq, xqo, dx, wq, dw = _oracle_state(O, X, Wt)
+    nOp = _pad32(nO)
+    Y = torch.full((M, N), float("nan"), dtype=torch.float32 if y_f32 else torch.bfloat16, device="cuda")
+    a1 = torch.full((M, N), -7, dtype=torch.int32, device="cuda")
+    a2 = torch.full((M, N), -7, dtype=torch.int32, device="cuda")
+    T = torch.empty((M, r), dtype=torch.bfloat16, device="cuda") if r else None
+    st = torch.zeros(4, dtype=torch.int32, device="cuda")
+    ws = torch.empty(max(256, Q.workspace_bytes(Q.QUAFF_WS_FWD, M, K, N, nOp, r)), dtype=torch.uint8, device="cuda")
+    Q.quaff_qlinear_fwd(dev(Xq), dev(xqo) if nOp else None, dev(dx), dev(Wq), dev(dW), dev(wq) if nOp else None,
+                        dev(dw), dev_bf16(X), dev_bf16(A) if r else None, dev_bf16(B) if r else None, 0.5,
+                        T, Y, ws, a1, a2, st)
+    torch.cuda.synchronize()
+    assert host(st)[0] == 0, "device-side wait timed out"
+    oY, oT, o1, o2 = oracle.qlinear_fwd(Xq, xqo, dx, Wq, dW, wq, dw, X, A, B, 0.5)
+    assert np.array_equal(host(a1), o1), "main INT32 accumulator"
+    assert np.array_equal(host(a2), o2), "outlier INT32 accumulator"
+    if r:
+        assert bf16_ulp_diff(host_bits(T), oT).max() <= 1.0
+    tol = TOL_F32 if (y_f32 and r == 0) else TOL_BF16
+    err = max_rel_err(host(Y), oY)
+    assert err <= tol, f"max rel err {err:.3e}"
+
+
+# ----------------------------------------------------------------------------- S6-S8 backward
+BWD_SHAPES = [(1, 128, 64, 0, 0), (128, 128, 128, 32, 16), (200, 320, 136, 5, 8), (256, 512, 512, 8, 8),
+              (384, 640, 1024, 40, 16), (130, 300 // 4 * 4 + 4, 2048, 33, 64), (100, 256, 256, 3, 0)]
+
+
+@pytest.mark.parametrize("M,K,N,nO,r", BWD_SHAPES)
+def test_qlinear_bwd(Q, M, K, N, nO, r):
+    import torch
+    K = (K + 7) // 8 * 8
+    O, X, Wt, A, B, dY = _mk_inputs(600 + M + N, M, K, N, nO, r)
+    Wq, dW, W_O, wmax, s, Xq, xqo, dx, wq, dw = _oracle_state(O, X, Wt)
+    nOp = _pad32(nO)
+    oY, oT, _, _ = oracle.qlinear_fwd(Xq, xqo, dx, Wq, dW, wq, dw, X, A, B, 0.5)
+    odX, odA, odB, oG = oracle.qlinear_bwd(dY, Wq, dW, wq, dw, O, s, X, oT, A, B, 0.5)
+    dX = torch.full((M, K), float("nan"), dtype=torch.bfloat16, device="cuda")
+    dA = torch.full((K, r), 1.0, dtype=torch.float32, device="cuda") if r else None
+    dB = torch.full((r, N), 1.0, dtype=torch.float32, device="cuda") if r else None
+    st = torch.zeros(4, dtype=torch.int32, device="cuda")
+    ws = torch.empty(Q.workspace_bytes(Q.QUAFF_WS_BWD, M, K, N, nOp, r), dtype=torch.uint8, device="cuda")
+    args = (dev_bf16(dY), dev(Wq), dev(dW), dev(wq) if nOp else None, dev(dw), dev(O) if nO else None,
+            dev(s) if nO else None, dev_bf16(X), dev_bf16(oT) if r else None, dev_bf16(A) if r else None,
+            dev_bf16(B) if r else None, 0.5, dX, dA, dB)
+    Q.quaff_qlinear_bwd(*args, False, ws, st)
+    torch.cuda.synchronize()
+    assert host(st)[0] == 0
+    err = max_rel_err(host(dX), odX)
+    assert err <= TOL_BF16, f"dX max rel err {err:.3e}"
+    if nO:
+        err_o = max_rel_err(host(dX)[:, O], odX[:, O])
+        assert err_o <= TOL_BF16, f"dX outlier columns max rel err {err_o:.3e}"
+    if r:
+        assert max_rel_err(host(dA), odA) <= TOL_BF16
+        assert max_rel_err(host(dB), odB) <= TOL_BF16
+        # gradient accumulation: a second call with accumulate adds the same gradients again
+        Q.quaff_qlinear_bwd(*args, True, ws, st)
+        torch.cuda.synchronize()
+        assert max_rel_err(host(dA), 2 * odA) <= TOL_BF16
+        assert max_rel_err(host(dB), 2 * odB) <= TOL_BF16
+
+
+# ----------------------------------------------------------------------------- whole path, several steps
+def test_tiny_workload_all_steps(Q):
+    """Configuration 'tiny': 10 iterations of forward + backward with drifting outliers and the
+    momentum state carried across steps; everything is compared at every step.  LoRA B is non-zero
+    so that the LoRA branch contributes."""
+    import torch
+    from paper_2505_14742_b200.layer import QuaffLinear
+    wl = synth.WORKLOADS["tiny"]
+    lin = synth.layer_inputs(wl, 0, b_std=0.02)
+    sp = lin.spec
+    scale = wl.lora_alpha / sp.r
+    layer = QuaffLinear(dev_bf16(lin.W), dev(lin.O_idx), dev_bf16(lin.A), dev_bf16(lin.B), scale, wl.gamma, wl.M,
+                        y_dtype=torch.bfloat16, debug_acc=True)
+    Wq, dW, W_O, wmax = oracle.prepare_weight(lin.W, lin.O_idx)
+    s = np.ones(sp.nO, np.float32)
+    nOp = _pad32(sp.nO)
+    for step in range(wl.steps):
+        X, dY = synth.step_inputs(wl, 0, step, lin)
+        Y = layer.forward(dev_bf16(X))
+        dX, dA, dB = layer.backward(dev_bf16(dY))
+        torch.cuda.synchronize()
+        assert host(layer.status)[0] == 0
+        s, _, _ = oracle.momentum_update(X, lin.O_idx, wmax, wl.gamma, s)
+        Xq, xqo, dx = oracle.quant_act(X, lin.O_idx, s, nOp)
+        wq, dw = oracle.requant_weight_rows(W_O, s, nOp)
+        oY, oT, o1, o2 = oracle.qlinear_fwd(Xq, xqo, dx, Wq, dW, wq, dw, X, lin.A, lin.B, scale)
+        odX, odA, odB, _ = oracle.qlinear_bwd(dY, Wq, dW, wq, dw, lin.O_idx, s, X, oT, lin.A, lin.B, scale)
+        assert np.array_equal(host(layer.s_O), s), f"s_O at step {step}"
+        assert np.array_equal(host(layer.Xq), Xq) and np.array_equal(host(layer.xq_O), xqo)
+        assert np.array_equal(host(layer.dx), dx)
+        assert np.array_equal(host(layer.wq_O), wq) and np.array_equal(host(layer.dw_O), dw)
+        assert np.array_equal(host(layer.acc_main), o1) and np.array_equal(host(layer.acc_out), o2)
+        assert max_rel_err(host(Y), oY) <= TOL_BF16
+        assert max_rel_err(host(dX), odX) <= TOL_BF16
+        assert max_rel_err(host(dA), odA) <= TOL_BF16 and max_rel_err(host(dB), odB) <= TOL_BF16
+
+
+# ----------------------------------------------------------------------------- host-side validation (no launch)
+def test_argument_validation(Q):
+    import torch
+    M, K, N = 32, 64, 48
+    X = torch.zeros((M, K), dtype=torch.bfloat16, device="cuda")
+    Xq = torch.zeros((M, K), dtype=torch.int8, device="cuda")
+    dx = torch.zeros(M, dtype=torch.float32, device="cuda")
+    with pytest.raises(Q.QuaffError) as e:
+        Q.quaff_quant_act(X[:, 1:], None, None, Xq[:, 1:], None, dx)          # misaligned base
+    assert e.value.code == Q.QUAFF_ERR_ALIGNMENT
+    O = torch.arange(70, dtype=torch.int32, device="cuda")
+    with pytest.raises(Q.QuaffError) as e:
+        Q.quaff_quant_act(X, O, dx, Xq, torch.zeros((M, 96), dtype=torch.int8, device="cuda"), dx)   # nO > K
+    assert e.value.code == Q.QUAFF_ERR_INVALID_ARG
+    with pytest.raises(Q.QuaffError) as e:
+        Q.quaff_momentum_update(X, O[:4], dx, 1.5, dx, torch.zeros(256, dtype=torch.uint8, device="cuda"))  # gamma
+    assert e.value.code == Q.QUAFF_ERR_INVALID_ARG
+    with pytest.raises(Q.QuaffError) as e:
+        Q.quaff_momentum_update(X, O[:4], dx, 0.5, dx, torch.zeros(8, dtype=torch.uint8, device="cuda"))
+    assert e.value.code == Q.QUAFF_ERR_WORKSPACE_TOO_SMALL
+    torch.cuda.synchronize()
