@@ -46,14 +46,5 @@ def max_rel_err(got, ref):
     return float(np.max(np.abs(got - ref) / np.maximum(np.abs(ref), floor))) if ref.size else 0.0
 
 
-def bf16_ulp_diff(a_bits, b_bits):
-    """|a - b| in units of bf16 ulps of the larger magnitude (same-sign finite values)."""
-    a = f32(a_bits).astype(np.float64)
-    b = f32(b_bits).astype(np.float64)
-    mag = np.maximum(np.abs(a), np.abs(b))
-    ulp = 2.0 ** (np.floor(np.log2(np.maximum(mag, 1e-300))) - 7)
-    return np.abs(a - b) / ulp
-
-
 TOL_F32 = 1e-3   # fp32 epilogue, no bf16 rounding anywhere on the path
 TOL_BF16 = 2e-2  # bf16 output and / or the bf16 LoRA branch
