@@ -1,0 +1,351 @@
+#!/usr/bin/env python
+"""Benchmark of the Quaff quantized linear layer hot path (forward + backward) on B200.
+
+A step is one pass of the whole path - momentum scale update, outlier weight-row re-quantization,
+activation scaling + quantization, INT8 forward GEMM with fused dequantization and LoRA, and the
+backward (grad-input through the dequantized INT8 weight, LoRA gradients) - over one batch of
+synthetic tokens through every linear layer of the workload.  Default workload: Phi-3-mini attention
+projections (2048 tokens; fused qkv 3072->9216 and o_proj 3072->3072; 32 outlier channels; LoRA r=16).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference]
+
+Prints ONE JSON line (rank 0).  `--impl reference` times the CPU oracle on a bounded token sample.
+"""
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2505_14742_b200 import synth  # noqa: E402
+
+METRIC = "qlinear fwd+bwd tokens/s"
+UNIT = "tokens/s"
+REPLICAS = 3  # rotating buffer sets, so that every step starts from cold HBM data
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        d = json.load(open(path))
+        return {"hbm_gbs": d["hbm_gbs"], "bf16_tflops": d["bf16_tflops"],
+                "bf16_tflops_sustained": d.get("bf16_tflops_sustained", d["bf16_tflops"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index = index
+        self.rows = []
+        self._stop = threading.Event()
+        self._t = threading.Thread(target=self._run, daemon=True)
+
+    def _run(self):
+        while not self._stop.is_set():
+            try:
+                out = subprocess.run(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-i", str(self.index)],
+                                     capture_output=True, text=True, timeout=5).stdout.strip()
+                if out:
+                    self.rows.append([c.strip() for c in out.split(",")])
+            except Exception:
+                pass
+            self._stop.wait(0.1)
+
+    def __enter__(self):
+        self._t.start()
+        return self
+
+    def __exit__(self, *a):
+        self._stop.set()
+        self._t.join(timeout=6)
+
+    def summary(self):
+        sm, mx, reasons = [], [], set()
+        for r in self.rows:
+            try:
+                sm.append(float(r[0])); mx.append(float(r[1]))
+            except Exception:
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), r[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def layer_ops(M, sp, nOp):
+    """Algorithmic work of one layer-step: INT8 ops of the forward GEMMs, bf16 flops of the grad-input GEMM."""
+    fwd_int8 = 2.0 * M * sp.N * (sp.K + nOp)
+    fwd_lora = 2.0 * M * sp.N * sp.r
+    bwd_bf16 = 2.0 * M * sp.N * sp.K + 2.0 * M * sp.N * 2 * nOp + 2.0 * M * sp.K * sp.r
+    return fwd_int8, fwd_lora, bwd_bf16
+
+
+# --------------------------------------------------------------------------------------- CPU oracle legs
+def oracle_sample_step(wl, sample_tokens, lins, state):
+    """One fwd+bwd of the oracle over `sample_tokens` tokens through every layer; returns seconds."""
+    import oracle
+    t0 = time.perf_counter()
+    for li, lin in enumerate(lins):
+        sp = lin.spec
+        st = state[li]
+        X, dY = st["X"], st["dY"]
+        nOp = synth.pad_to(sp.nO, 32)
+        scale = wl.lora_alpha / sp.r
+        st["s"], _, _ = oracle.momentum_update(X, lin.O_idx, st["wmax"], wl.gamma, st["s"])
+        wq, dw = oracle.requant_weight_rows(st["W_O"], st["s"], nOp)
+        Xq, xqo, dx = oracle.quant_act(X, lin.O_idx, st["s"], nOp)
+        Y, T, _, _ = oracle.qlinear_fwd(Xq, xqo, dx, st["Wq"], st["dW"], wq, dw, X, lin.A, lin.B, scale)
+        oracle.qlinear_bwd(dY, st["Wq"], st["dW"], wq, dw, lin.O_idx, st["s"], X, T, lin.A, lin.B, scale)
+    return time.perf_counter() - t0
+
+
+def oracle_setup(wl, sample_tokens):
+    import oracle
+    oracle.build()
+    lins = [synth.layer_inputs(wl, li, b_std=0.02) for li in range(len(wl.layers))]
+    state = []
+    for li, lin in enumerate(lins):
+        Wq, dW, W_O, wmax = oracle.prepare_weight(lin.W, lin.O_idx)
+        X, dY = synth.step_inputs(wl, li, 0, lin)
+        state.append({"Wq": Wq, "dW": dW, "W_O": W_O, "wmax": wmax, "s": np.ones(lin.spec.nO, np.float32),
+                      "X": np.ascontiguousarray(X[:sample_tokens]), "dY": np.ascontiguousarray(dY[:sample_tokens])})
+    return lins, state
+
+
+def cpu_baseline(wl, sample_tokens=16, reps=1):
+    import oracle
+    lins, state = oracle_setup(wl, sample_tokens)
+    best = min(oracle_sample_step(wl, sample_tokens, lins, state) for _ in range(reps))
+    return {"value": sample_tokens / best, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+            "sample": f"{sample_tokens} of {wl.M} tokens through all {len(wl.layers)} layers, fwd+bwd, {best:.2f} s"}
+
+
+def run_reference(args, wl):
+    """--impl reference: the CPU oracle, as it stands, on the host cores (rank 0 only)."""
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    import oracle
+    sample = args.sample_tokens
+    lins, state = oracle_setup(wl, sample)
+    for _ in range(args.warmup):
+        oracle_sample_step(wl, sample, lins, state)
+    times = [oracle_sample_step(wl, sample, lins, state) for _ in range(args.steps)]
+    ms = 1e3 * float(np.mean(times))
+    value = sample / (ms / 1e3)
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "int8 forward (int64 accumulate), f64 backward", "data": "synthetic",
+            "config": {"workload": wl.name, "tokens": wl.M, "sample_tokens_per_step": sample,
+                       "layers": [f"{l.name} {l.K}->{l.N}" for l in wl.layers]},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+                             "sample": f"{sample} of {wl.M} tokens per step through all layers, fwd+bwd"},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+# --------------------------------------------------------------------------------------- GPU arm
+def run_gpu(args, wl):
+    import torch
+    import torch.distributed as dist
+    from paper_2505_14742_b200 import binding as Q, build
+    from paper_2505_14742_b200.layer import QuaffLinear
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    if rank == 0:
+        build.build_library()
+    if world > 1:
+        dist.barrier()
+    Q.lib()  # raises when the CUDA library is missing: there is no fallback path
+
+    def to_bf16(bits):
+        return torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).cuda().view(torch.bfloat16)
+
+    # Each rank owns its own batch of tokens (weak scaling, no data-path collective): rank-specific seed offset.
+    M = wl.M
+    nl = len(wl.layers)
+    lins = [synth.layer_inputs(wl, li, b_std=0.02) for li in range(nl)]
+    sets = []  # REPLICAS x layers
+    host_in = []
+    for rep in range(REPLICAS):
+        layers, xs, dys, hx, hdy = [], [], [], [], []
+        for li, lin in enumerate(lins):
+            sp = lin.spec
+            layer = QuaffLinear(to_bf16(lin.W), torch.from_numpy(lin.O_idx).cuda(), to_bf16(lin.A), to_bf16(lin.B),
+                                wl.lora_alpha / sp.r, wl.gamma, M)
+            X, dY = synth.step_inputs(wl, li, rep + 1000 * rank, lin)
+            layers.append(layer)
+            xs.append(to_bf16(X)); dys.append(to_bf16(dY))
+            hx.append(torch.from_numpy(X.view(np.int16)).pin_memory()); hdy.append(torch.from_numpy(dY.view(np.int16)).pin_memory())
+        sets.append((layers, xs, dys))
+        host_in.append((hx, hdy))
+    torch.cuda.synchronize()
+
+    def step(i, timing=None):
+        layers, xs, dys = sets[i % REPLICAS]
+        for li in range(nl):
+            if timing is not None:
+                ev = timing[li][i]
+                Q.quaff_debug_time_gemm(0, ev[0], ev[1])
+                Q.quaff_debug_time_gemm(1, ev[2], ev[3])
+            layers[li].forward(xs[li])
+            layers[li].backward(dys[li])
+
+    def sync_all():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    for i in range(args.warmup):
+        step(i)
+    sync_all()
+    for layers, _, _ in sets:
+        for l in layers:
+            assert int(l.status[0].item()) == 0, "device-side wait timed out"
+
+    # ---- device-resident timed region
+    # torch creates the CUDA event lazily at its first record(): materialise every handle before the timed region
+    timing = [[[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(args.steps)] for _ in range(nl)]
+    for per_layer_events in timing:
+        for evs in per_layer_events:
+            for e in evs:
+                e.record()
+    launches0 = Q.quaff_debug_launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with ClockSampler(local) as clocks:
+        sync_all()
+        e0.record()
+        for i in range(args.steps):
+            step(i, timing)
+        e1.record()
+        sync_all()
+    launches = Q.quaff_debug_launch_count() - launches0
+    ms_total = e0.elapsed_time(e1)
+    t = torch.tensor([ms_total], dtype=torch.float64, device="cuda")
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms_per_step = float(t.item()) / args.steps
+
+    # ---- end to end: host buffers in, host buffers out, copies inside the timed region
+    h_out = []
+    for li, lin in enumerate(lins):
+        sp = lin.spec
+        h_out.append((torch.empty((M, sp.N), dtype=torch.bfloat16).pin_memory(), torch.empty((M, sp.K), dtype=torch.bfloat16).pin_memory()))
+    h2d = sum(M * (sp.K + sp.N) * 2 for sp in wl.layers)
+    d2h = sum(M * (sp.N + sp.K) * 2 for sp in wl.layers)
+
+    def step_e2e(i):
+        layers, xs, dys = sets[i % REPLICAS]
+        hx, hdy = host_in[i % REPLICAS]
+        for li in range(nl):
+            xs[li].view(torch.int16).copy_(hx[li], non_blocking=True)
+            dys[li].view(torch.int16).copy_(hdy[li], non_blocking=True)
+            Y = layers[li].forward(xs[li])
+            dX, _, _ = layers[li].backward(dys[li])
+            h_out[li][0].copy_(Y, non_blocking=True)
+            h_out[li][1].copy_(dX, non_blocking=True)
+
+    e2e_steps = max(3, min(args.steps, 20))
+    for i in range(2):
+        step_e2e(i)
+    sync_all()
+    e0.record()
+    for i in range(e2e_steps):
+        step_e2e(i)
+    e1.record()
+    sync_all()
+    t2 = torch.tensor([e0.elapsed_time(e1)], dtype=torch.float64, device="cuda")
+    if world > 1:
+        dist.all_reduce(t2, op=dist.ReduceOp.MAX)
+    e2e_ms = float(t2.item()) / e2e_steps
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    # ---- per-kernel figures and the roofline of the dominant kernel
+    peaks = load_peaks()
+    per_layer = []
+    dominant = None
+    for li, sp in enumerate(wl.layers):
+        nOp = synth.pad_to(sp.nO, 32)
+        f_ms = float(np.mean([ev[0].elapsed_time(ev[1]) for ev in timing[li]]))
+        b_ms = float(np.mean([ev[2].elapsed_time(ev[3]) for ev in timing[li]]))
+        fwd_int8, fwd_lora, bwd_bf16 = layer_ops(M, sp, nOp)
+        entry = {"layer": sp.name, "K": sp.K, "N": sp.N, "nO": sp.nO, "r": sp.r,
+                 "fwd_gemm_ms": f_ms, "fwd_int8_tops": fwd_int8 / (f_ms * 1e-3) / 1e12,
+                 "fwd_pct_of_int8_nominal_4500": 100.0 * fwd_int8 / (f_ms * 1e-3) / 4.5e15,
+                 "bwd_gemm_ms": b_ms, "bwd_bf16_tflops": bwd_bf16 / (b_ms * 1e-3) / 1e12,
+                 "bwd_pct_of_bf16_nominal_2250": 100.0 * bwd_bf16 / (b_ms * 1e-3) / 2.25e15}
+        per_layer.append(entry)
+        for kind, ms, work in (("fwd_int8_gemm", f_ms, fwd_int8 + fwd_lora), ("bwd_bf16_gemm", b_ms, bwd_bf16)):
+            if dominant is None or ms > dominant[2]:
+                dominant = (sp.name, kind, ms, work)
+    sustained = ms_per_step * args.steps > 1000.0
+    bf16_peak = peaks["bf16_tflops_sustained"] if sustained else peaks["bf16_tflops"]
+    name, kind, ms, work = dominant
+    achieved = work / (ms * 1e-3) / 1e12
+    peak = bf16_peak * (2.0 if kind == "fwd_int8_gemm" else 1.0)
+    roofline = {"bound": "tensor", "kernel": f"umma_gemm_kernel<{'EPI_FWD' if kind == 'fwd_int8_gemm' else 'EPI_BWD'}> ({name})",
+                "achieved": achieved, "peak": peak, "unit": "TFLOP/s" if kind == "bwd_bf16_gemm" else "TOP/s",
+                "frac": achieved / peak, "traffic": None,
+                "peak_source": f"{peaks['source']} cuBLAS bf16 {'sustained' if sustained else 'burst'}"
+                               + (" x2 (nominal int8:bf16 ratio)" if kind == "fwd_int8_gemm" else ""),
+                "avg_launch_ms": ms}
+
+    cpu = cpu_baseline(wl, min(wl.M, 8 * args.sample_tokens)) if not args.no_cpu_baseline else None
+    line = {"metric": METRIC, "value": world * M / (ms_per_step * 1e-3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "int8 forward (int32 accumulate), bf16 backward (f32 accumulate)",
+            "data": "synthetic",
+            "config": {"workload": wl.name, "tokens_per_gpu": M,
+                       "layers": [f"{l.name} {l.K}->{l.N} nO={l.nO} r={l.r}" for l in wl.layers], "gamma": wl.gamma,
+                       "l2": f"rotating {REPLICAS} full buffer sets (weights, activations, outputs); one set alone exceeds the 126 MB L2"},
+            "clocks": clocks.summary(),
+            "e2e": {"value": world * M / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                    "ms_per_step": e2e_ms, "steps": e2e_steps},
+            "gpu_launches": int(launches),
+            "roofline": roofline, "layers": per_layer, "cpu_baseline": cpu}
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--workload", default="phi3_attn", choices=sorted(synth.WORKLOADS))
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--sample-tokens", type=int, default=128, help="tokens per step of the CPU oracle (reference arm); the cpu_baseline leg uses 8x this")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    wl = synth.WORKLOADS[args.workload]
+    if args.impl == "reference":
+        run_reference(args, wl)
+    else:
+        run_gpu(args, wl)
+
+
+if __name__ == "__main__":
+    main()

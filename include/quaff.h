@@ -169,6 +169,19 @@ quaff_status_t quaff_qlinear_bwd(int M, int K, int N,
                                  float* dA, float* dB, int accumulate,
                                  int32_t* status_opt, void* ws, size_t ws_bytes, quaff_stream_t stream);
 
+/*
+ * Measurement aids (no counterpart in the paper; process-wide state, not thread-safe).
+ *
+ * quaff_debug_launch_count: number of kernels this library has launched since it was loaded.
+ *
+ * quaff_debug_time_gemm: arm a one-shot pair of CUDA events (cudaEvent_t, created by the caller
+ * with timing enabled) around the next launch of the forward (which = 0) or grad-input
+ * (which = 1) tensor-core GEMM kernel: `start` is recorded on the launch stream right before the
+ * kernel, `stop` right after, then the pair is disarmed.  Null events disarm.
+ */
+uint64_t quaff_debug_launch_count(void);
+void quaff_debug_time_gemm(int which, void* start_event, void* stop_event);
+
 #ifdef __cplusplus
 }
 #endif

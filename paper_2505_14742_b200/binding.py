@@ -24,7 +24,7 @@ QUAFF_ERR_TIMEOUT = 6
 QUAFF_BF16, QUAFF_F32 = 0, 1
 QUAFF_WS_PREPARE, QUAFF_WS_MOMENTUM, QUAFF_WS_FWD, QUAFF_WS_BWD = 0, 1, 2, 3
 
-EXPORTS = ("quaff_status_string", "quaff_workspace_bytes", "quaff_prepare_weight", "quaff_momentum_update",
+EXPORTS = ("quaff_status_string", "quaff_workspace_bytes", "quaff_debug_launch_count", "quaff_debug_time_gemm", "quaff_prepare_weight", "quaff_momentum_update",
            "quaff_quant_act", "quaff_requant_weight_rows", "quaff_qlinear_fwd", "quaff_qlinear_bwd")
 
 _lib = None
@@ -68,6 +68,10 @@ def lib() -> ctypes.CDLL:
         L.quaff_qlinear_bwd.restype = _i32
         L.quaff_qlinear_bwd.argtypes = [_i32, _i32, _i32, _vp, _i64, _vp, _i64, _vp, _vp, _i64, _vp, _i32, _vp, _i32, _vp,
                                         _vp, _i64, _vp, _vp, _vp, _i32, _f32, _vp, _i64, _vp, _vp, _i32, _vp, _vp, _sz, _vp]
+        L.quaff_debug_launch_count.restype = ctypes.c_uint64
+        L.quaff_debug_launch_count.argtypes = []
+        L.quaff_debug_time_gemm.restype = None
+        L.quaff_debug_time_gemm.argtypes = [_i32, _vp, _vp]
         _lib = L
     return _lib
 
@@ -78,6 +82,16 @@ def status_string(code: int) -> str:
 
 def workspace_bytes(which: int, M: int, K: int, N: int, nOp: int, r: int) -> int:
     return int(lib().quaff_workspace_bytes(which, M, K, N, nOp, r))
+
+
+def quaff_debug_launch_count() -> int:
+    return int(lib().quaff_debug_launch_count())
+
+
+def quaff_debug_time_gemm(which: int, start: Optional["torch.cuda.Event"], stop: Optional["torch.cuda.Event"]) -> None:
+    """Arm (or, with None, disarm) event recording around the next forward (0) / grad-input (1) GEMM launch."""
+    lib().quaff_debug_time_gemm(which, start.cuda_event if start is not None else None,
+                                stop.cuda_event if stop is not None else None)
 
 
 def _ptr(t: Optional[torch.Tensor]):

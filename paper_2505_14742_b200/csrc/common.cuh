@@ -20,7 +20,11 @@ inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 
 inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
 inline size_t round_up(size_t a, size_t b) { return (a + b - 1) / b * b; }
 
+extern unsigned long long g_launch_count;  // kernels launched by this library (diagnostics)
+
+// Call right after every kernel launch: counts it and turns a launch error into a status.
 inline quaff_status_t launch_status() {
+    ++g_launch_count;
     return cudaGetLastError() == cudaSuccess ? QUAFF_OK : QUAFF_ERR_CUDA;
 }
 

@@ -40,6 +40,9 @@ quaff_status_t make_tmap_2d(CUtensorMap* map, const void* base, int elem_bytes, 
     return rc == CUDA_SUCCESS ? QUAFF_OK : QUAFF_ERR_CUDA;
 }
 
+static cudaEvent_t g_time_start[2] = {nullptr, nullptr};
+static cudaEvent_t g_time_stop[2] = {nullptr, nullptr};
+
 template <int EPI>
 static quaff_status_t launch_gemm(const GemmParams& p, cudaStream_t st) {
     static bool configured[64] = {false};
@@ -53,8 +56,15 @@ static quaff_status_t launch_gemm(const GemmParams& p, cudaStream_t st) {
     const int ntiles = p.tiles_m * p.tiles_n;
     if (ntiles == 0) return QUAFF_OK;
     const int grid = min(ntiles, sm_count());
+    const bool timed = g_time_start[EPI] && g_time_stop[EPI];
+    if (timed) cudaEventRecord(g_time_start[EPI], st);
     umma_gemm_kernel<EPI><<<grid, kGemmThreads, kGemmSmemBytes, st>>>(p);
-    return launch_status();
+    const quaff_status_t rc = launch_status();
+    if (timed) {
+        cudaEventRecord(g_time_stop[EPI], st);
+        g_time_start[EPI] = g_time_stop[EPI] = nullptr;
+    }
+    return rc;
 }
 
 // ------------------------------------------------------------------ small kernels
@@ -277,6 +287,14 @@ static BwdWorkspace bwd_workspace(int M, int K, int N, int nOp, int r) {
 }  // namespace quaff
 
 using namespace quaff;
+
+extern "C" uint64_t quaff_debug_launch_count(void) { return g_launch_count; }
+
+extern "C" void quaff_debug_time_gemm(int which, void* start_event, void* stop_event) {
+    if (which < 0 || which > 1) return;
+    g_time_start[which] = (cudaEvent_t)start_event;
+    g_time_stop[which] = (cudaEvent_t)stop_event;
+}
 
 extern "C" const char* quaff_status_string(quaff_status_t s) {
     switch (s) {

@@ -9,6 +9,8 @@
 
 namespace quaff {
 
+unsigned long long g_launch_count = 0;
+
 int sm_count() {
     static int cached[64] = {0};
     int dev = 0;
