@@ -131,7 +131,7 @@ quaff_status_t quaff_requant_weight_rows(const quaff_bf16* W_O, int64_t ldwo, in
  *   status_opt: optional int32[4] device word, must be zero on entry; see QUAFF_ERR_TIMEOUT
  *   ws: QUAFF_WS_FWD bytes
  * Alignment: all matrix bases 16-byte aligned; ldxq, ldxo, ldwq_main, ldwq multiples of 16;
- * ldx multiple of 8; r multiple of 8, r <= 256; nOp multiple of 32 (0 allowed).
+ * ldx multiple of 8; r multiple of 8, r <= 64; nOp multiple of 32 (0 allowed).
  */
 quaff_status_t quaff_qlinear_fwd(int M, int K, int N,
                                  const int8_t* Xq, int64_t ldxq, const int8_t* xq_O, int64_t ldxo, int nOp,
