@@ -170,6 +170,31 @@ quaff_status_t quaff_qlinear_bwd(int M, int K, int N,
                                  int32_t* status_opt, void* ws, size_t ws_bytes, quaff_stream_t stream);
 
 /*
+ * quaff_momentum_update without a caller-supplied workspace (the paper has no counterpart: this
+ * is a packaging variant of the call above, same arithmetic, same outputs).
+ *
+ * For callers that cannot hand the library device scratch because they cannot allocate any: code
+ * running where cudaMalloc is off limits - a plug-in inside a host framework that owns the whole
+ * device-memory budget and forbids allocations outside its own pool, or a step on a latency-critical
+ * path where the implicit device-wide synchronisation of cudaMalloc/cudaFree is unacceptable.  The
+ * scratch (column maxima and a block counter) lives in a fixed array compiled into the library, so
+ * this entry point calls no cudaMalloc, cudaFree or allocating library routine.
+ *
+ *  - Limit: nO <= 4096 outlier channels (16 KB + 4 B of device memory, held by every GPU that loads
+ *    the library until the process exits).  A larger nO returns QUAFF_ERR_UNSUPPORTED_SHAPE; use
+ *    quaff_momentum_update with a workspace then.
+ *  - The first call on each device looks up the array's device address (cudaGetSymbolAddress, with
+ *    that device current) and caches it.  Make that first call outside any stream capture.
+ *  - All calls on a device share the one array.  Each call clears what must start at zero, but two
+ *    calls whose kernels overlap on the GPU (different streams) race on it: serialise them.
+ * Arguments and results are exactly those of quaff_momentum_update, minus `ws` / `ws_bytes`.
+ */
+quaff_status_t quaff_momentum_update_static(const quaff_bf16* X, int64_t ldx, int M, int K,
+                                            const int32_t* O_idx, int nO, const float* wmax_O, float gamma,
+                                            float* s_O, float* colmax_O_opt, float* beta_O_opt,
+                                            quaff_stream_t stream);
+
+/*
  * Measurement aids (no counterpart in the paper; process-wide state, not thread-safe).
  *
  * quaff_debug_launch_count: number of kernels this library has launched since it was loaded.

@@ -25,7 +25,7 @@ QUAFF_BF16, QUAFF_F32 = 0, 1
 QUAFF_WS_PREPARE, QUAFF_WS_MOMENTUM, QUAFF_WS_FWD, QUAFF_WS_BWD = 0, 1, 2, 3
 
 EXPORTS = ("quaff_status_string", "quaff_workspace_bytes", "quaff_debug_launch_count", "quaff_debug_time_gemm", "quaff_prepare_weight", "quaff_momentum_update",
-           "quaff_quant_act", "quaff_requant_weight_rows", "quaff_qlinear_fwd", "quaff_qlinear_bwd")
+           "quaff_momentum_update_static", "quaff_quant_act", "quaff_requant_weight_rows", "quaff_qlinear_fwd", "quaff_qlinear_bwd")
 
 _lib = None
 _vp, _i64, _i32, _f32, _sz = ctypes.c_void_p, ctypes.c_int64, ctypes.c_int, ctypes.c_float, ctypes.c_size_t
@@ -58,6 +58,8 @@ def lib() -> ctypes.CDLL:
         L.quaff_prepare_weight.argtypes = [_vp, _i64, _i32, _i32, _vp, _i32, _vp, _i64, _vp, _vp, _i64, _vp, _vp]
         L.quaff_momentum_update.restype = _i32
         L.quaff_momentum_update.argtypes = [_vp, _i64, _i32, _i32, _vp, _i32, _vp, _f32, _vp, _vp, _vp, _vp, _sz, _vp]
+        L.quaff_momentum_update_static.restype = _i32
+        L.quaff_momentum_update_static.argtypes = [_vp, _i64, _i32, _i32, _vp, _i32, _vp, _f32, _vp, _vp, _vp, _vp]
         L.quaff_quant_act.restype = _i32
         L.quaff_quant_act.argtypes = [_vp, _i64, _i32, _i32, _vp, _i32, _vp, _vp, _i64, _vp, _i64, _i32, _vp, _vp]
         L.quaff_requant_weight_rows.restype = _i32
@@ -129,6 +131,16 @@ def quaff_momentum_update(X, O_idx, wmax_O, gamma: float, s_O, ws, colmax_O=None
     _check(lib().quaff_momentum_update(_ptr(X), _ld(X), M, K, _ptr(O_idx), nO, _ptr(wmax_O), float(gamma), _ptr(s_O),
                                        _ptr(colmax_O), _ptr(beta_O), _ptr(ws), ws.numel() * ws.element_size() if ws is not None else 0,
                                        _stream()), "quaff_momentum_update")
+
+
+def quaff_momentum_update_static(X, O_idx, wmax_O, gamma: float, s_O, colmax_O=None, beta_O=None) -> None:
+    """quaff_momentum_update for callers that cannot allocate a workspace: the scratch is a fixed array
+    inside the library (nO <= 4096; calls that overlap on one GPU race on it)."""
+    M, K = X.shape
+    nO = 0 if O_idx is None else O_idx.numel()
+    _check(lib().quaff_momentum_update_static(_ptr(X), _ld(X), M, K, _ptr(O_idx), nO, _ptr(wmax_O), float(gamma),
+                                              _ptr(s_O), _ptr(colmax_O), _ptr(beta_O), _stream()),
+           "quaff_momentum_update_static")
 
 
 def quaff_quant_act(X, O_idx, s_O, Xq, xq_O, dx) -> None:

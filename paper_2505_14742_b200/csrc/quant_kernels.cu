@@ -314,6 +314,11 @@ __global__ void __launch_bounds__(256) gather_outlier_rows_kernel(const uint16_t
     }
 }
 
+// Scratch of quaff_momentum_update_static: column-maximum bit patterns [0, nO) and the block
+// ticket counter at [nO].  Lives in every device that loads the library until the process exits.
+constexpr int kStaticMaxNO = 4096;
+static __device__ __align__(256) unsigned int g_momentum_scratch[kStaticMaxNO + 1];
+
 static bool valid_outlier_args(const int32_t* O_idx, int nO, int K) {
     return nO >= 0 && nO <= K && nO <= 4096 && (nO == 0 || O_idx != nullptr);
 }
@@ -379,4 +384,34 @@ extern "C" quaff_status_t quaff_prepare_weight(const quaff_bf16* Wt, int64_t ldw
         rc = launch_status();
     }
     return rc;
+}
+
+extern "C" quaff_status_t quaff_momentum_update_static(const quaff_bf16* X, int64_t ldx, int M, int K,
+                                                       const int32_t* O_idx, int nO, const float* wmax_O, float gamma,
+                                                       float* s_O, float* colmax_O_opt, float* beta_O_opt,
+                                                       quaff_stream_t stream) {
+    QUAFF_RETURN_IF(!X || M < 0 || K <= 0 || ldx < K, QUAFF_ERR_INVALID_ARG);
+    QUAFF_RETURN_IF(nO < 0 || nO > K || (nO > 0 && !O_idx), QUAFF_ERR_INVALID_ARG);
+    QUAFF_RETURN_IF(!(gamma >= 0.0f && gamma <= 1.0f), QUAFF_ERR_INVALID_ARG);
+    QUAFF_RETURN_IF(nO > kStaticMaxNO, QUAFF_ERR_UNSUPPORTED_SHAPE);  // more outlier channels than the built-in scratch holds
+    if (nO == 0) return QUAFF_OK;
+    QUAFF_RETURN_IF(!wmax_O || !s_O, QUAFF_ERR_INVALID_ARG);
+
+    // In host code `g_momentum_scratch` is only a stand-in for the device array; the address a kernel
+    // may use comes from cudaGetSymbolAddress, once per device, with that device current.
+    static unsigned int* scratch_of_device[64] = {nullptr};
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return QUAFF_ERR_CUDA;
+    if (!scratch_of_device[dev]) {
+        void* ptr = nullptr;
+        if (cudaGetSymbolAddress(&ptr, g_momentum_scratch) != cudaSuccess || !ptr) return QUAFF_ERR_CUDA;
+        scratch_of_device[dev] = static_cast<unsigned int*>(ptr);
+    }
+    unsigned int* scratch = scratch_of_device[dev];
+    cudaStream_t st = (cudaStream_t)stream;
+    // the array keeps the previous call's maxima and ticket count: both must start at zero
+    if (cudaMemsetAsync(scratch, 0, (size_t)(nO + 1) * sizeof(unsigned int), st) != cudaSuccess) return QUAFF_ERR_CUDA;
+    const int grid = max(1, min(ceil_div(M, 16), sm_count() * 2));
+    momentum_kernel<<<grid, 256, 0, st>>>(X, ldx, M, O_idx, nO, wmax_O, gamma, s_O, colmax_O_opt, beta_O_opt, scratch);
+    return launch_status();
 }
