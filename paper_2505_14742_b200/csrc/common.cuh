@@ -89,13 +89,17 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 // broken pipeline ends with an error status instead of hanging the device.  Other waiters see the
 // flag and give up as well.
 constexpr uint32_t kWaitLimit = 1u << 24;
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+static __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
     for (uint32_t it = 0; it < kWaitLimit; ++it) {
         if (mbar_try_wait(bar, parity)) return true;
         if ((it & 1023u) == 1023u && *abort_flag) return false;
     }
     *abort_flag = 1;
     return false;
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+    if (mbar_try_wait(bar, parity)) return true;   // fast path: keeps the issue loops of the single-thread roles short
+    return mbar_wait_slow(bar, parity, abort_flag);
 }
 
 // ------------------------------------------------------------------ PTX: TMA (no multicast anywhere)

@@ -1,6 +1,7 @@
 // quaff_qlinear_fwd / quaff_qlinear_bwd: host side (validation, tensor maps, workspace carving,
 // launches) and the small kernels around the two tcgen05 GEMMs (LoRA projections, weight
 // dequantization for the backward, outlier-column fix-up, LoRA gradients).
+#include <stdlib.h>
 #include <string.h>
 
 #include "umma_gemm.cuh"
@@ -56,114 +57,34 @@ static quaff_status_t launch_gemm(const GemmParams& p, cudaStream_t st) {
     const int ntiles = p.tiles_m * p.tiles_n;
     if (ntiles == 0) return QUAFF_OK;
     const int grid = min(ntiles, sm_count());
-    const bool timed = g_time_start[EPI] && g_time_stop[EPI];
-    if (timed) cudaEventRecord(g_time_start[EPI], st);
+    const bool timed = EPI < 2 && g_time_start[EPI % 2] && g_time_stop[EPI % 2];
+    if (timed) cudaEventRecord(g_time_start[EPI % 2], st);
     umma_gemm_kernel<EPI><<<grid, kGemmThreads, kGemmSmemBytes, st>>>(p);
     const quaff_status_t rc = launch_status();
     if (timed) {
-        cudaEventRecord(g_time_stop[EPI], st);
-        g_time_start[EPI] = g_time_stop[EPI] = nullptr;
+        cudaEventRecord(g_time_stop[EPI % 2], st);
+        g_time_start[EPI % 2] = g_time_stop[EPI % 2] = nullptr;
     }
     return rc;
 }
 
 // ------------------------------------------------------------------ small kernels
-// Bt[n][j] = B[j][n] for j < r, 0 for r <= j < rp  (K-major LoRA-up operand for the fused MMA)
-__global__ void transpose_pad_kernel(const uint16_t* __restrict__ B, int r, int N, uint16_t* __restrict__ Bt, int rp) {
+// dst[c][j] = src[j][c] for j < rows, 0 for rows <= j < rows_pad   (src is [rows][cols], dst is [cols][rows_pad])
+__global__ void transpose_pad_kernel(const uint16_t* __restrict__ src, int rows, int cols, uint16_t* __restrict__ dst, int rows_pad) {
     const int idx = blockIdx.x * blockDim.x + threadIdx.x;
-    if (idx >= N * rp) return;
-    const int n = idx / rp, j = idx % rp;
-    Bt[idx] = j < r ? B[(int64_t)j * N + n] : (uint16_t)0;
+    if (idx >= cols * rows_pad) return;
+    const int c = idx / rows_pad, j = idx % rows_pad;
+    dst[idx] = j < rows ? src[(int64_t)j * cols + c] : (uint16_t)0;
 }
 
-// out[m][j] = bf16(scale * sum_c Big[m][c] * S(c, j)), one warp per row m, fp32 accumulation.
-// S_IS_CJ: S stored [C][r] (LoRA A: T = X A); otherwise S stored [r][C] (LoRA B: G = dY B^T).
-template <int R, bool S_IS_CJ>
-__global__ void __launch_bounds__(256) row_times_small_kernel(const uint16_t* __restrict__ Big, int64_t ldb, int M, int C,
-                                                             const uint16_t* __restrict__ S, int r, float scale,
-                                                             uint16_t* __restrict__ out) {
-    const int m = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-    const int lane = threadIdx.x & 31;
-    if (m >= M) return;
-    float acc[R];
-#pragma unroll
-    for (int j = 0; j < R; ++j) acc[j] = 0.0f;
-    const uint16_t* row = Big + (int64_t)m * ldb;
-    for (int c0 = lane * 8; c0 < C; c0 += 256) {
-        float x[8];
-        if (c0 + 8 <= C) {
-            const uint4 v = __ldg(reinterpret_cast<const uint4*>(row + c0));
-            x[0] = bf16_lo(v.x); x[1] = bf16_hi(v.x); x[2] = bf16_lo(v.y); x[3] = bf16_hi(v.y);
-            x[4] = bf16_lo(v.z); x[5] = bf16_hi(v.z); x[6] = bf16_lo(v.w); x[7] = bf16_hi(v.w);
-        } else {
-            for (int e = 0; e < 8; ++e) x[e] = c0 + e < C ? bf16_bits_to_f32(row[c0 + e]) : 0.0f;
-        }
-#pragma unroll
-        for (int e = 0; e < 8; ++e) {
-            const int c = min(c0 + e, C - 1);
-#pragma unroll
-            for (int j = 0; j < R; ++j) {
-                if (j < r) {
-                    const float s = bf16_bits_to_f32(S_IS_CJ ? __ldg(S + (int64_t)c * r + j) : __ldg(S + (int64_t)j * C + c));
-                    acc[j] = fmaf(x[e], s, acc[j]);
-                }
-            }
-        }
-    }
-#pragma unroll
-    for (int j = 0; j < R; ++j) {
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) acc[j] += __shfl_xor_sync(0xffffffffu, acc[j], o);
-    }
-    if (lane == 0)
-        for (int j = 0; j < r; ++j) out[(int64_t)m * r + j] = (uint16_t)f32_to_bf16_bits(scale * acc[j]);
-}
-
-// part[s][c][j] = sum over the s-th slice of rows m of Big[m][c] * Small[m][j]   (fp32)
-template <int R>
-__global__ void __launch_bounds__(128) cols_times_small_kernel(const uint16_t* __restrict__ Big, int64_t ldb, int M, int C,
-                                                              const uint16_t* __restrict__ Small, int r,
-                                                              float* __restrict__ part, int rows_per_split) {
-    __shared__ float sm_small[32][R];
-    const int c = (blockIdx.x * 128 + threadIdx.x) * 2;
-    const int m_begin = blockIdx.y * rows_per_split;
-    const int m_end = min(M, m_begin + rows_per_split);
-    float acc0[R], acc1[R];
-#pragma unroll
-    for (int j = 0; j < R; ++j) { acc0[j] = 0.0f; acc1[j] = 0.0f; }
-    for (int mb = m_begin; mb < m_end; mb += 32) {
-        __syncthreads();
-        for (int i = threadIdx.x; i < 32 * R; i += 128) {
-            const int mm = i / R, j = i % R;
-            sm_small[mm][j] = (mb + mm < m_end && j < r) ? bf16_bits_to_f32(Small[(int64_t)(mb + mm) * r + j]) : 0.0f;
-        }
-        __syncthreads();
-        if (c < C) {
-            const int rows = min(32, m_end - mb);
-            for (int mm = 0; mm < rows; ++mm) {
-                const uint16_t* row = Big + (int64_t)(mb + mm) * ldb;
-                float x0, x1;
-                if (c + 1 < C && (ldb % 2 == 0)) {
-                    const uint32_t v = __ldg(reinterpret_cast<const uint32_t*>(row + c));
-                    x0 = bf16_lo(v); x1 = bf16_hi(v);
-                } else {
-                    x0 = bf16_bits_to_f32(row[c]);
-                    x1 = c + 1 < C ? bf16_bits_to_f32(row[c + 1]) : 0.0f;
-                }
-#pragma unroll
-                for (int j = 0; j < R; ++j) {
-                    const float s = sm_small[mm][j];
-                    acc0[j] = fmaf(x0, s, acc0[j]);
-                    acc1[j] = fmaf(x1, s, acc1[j]);
-                }
-            }
-        }
-    }
-    if (c < C) {
-        float* o = part + ((int64_t)blockIdx.y * C + c) * r;
-        for (int j = 0; j < r; ++j) o[j] = acc0[j];
-        if (c + 1 < C) for (int j = 0; j < r; ++j) o[r + j] = acc1[j];
-    }
+// out[m][j] = bf16(scale * sum_s part[s][m][j])
+__global__ void reduce_parts_bf16_kernel(const float* __restrict__ part, int S, int rows, int r, float scale,
+                                         uint16_t* __restrict__ out) {
+    const int idx = blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= rows * r) return;
+    float sum = 0.0f;
+    for (int s = 0; s < S; ++s) sum += part[(int64_t)s * rows * r + idx];
+    out[idx] = (uint16_t)f32_to_bf16_bits(scale * sum);
 }
 
 // dst = (accumulate ? dst : 0) + scale * sum_s part[s][c][j];  dst index c*r + j, or j*C + c when transposed
@@ -230,38 +151,83 @@ __global__ void bwd_fixup_kernel(const float* __restrict__ P, int64_t ldp, int M
     dX[(int64_t)m * lddx + k] = (uint16_t)f32_to_bf16_bits(v + l);
 }
 
-template <bool S_IS_CJ>
-static quaff_status_t launch_row_times_small(const uint16_t* Big, int64_t ldb, int M, int C, const uint16_t* S, int r,
-                                             float scale, uint16_t* out, cudaStream_t st) {
-    const int grid = ceil_div(M, 8);
-    if (r <= 16) row_times_small_kernel<16, S_IS_CJ><<<grid, 256, 0, st>>>(Big, ldb, M, C, S, r, scale, out);
-    else if (r <= 32) row_times_small_kernel<32, S_IS_CJ><<<grid, 256, 0, st>>>(Big, ldb, M, C, S, r, scale, out);
-    else row_times_small_kernel<64, S_IS_CJ><<<grid, 256, 0, st>>>(Big, ldb, M, C, S, r, scale, out);
-    return launch_status();
-}
-
-static int split_count(int M, int C) {
-    const int blocks_c = ceil_div(C, 256);
-    int S = ceil_div(2 * sm_count(), blocks_c);
-    S = max(1, min(S, ceil_div(M, 64)));
-    return S;
-}
-
-static quaff_status_t launch_cols_times_small(const uint16_t* Big, int64_t ldb, int M, int C, const uint16_t* Small, int r,
-                                              float scale, int transposed, int accumulate, float* part, float* dst,
-                                              cudaStream_t st) {
-    const int S = split_count(M, C);
-    const int rows_per_split = ceil_div(ceil_div(M, S), 32) * 32;
-    const dim3 grid(ceil_div(C, 256), S);
-    if (r <= 16) cols_times_small_kernel<16><<<grid, 128, 0, st>>>(Big, ldb, M, C, Small, r, part, rows_per_split);
-    else if (r <= 32) cols_times_small_kernel<32><<<grid, 128, 0, st>>>(Big, ldb, M, C, Small, r, part, rows_per_split);
-    else cols_times_small_kernel<64><<<grid, 128, 0, st>>>(Big, ldb, M, C, Small, r, part, rows_per_split);
-    if (launch_status() != QUAFF_OK) return QUAFF_ERR_CUDA;
-    reduce_parts_kernel<<<ceil_div(C * r, 256), 256, 0, st>>>(part, S, C, r, scale, transposed, accumulate, dst);
-    return launch_status();
-}
-
 static int pad16(int r) { return (r + 15) / 16 * 16; }
+
+constexpr int kPlanSMs = 148;   // split-K plans (and so workspace sizes) are fixed for the B200's 148 SMs
+
+// Split-K plan of a skinny GEMM with `rows_out` output rows and a contraction of `kc` elements (bf16,
+// 64 per k-block): enough splits to give every SM a tile, at least two k-blocks per split.
+struct SplitPlan { int S, kblk; };
+static SplitPlan split_plan(int rows_out, int kc) {
+    const int tiles = ceil_div(rows_out, kTileM);
+    const int nblk = max(1, ceil_div(kc, 64));
+    int S = max(1, min(ceil_div(kPlanSMs, tiles), ceil_div(nblk, 2)));
+    SplitPlan p;
+    p.kblk = ceil_div(nblk, S);
+    p.S = ceil_div(nblk, p.kblk);
+    return p;
+}
+static size_t split_part_bytes(int rows_out, int kc, int r) {
+    return (size_t)split_plan(rows_out, kc).S * rows_out * max(r, 1) * 4;
+}
+
+static void fill_phase(GemmPhase& ph, int is_i8, int kext, int acc_slot, int fresh, int tn_limit, int n_mma, int b_box_rows) {
+    const int kbox = is_i8 ? 128 : 64, kins = is_i8 ? 32 : 16;
+    ph.nblk = ceil_div(kext, kbox);
+    ph.is_i8 = is_i8;
+    ph.nmma_last = ceil_div(kext - (ph.nblk - 1) * kbox, kins);
+    ph.acc_slot = acc_slot;
+    ph.fresh = fresh;
+    ph.tn_limit = tn_limit;
+    ph.mn_major = 0;
+    ph.n_mma = n_mma;
+    ph.tx_bytes = (uint32_t)(kOperandBytes + b_box_rows * 128);
+    ph.kblk_per_tn = 0;
+    ph.b_rows_per_tn = kTileN;
+}
+
+// part[s][row][j] (f32, row pitch r) = sum over the s-th slice of the contraction of A(row, :) * B(j, :).
+//   K-major  (mn_major = 0): A is [rows_out][kc] with pitch lda, B is [r][kc] with pitch ldb.
+//   MN-major (mn_major = 1): A is [kc][rows_out] with pitch lda, B is [kc][r] with pitch ldb.
+static quaff_status_t skinny_gemm(int mn_major, const void* A, int64_t lda, const void* B, int64_t ldb, int rows_out,
+                                  int kc, int r, float* part, int32_t* status, cudaStream_t st, int* S_out) {
+    const SplitPlan sp = split_plan(rows_out, kc);
+    const int rp = pad16(r);
+    GemmParams p;
+    memset(&p, 0, sizeof(p));
+    GemmPhase& ph = p.ph[0];
+    quaff_status_t rc;
+    if (!mn_major) {
+        if ((rc = make_tmap_2d(&ph.map_a, A, 2, rows_out, kc, lda, kTileM, 64)) != QUAFF_OK) return rc;
+        if ((rc = make_tmap_2d(&ph.map_b, B, 2, r, kc, ldb, rp, 64)) != QUAFF_OK) return rc;
+        ph.tx_bytes = (uint32_t)(kOperandBytes + rp * 128);
+    } else {
+        if ((rc = make_tmap_2d(&ph.map_a, A, 2, kc, rows_out, lda, 64, 64)) != QUAFF_OK) return rc;
+        if ((rc = make_tmap_2d(&ph.map_b, B, 2, kc, r, ldb, 64, 64)) != QUAFF_OK) return rc;
+        ph.tx_bytes = (uint32_t)(kOperandBytes + 8192);
+    }
+    ph.nblk = sp.kblk; ph.is_i8 = 0; ph.nmma_last = 4; ph.acc_slot = 0; ph.fresh = 1; ph.tn_limit = 1 << 30;
+    ph.mn_major = mn_major; ph.n_mma = rp; ph.kblk_per_tn = sp.kblk; ph.b_rows_per_tn = 0;
+    p.nphases = 1;
+    p.M = rows_out; p.N = rp;
+    p.tiles_m = ceil_div(rows_out, kTileM); p.tiles_n = sp.S;
+    p.status = status;
+    p.part = part; p.part_ld = r; p.part_cols = r;
+    *S_out = sp.S;
+    return launch_gemm<EPI_PART>(p, st);
+}
+
+struct FwdWorkspace { size_t off_bt, off_at, off_part, total; };
+static FwdWorkspace fwd_workspace(int M, int K, int N, int r) {
+    FwdWorkspace w;
+    const int rp = pad16(max(r, 1));
+    size_t off = 0;
+    w.off_bt = off;   off += round_up((size_t)N * rp * 2, 256);          // B^T, K-major LoRA-up operand
+    w.off_at = off;   off += round_up((size_t)rp * K * 2, 256);          // A^T, K-major LoRA-down operand
+    w.off_part = off; off += round_up(split_part_bytes(M, K, r), 256);   // split-K partials of T = X A
+    w.total = off;
+    return w;
+}
 
 struct BwdWorkspace {
     size_t off_wext, off_g, off_p, off_part, total;
@@ -277,9 +243,10 @@ static BwdWorkspace bwd_workspace(int M, int K, int N, int nOp, int r) {
     w.off_g = off;    off += round_up((size_t)M * (size_t)max(r, 1) * 2, 256);
     w.off_p = off;    off += round_up((size_t)M * (size_t)max(2 * nOp, 1) * 4, 256);
     w.off_part = off;
-    const size_t pa = (size_t)split_count(M, K) * K * max(r, 1) * 4;
-    const size_t pb = (size_t)split_count(M, N) * N * max(r, 1) * 4;
-    off += round_up(pa > pb ? pa : pb, 256);
+    size_t pmax = split_part_bytes(M, N, r);                 // G = dY B^T
+    pmax = max(pmax, split_part_bytes(K, M, r));             // dA = X^T G
+    pmax = max(pmax, split_part_bytes(N, M, r));             // dB^T = dY^T T
+    off += round_up(pmax, 256);
     w.total = off;
     return w;
 }
@@ -313,7 +280,7 @@ extern "C" size_t quaff_workspace_bytes(int which, int M, int K, int N, int nOp,
     switch (which) {
         case QUAFF_WS_PREPARE: return 0;
         case QUAFF_WS_MOMENTUM: return round_up((size_t)(nOp + 1) * 4, 256);
-        case QUAFF_WS_FWD: return round_up((size_t)N * (size_t)pad16(max(r, 1)) * 2, 256);
+        case QUAFF_WS_FWD: return fwd_workspace(M, K, N, r).total;
         case QUAFF_WS_BWD: return bwd_workspace(M, K, N, nOp, r).total;
     }
     return 0;
@@ -332,16 +299,20 @@ extern "C" quaff_status_t quaff_qlinear_fwd(int M, int K, int N, const int8_t* X
     QUAFF_RETURN_IF(r > 0 && (!X || !A || !B || !T_out || ldx < K), QUAFF_ERR_INVALID_ARG);
     QUAFF_RETURN_IF(y_dtype != QUAFF_BF16 && y_dtype != QUAFF_F32, QUAFF_ERR_INVALID_ARG);
     QUAFF_RETURN_IF((nOp % 32) || (r % 8) || r > 64, QUAFF_ERR_UNSUPPORTED_SHAPE);
+    QUAFF_RETURN_IF(r > 0 && (K % 8), QUAFF_ERR_UNSUPPORTED_SHAPE);
     QUAFF_RETURN_IF(!aligned16(Xq) || !aligned16(Wq) || (ldxq % 16) || (ldwq_main % 16), QUAFF_ERR_ALIGNMENT);
     QUAFF_RETURN_IF(nOp > 0 && (!aligned16(xq_O) || !aligned16(wq_O) || (ldxo % 16) || (ldwq % 16)), QUAFF_ERR_ALIGNMENT);
     QUAFF_RETURN_IF(r > 0 && (!aligned16(X) || !aligned16(T_out) || (ldx % 8)), QUAFF_ERR_ALIGNMENT);
     QUAFF_RETURN_IF(!aligned16(Y), QUAFF_ERR_ALIGNMENT);
-    QUAFF_RETURN_IF(r > 0 && (!ws || !aligned16(ws) || ws_bytes < quaff_workspace_bytes(QUAFF_WS_FWD, M, K, N, nOp, r)),
-                    QUAFF_ERR_WORKSPACE_TOO_SMALL);
+    const FwdWorkspace w = fwd_workspace(M, K, N, r);
+    QUAFF_RETURN_IF(r > 0 && (!ws || !aligned16(ws) || ws_bytes < w.total), QUAFF_ERR_WORKSPACE_TOO_SMALL);
     if (M == 0) return QUAFF_OK;
     cudaStream_t st = (cudaStream_t)stream;
     const int rp = pad16(r);
-    uint16_t* Bt = reinterpret_cast<uint16_t*>(ws);
+    unsigned char* base = reinterpret_cast<unsigned char*>(ws);
+    uint16_t* Bt = reinterpret_cast<uint16_t*>(base + w.off_bt);
+    uint16_t* At = reinterpret_cast<uint16_t*>(base + w.off_at);
+    float* part = reinterpret_cast<float*>(base + w.off_part);
 
     GemmParams p;
     memset(&p, 0, sizeof(p));
@@ -351,22 +322,29 @@ extern "C" quaff_status_t quaff_qlinear_fwd(int M, int K, int N, const int8_t* X
         GemmPhase& ph = p.ph[np++];
         if ((rc = make_tmap_2d(&ph.map_a, Xq, 1, M, K, ldxq, kTileM, 128)) != QUAFF_OK) return rc;
         if ((rc = make_tmap_2d(&ph.map_b, Wq, 1, N, K, ldwq_main, kTileN, 128)) != QUAFF_OK) return rc;
-        ph.nblk = ceil_div(K, 128); ph.is_i8 = 1; ph.kext = K; ph.acc_slot = 0; ph.fresh = 1; ph.tn_limit = 1 << 30;
+        fill_phase(ph, 1, K, 0, 1, 1 << 30, kTileN, kTileN);
     }
     if (nOp > 0) {   // outlier: acc2 = xq_O wq_O^T over nOp
         GemmPhase& ph = p.ph[np++];
         if ((rc = make_tmap_2d(&ph.map_a, xq_O, 1, M, nOp, ldxo, kTileM, 128)) != QUAFF_OK) return rc;
         if ((rc = make_tmap_2d(&ph.map_b, wq_O, 1, N, nOp, ldwq, kTileN, 128)) != QUAFF_OK) return rc;
-        ph.nblk = ceil_div(nOp, 128); ph.is_i8 = 1; ph.kext = nOp; ph.acc_slot = 1; ph.fresh = 1; ph.tn_limit = 1 << 30;
+        fill_phase(ph, 1, nOp, 1, 1, 1 << 30, kTileN, kTileN);
     }
-    if (r > 0) {     // LoRA up: acc3 = T Bt^T over r
-        transpose_pad_kernel<<<ceil_div(N * rp, 256), 256, 0, st>>>(B, r, N, Bt, rp);
+    if (r > 0) {
+        // LoRA down-projection T = bf16(X A): split-K tensor-core GEMM over K, then a reduction to bf16
+        transpose_pad_kernel<<<ceil_div(K * rp, 256), 256, 0, st>>>(A, K, r, At, K);   // At[j][k] = A[k][j]
         if ((rc = launch_status()) != QUAFF_OK) return rc;
-        if ((rc = launch_row_times_small<true>(X, ldx, M, K, A, r, 1.0f, T_out, st)) != QUAFF_OK) return rc;
+        transpose_pad_kernel<<<ceil_div(N * rp, 256), 256, 0, st>>>(B, r, N, Bt, rp);  // Bt[n][j] = B[j][n]
+        if ((rc = launch_status()) != QUAFF_OK) return rc;
+        int S = 1;
+        if ((rc = skinny_gemm(0, X, ldx, At, K, M, K, r, part, status_opt, st, &S)) != QUAFF_OK) return rc;
+        reduce_parts_bf16_kernel<<<ceil_div(M * r, 256), 256, 0, st>>>(part, S, M, r, 1.0f, T_out);
+        if ((rc = launch_status()) != QUAFF_OK) return rc;
+        // LoRA up: acc3 = T Bt^T over r
         GemmPhase& ph = p.ph[np++];
         if ((rc = make_tmap_2d(&ph.map_a, T_out, 2, M, r, r, kTileM, 64)) != QUAFF_OK) return rc;
         if ((rc = make_tmap_2d(&ph.map_b, Bt, 2, N, rp, rp, kTileN, 64)) != QUAFF_OK) return rc;
-        ph.nblk = ceil_div(rp, 64); ph.is_i8 = 0; ph.kext = rp; ph.acc_slot = 2; ph.fresh = 1; ph.tn_limit = 1 << 30;
+        fill_phase(ph, 0, rp, 2, 1, 1 << 30, kTileN, kTileN);
     }
     p.nphases = np;
     p.M = M; p.N = N;
@@ -394,9 +372,11 @@ extern "C" quaff_status_t quaff_qlinear_bwd(int M, int K, int N, const quaff_bf1
     QUAFF_RETURN_IF(r > 0 && (dA || dB) && (!dA || !dB || !X || !T || ldx < K), QUAFF_ERR_INVALID_ARG);
     QUAFF_RETURN_IF(dX && lddx < K, QUAFF_ERR_INVALID_ARG);
     QUAFF_RETURN_IF((nOp % 32) || (r % 8) || r > 64, QUAFF_ERR_UNSUPPORTED_SHAPE);
+    QUAFF_RETURN_IF(r > 0 && (N % 8), QUAFF_ERR_UNSUPPORTED_SHAPE);
     QUAFF_RETURN_IF(!aligned16(dY) || (lddy % 8), QUAFF_ERR_ALIGNMENT);
     QUAFF_RETURN_IF(dX && (!aligned16(dX) || (lddx % 8)), QUAFF_ERR_ALIGNMENT);
-    QUAFF_RETURN_IF(r > 0 && !aligned16(A), QUAFF_ERR_ALIGNMENT);
+    QUAFF_RETURN_IF(r > 0 && (!aligned16(A) || !aligned16(B)), QUAFF_ERR_ALIGNMENT);
+    QUAFF_RETURN_IF(r > 0 && dA && (!aligned16(X) || !aligned16(T) || (ldx % 8)), QUAFF_ERR_ALIGNMENT);
     const BwdWorkspace w = bwd_workspace(M, K, N, nOp, r);
     QUAFF_RETURN_IF(!ws || !aligned16(ws) || ws_bytes < w.total, QUAFF_ERR_WORKSPACE_TOO_SMALL);
     if (M == 0) return QUAFF_OK;
@@ -407,9 +387,12 @@ extern "C" quaff_status_t quaff_qlinear_bwd(int M, int K, int N, const quaff_bf1
     float* P = reinterpret_cast<float*>(base + w.off_p);
     float* part = reinterpret_cast<float*>(base + w.off_part);
     quaff_status_t rc;
+    int S = 1;
 
-    if (r > 0) {   // G = bf16(lora_scale * dY B^T)
-        if ((rc = launch_row_times_small<false>(dY, lddy, M, N, B, r, lora_scale, G, st)) != QUAFF_OK) return rc;
+    if (r > 0) {   // G = bf16(lora_scale * dY B^T): B [r][N] is already K-major for this contraction over N
+        if ((rc = skinny_gemm(0, dY, lddy, B, N, M, N, r, part, status_opt, st, &S)) != QUAFF_OK) return rc;
+        reduce_parts_bf16_kernel<<<ceil_div(M * r, 256), 256, 0, st>>>(part, S, M, r, lora_scale, G);
+        if ((rc = launch_status()) != QUAFF_OK) return rc;
     }
     if (dX) {
         const int Kpad = ceil_div(K, kTileN) * kTileN;
@@ -424,14 +407,13 @@ extern "C" quaff_status_t quaff_qlinear_bwd(int M, int K, int N, const quaff_bf1
             GemmPhase& ph = p.ph[np++];
             if ((rc = make_tmap_2d(&ph.map_a, dY, 2, M, N, lddy, kTileM, 64)) != QUAFF_OK) return rc;
             if ((rc = make_tmap_2d(&ph.map_b, Wext, 2, Kext, N, w.ldw, kTileN, 64)) != QUAFF_OK) return rc;
-            ph.nblk = ceil_div(N, 64); ph.is_i8 = 0; ph.kext = N; ph.acc_slot = 0; ph.fresh = 1; ph.tn_limit = 1 << 30;
+            fill_phase(ph, 0, N, 0, 1, 1 << 30, kTileN, kTileN);
         }
         if (r > 0) {   // + G A^T over r, only for the real dX columns
             GemmPhase& ph = p.ph[np++];
             if ((rc = make_tmap_2d(&ph.map_a, G, 2, M, r, r, kTileM, 64)) != QUAFF_OK) return rc;
             if ((rc = make_tmap_2d(&ph.map_b, A, 2, K, r, r, kTileN, 64)) != QUAFF_OK) return rc;
-            ph.nblk = ceil_div(r, 64); ph.is_i8 = 0; ph.kext = pad16(r); ph.acc_slot = 0; ph.fresh = 0;
-            ph.tn_limit = ceil_div(K, kTileN);
+            fill_phase(ph, 0, pad16(r), 0, 0, ceil_div(K, kTileN), kTileN, kTileN);
         }
         p.nphases = np;
         p.M = M;
@@ -450,8 +432,14 @@ extern "C" quaff_status_t quaff_qlinear_bwd(int M, int K, int N, const quaff_bf1
         }
     }
     if (r > 0 && dA && dB) {
-        if ((rc = launch_cols_times_small(X, ldx, M, K, G, r, 1.0f, 0, accumulate, part, dA, st)) != QUAFF_OK) return rc;
-        if ((rc = launch_cols_times_small(dY, lddy, M, N, T, r, lora_scale, 1, accumulate, part, dB, st)) != QUAFF_OK) return rc;
+        // dA = X^T G and dB^T = dY^T T: the contraction runs over the tokens, the slow axis of X, G, dY and T,
+        // so both operands are MN-major
+        if ((rc = skinny_gemm(1, X, ldx, G, r, K, M, r, part, status_opt, st, &S)) != QUAFF_OK) return rc;
+        reduce_parts_kernel<<<ceil_div(K * r, 256), 256, 0, st>>>(part, S, K, r, 1.0f, 0, accumulate, dA);
+        if ((rc = launch_status()) != QUAFF_OK) return rc;
+        if ((rc = skinny_gemm(1, dY, lddy, T, r, N, M, r, part, status_opt, st, &S)) != QUAFF_OK) return rc;
+        reduce_parts_kernel<<<ceil_div(N * r, 256), 256, 0, st>>>(part, S, N, r, lora_scale, 1, accumulate, dB);
+        if ((rc = launch_status()) != QUAFF_OK) return rc;
     }
     return QUAFF_OK;
 }

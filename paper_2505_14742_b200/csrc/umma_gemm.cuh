@@ -1,20 +1,28 @@
-// Persistent, warp-specialised tcgen05 GEMM pipeline shared by the forward (Eq. 9 + LoRA) and the
-// grad-input kernels.
+// Persistent, warp-specialised tcgen05 GEMM pipeline shared by the forward (Eq. 9 + LoRA), the
+// grad-input GEMM and the skinny LoRA GEMMs (T = X A, G = dY B^T, dA = X^T G, dB = T^T dY).
 //
 //   warp 0      : TMA producer (one elected lane) - 128-byte-swizzled operand tiles into a ring of stages
 //   warp 1      : TMEM allocation + MMA issue (one elected lane) - tcgen05.mma, accumulators in TMEM
 //   warps 2..5  : epilogue - tcgen05.ld of the finished accumulators, dequantization / conversion, stores
 //
-// An output tile is 128 x 128.  Its contraction is a list of up to three PHASES, each a run of
-// k-blocks with its own pair of tensor maps, operand type and accumulator:
-//   forward : main INT8 (over K) -> acc slot 0 | outlier INT8 (over nOp) -> slot 1 | LoRA bf16 (over r) -> slot 2
-//   backward: main bf16 (over N) -> slot 0     | LoRA bf16 (over r) -> slot 0 (accumulating)
-// Every k-block is one stage: an A tile and a B tile of 128 rows x 128 bytes each, both K-major.
+// An output tile is 128 rows x up to 128 columns.  Its contraction is a list of up to three PHASES,
+// each a run of k-blocks with its own pair of tensor maps, operand type and accumulator:
+//   forward : main INT8 (over K) -> slot 0 | outlier INT8 (over nOp) -> slot 1 | LoRA bf16 (over r) -> slot 2
+//   backward: main bf16 (over N) -> slot 0 | LoRA bf16 (over r) -> slot 0 (accumulating)
+//   skinny  : one bf16 phase over a slice of the contraction (split-K); partial sums go to a workspace
+// Every k-block is one stage: an A tile (128 rows) and a B tile (up to 128 rows) of 128 bytes per row.
+// Operands are either K-major (rows = output index, the 128 bytes run along the contraction) or
+// MN-major (rows = contraction index, the 128 bytes run along the output index; used where the
+// contraction is the slow axis of the caller's matrix, i.e. X^T G and T^T dY).
 // Tails need no special case: TMA zero-fills out-of-range rows and columns, and the epilogue masks stores.
 //
 // TMEM (512 columns): slot 0 is double-buffered at columns [0,128) and [128,256) so the main
 // contraction of tile t+1 overlaps the epilogue of tile t; slots 1 and 2 live at [256,384) and
 // [384,512) and are written only after the epilogue of the previous tile has drained them.
+//
+// The producer and the MMA issuer are single threads; their per-k-block instruction count bounds the
+// tensor-pipe utilisation, so everything that does not change inside a phase is hoisted out of the
+// k-block loops.
 //
 // Every wait is bounded (see mbar_wait); on expiry all roles fall through to the common exit, TMEM is
 // freed, and QUAFF_ERR_TIMEOUT is written to the status word.
@@ -33,17 +41,22 @@ constexpr int kGemmThreads = 192;
 constexpr int kMaxPhases = 3;
 
 struct GemmPhase {
-    CUtensorMap map_a;   // rows = output rows (M side), columns = contraction
-    CUtensorMap map_b;   // rows = output columns (N side), columns = contraction
-    int nblk;            // k-blocks in this phase
+    CUtensorMap map_a;   // K-major: [rows = output rows][cols = contraction]; MN-major: [rows = contraction][cols = output rows]
+    CUtensorMap map_b;   // same, for the output columns
+    int nblk;            // k-blocks per tile in this phase
     int is_i8;           // 1: kind::i8 (128 elements per block, 32 per MMA); 0: kind::f16 bf16 (64 per block, 16 per MMA)
-    int kext;            // contraction extent in elements
+    int nmma_last;       // MMAs issued for the last k-block (1..4); every other block issues 4
     int acc_slot;        // 0 main (double-buffered), 1, 2 auxiliary
-    int fresh;           // 1: first MMA of the phase overwrites the accumulator
+    int fresh;           // 1: the first MMA of the phase overwrites the accumulator
     int tn_limit;        // the phase runs only for column tiles tn < tn_limit
+    int mn_major;        // 0: both operands K-major; 1: both MN-major
+    int n_mma;           // N of the MMA instruction (multiple of 16, <= 128)
+    uint32_t tx_bytes;   // bytes that land in one stage
+    int kblk_per_tn;     // split-K: first k-block of a tile is tn * kblk_per_tn (0 otherwise)
+    int b_rows_per_tn;   // B row offset per tn (128 for an ordinary GEMM, 0 for split-K)
 };
 
-enum { EPI_FWD = 0, EPI_BWD = 1 };
+enum { EPI_FWD = 0, EPI_BWD = 1, EPI_PART = 2 };
 
 struct GemmParams {
     GemmPhase ph[kMaxPhases];
@@ -70,6 +83,10 @@ struct GemmParams {
     int64_t lddx;
     float* P;
     int64_t ldp;
+    // partial-sum epilogue (split-K): part[(tn * M + m) * part_ld + j] = accumulator[m][j], j < part_cols
+    float* part;
+    int part_ld;
+    int part_cols;
 };
 
 struct GemmSmem {
@@ -85,6 +102,14 @@ struct GemmSmem {
 
 constexpr size_t kGemmSmemBytes = 1024 + (size_t)kStages * kStageBytes + sizeof(GemmSmem);
 
+// high word of the shared-memory matrix descriptor: stride byte offset 1024 (8 rows x 128 bytes),
+// descriptor version 1, SWIZZLE_128B
+constexpr uint32_t kDescHi = (1024u >> 4) | (1u << 14) | (2u << 29);
+
+__device__ __forceinline__ uint64_t make_desc(uint32_t lo, uint32_t hi) {
+    return (static_cast<uint64_t>(hi) << 32) | lo;
+}
+
 template <int EPI>
 __global__ void __launch_bounds__(kGemmThreads, 1) umma_gemm_kernel(const __grid_constant__ GemmParams p) {
     extern __shared__ unsigned char smem_dyn[];
@@ -97,11 +122,13 @@ __global__ void __launch_bounds__(kGemmThreads, 1) umma_gemm_kernel(const __grid
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
     const int ntiles = p.tiles_m * p.tiles_n;
+    const uint32_t full0 = smem_u32(&sm->full[0]);
+    const uint32_t empty0 = smem_u32(&sm->empty[0]);
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; ++s) {
-            mbar_init(smem_u32(&sm->full[s]), 1);
-            mbar_init(smem_u32(&sm->empty[s]), 1);
+            mbar_init(full0 + 8u * s, 1);
+            mbar_init(empty0 + 8u * s, 1);
         }
         mbar_init(smem_u32(&sm->tmem_full), 1);
         mbar_init(smem_u32(&sm->tmem_empty), 4);
@@ -124,23 +151,35 @@ __global__ void __launch_bounds__(kGemmThreads, 1) umma_gemm_kernel(const __grid
                 prefetch_tmap(&p.ph[i].map_a);
                 prefetch_tmap(&p.ph[i].map_b);
             }
-            int stage = 0;
-            uint32_t phase = 0;
+            uint32_t stage = 0, phase = 0;
             bool ok = true;
             for (int tile = blockIdx.x; tile < ntiles && ok; tile += gridDim.x) {
                 const int tm = tile % p.tiles_m, tn = tile / p.tiles_m;
-                const int m0 = tm * kTileM, n0 = tn * kTileN;
+                const int m0 = tm * kTileM;
                 for (int i = 0; i < p.nphases && ok; ++i) {
                     const GemmPhase& ph = p.ph[i];
                     if (tn >= ph.tn_limit) continue;
-                    const int kbox = ph.is_i8 ? 128 : 64;
-                    for (int b = 0; b < ph.nblk; ++b) {
-                        if (!mbar_wait(smem_u32(&sm->empty[stage]), phase ^ 1u, abort_flag)) { ok = false; break; }
-                        const uint32_t bar = smem_u32(&sm->full[stage]);
+                    const CUtensorMap* map_a = &ph.map_a;
+                    const CUtensorMap* map_b = &ph.map_b;
+                    const int nblk = ph.nblk;
+                    const uint32_t tx = ph.tx_bytes;
+                    const int n0 = tn * ph.b_rows_per_tn;
+                    const int kstep = ph.is_i8 ? 128 : 64;
+                    int kc = tn * ph.kblk_per_tn * kstep;      // contraction coordinate of the next block
+                    const bool mn = ph.mn_major != 0;
+                    for (int b = 0; b < nblk; ++b, kc += kstep) {
+                        if (!mbar_wait(empty0 + 8u * stage, phase ^ 1u, abort_flag)) { ok = false; break; }
+                        const uint32_t bar = full0 + 8u * stage;
                         const uint32_t dst = tiles_base + stage * kStageBytes;
-                        mbar_arrive_expect_tx(bar, kStageBytes);
-                        tma_load_2d(dst, &ph.map_a, b * kbox, m0, bar);
-                        tma_load_2d(dst + kOperandBytes, &ph.map_b, b * kbox, n0, bar);
+                        mbar_arrive_expect_tx(bar, tx);
+                        if (!mn) {
+                            tma_load_2d(dst, map_a, kc, m0, bar);
+                            tma_load_2d(dst + kOperandBytes, map_b, kc, n0, bar);
+                        } else {   // 64 output indices x 64 contraction rows per box
+                            tma_load_2d(dst, map_a, m0, kc, bar);
+                            tma_load_2d(dst + 8192, map_a, m0 + 64, kc, bar);
+                            tma_load_2d(dst + kOperandBytes, map_b, n0, kc, bar);
+                        }
                         if (++stage == kStages) { stage = 0; phase ^= 1u; }
                     }
                 }
@@ -149,43 +188,54 @@ __global__ void __launch_bounds__(kGemmThreads, 1) umma_gemm_kernel(const __grid
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer
         if (elect_one()) {
-            const uint32_t idesc_i8 = umma_idesc(kCFmtS32, kFmtS8, kTileM, kTileN);
-            const uint32_t idesc_bf = umma_idesc(kCFmtF32, kFmtBF16, kTileM, kTileN);
-            int stage = 0;
-            uint32_t phase = 0;
+            uint32_t stage = 0, phase = 0;
             bool ok = true;
             int t = 0;
+            const uint32_t tmem_empty_bar = smem_u32(&sm->tmem_empty);
+            const uint32_t tmem_full_bar = smem_u32(&sm->tmem_full);
             for (int tile = blockIdx.x; tile < ntiles && ok; tile += gridDim.x, ++t) {
                 const int tn = tile / p.tiles_m;
                 for (int i = 0; i < p.nphases && ok; ++i) {
                     const GemmPhase& ph = p.ph[i];
                     if (tn < ph.tn_limit) {
                         const uint32_t acc = tmem_base + (ph.acc_slot == 0 ? (uint32_t)((t & 1) * kTileN) : (uint32_t)((ph.acc_slot + 1) * kTileN));
-                        const int kbox = ph.is_i8 ? 128 : 64;
-                        const int kins = ph.is_i8 ? 32 : 16;
-                        for (int b = 0; b < ph.nblk; ++b) {
-                            if (!mbar_wait(smem_u32(&sm->full[stage]), phase, abort_flag)) { ok = false; break; }
+                        const int nblk = ph.nblk;
+                        const int nmma_last = ph.nmma_last;
+                        const bool i8 = ph.is_i8 != 0;
+                        const bool mn = ph.mn_major != 0;
+                        // K-major: the leading byte offset is unused (encoded 1), a 32-byte K step inside the swizzled row.
+                        // MN-major: 64-wide output atoms are 8192 bytes apart (A tile = two TMA boxes); one MMA consumes
+                        // 16 contraction rows = 2048 bytes.
+                        const uint32_t lbo = mn ? ((8192u >> 4) << 16) : (1u << 16);
+                        const uint32_t kadv = mn ? (2048u >> 4) : (32u >> 4);
+                        const uint32_t idesc = (i8 ? umma_idesc(kCFmtS32, kFmtS8, kTileM, 0) : umma_idesc(kCFmtF32, kFmtBF16, kTileM, 0)) |
+                                               ((uint32_t)(ph.n_mma >> 3) << 17) | (mn ? ((1u << 15) | (1u << 16)) : 0u);
+                        uint32_t accumulate = ph.fresh ? 0u : 1u;
+                        for (int b = 0; b < nblk; ++b) {
+                            if (!mbar_wait(full0 + 8u * stage, phase, abort_flag)) { ok = false; break; }
                             tc_fence_after();
-                            const uint32_t a_addr = tiles_base + stage * kStageBytes;
-                            const uint64_t da = smem_desc_k_sw128(a_addr);
-                            const uint64_t db = smem_desc_k_sw128(a_addr + kOperandBytes);
-                            const int left = ph.kext - b * kbox;
-                            const int nmma = (min(kbox, left) + kins - 1) / kins;
-                            for (int k = 0; k < nmma; ++k) {
-                                const uint32_t accumulate = (ph.fresh && b == 0 && k == 0) ? 0u : 1u;
-                                if (ph.is_i8) umma_i8(acc, da + 2u * k, db + 2u * k, idesc_i8, accumulate);
-                                else          umma_f16(acc, da + 2u * k, db + 2u * k, idesc_bf, accumulate);
+                            const uint32_t a_lo = (((tiles_base + stage * kStageBytes) & 0x3FFFFu) >> 4) | lbo;
+                            const uint32_t b_lo = a_lo + (kOperandBytes >> 4);
+                            const int nmma = (b == nblk - 1) ? nmma_last : 4;
+                            if (i8) {
+#pragma unroll
+                                for (int k = 0; k < 4; ++k)
+                                    if (k < nmma) { umma_i8(acc, make_desc(a_lo + k * kadv, kDescHi), make_desc(b_lo + k * kadv, kDescHi), idesc, accumulate); accumulate = 1u; }
+                            } else {
+#pragma unroll
+                                for (int k = 0; k < 4; ++k)
+                                    if (k < nmma) { umma_f16(acc, make_desc(a_lo + k * kadv, kDescHi), make_desc(b_lo + k * kadv, kDescHi), idesc, accumulate); accumulate = 1u; }
                             }
-                            umma_commit(smem_u32(&sm->empty[stage]));
+                            umma_commit(empty0 + 8u * stage);
                             if (++stage == kStages) { stage = 0; phase ^= 1u; }
                         }
                     }
                     // After the main phase: the auxiliary accumulators of this tile, and the main buffer of
                     // the next tile, may be written only once the epilogue has drained the previous tile.
-                    if (ok && i == 0 && t > 0 && !mbar_wait(smem_u32(&sm->tmem_empty), (uint32_t)((t - 1) & 1), abort_flag)) ok = false;
+                    if (ok && i == 0 && t > 0 && !mbar_wait(tmem_empty_bar, (uint32_t)((t - 1) & 1), abort_flag)) ok = false;
                 }
                 if (!ok) break;
-                umma_commit(smem_u32(&sm->tmem_full));
+                umma_commit(tmem_full_bar);
             }
         }
     } else {
@@ -209,76 +259,94 @@ __global__ void __launch_bounds__(kGemmThreads, 1) umma_gemm_kernel(const __grid
             tc_fence_after();
             const int m = m0 + row;
             const uint32_t lane_addr = tmem_base + ((uint32_t)(q * 32) << 16);
+            if (EPI == EPI_PART) {
+                // accumulator columns [0, part_cols) of this split -> workspace
 #pragma unroll 1
-            for (int c = 0; c < kTileN / 32; ++c) {
-                const int nc = n0 + c * 32;
-                if (nc >= p.N) break;            // uniform across the warp
-                uint32_t r0[32];
-                tmem_ld_32x32(lane_addr + (uint32_t)(buf * kTileN + c * 32), r0);
-                if (EPI == EPI_FWD) {
-                    uint32_t r1[32], r2[32];
-                    if (p.has_outlier) tmem_ld_32x32(lane_addr + (uint32_t)(2 * kTileN + c * 32), r1);
-                    if (p.has_lora) tmem_ld_32x32(lane_addr + (uint32_t)(3 * kTileN + c * 32), r2);
+                for (int c = 0; c * 32 < p.part_cols; ++c) {
+                    uint32_t r0[32];
+                    tmem_ld_32x32(lane_addr + (uint32_t)(buf * kTileN + c * 32), r0);
                     tmem_ld_wait();
                     if (m < p.M) {
-                        const float dxm = p.dx[m];
-                        float y[32];
+                        float* out = p.part + ((int64_t)tn * p.M + m) * p.part_ld + c * 32;
 #pragma unroll
-                        for (int j = 0; j < 32; ++j) {
-                            float w = (float)(int)r0[j] * sm->scale_w[buf][c * 32 + j];
-                            if (p.has_outlier) w += (float)(int)r1[j] * sm->scale_o[buf][c * 32 + j];
-                            float v = dxm * w;
-                            if (p.has_lora) v += p.lora_scale * __uint_as_float(r2[j]);
-                            y[j] = v;
-                        }
-                        const bool full = (nc + 32 <= p.N);
-                        if (p.y_f32) {
-                            float* out = reinterpret_cast<float*>(p.Y) + (int64_t)m * p.ldy + nc;
-                            if (full && (p.ldy % 4 == 0)) {
-#pragma unroll
-                                for (int j = 0; j < 32; j += 4) *reinterpret_cast<float4*>(out + j) = make_float4(y[j], y[j + 1], y[j + 2], y[j + 3]);
-                            } else {
-                                for (int j = 0; j < 32; ++j) if (nc + j < p.N) out[j] = y[j];
-                            }
-                        } else {
-                            uint16_t* out = reinterpret_cast<uint16_t*>(p.Y) + (int64_t)m * p.ldy + nc;
-                            if (full && (p.ldy % 8 == 0)) {
-#pragma unroll
-                                for (int j = 0; j < 32; j += 8)
-                                    *reinterpret_cast<uint4*>(out + j) = make_uint4(pack_bf16x2(y[j], y[j + 1]), pack_bf16x2(y[j + 2], y[j + 3]),
-                                                                                    pack_bf16x2(y[j + 4], y[j + 5]), pack_bf16x2(y[j + 6], y[j + 7]));
-                            } else {
-                                for (int j = 0; j < 32; ++j) if (nc + j < p.N) out[j] = (uint16_t)f32_to_bf16_bits(y[j]);
-                            }
-                        }
-                        if (p.dbg_main) {
-                            int32_t* d = p.dbg_main + (int64_t)m * p.N + nc;
-                            for (int j = 0; j < 32; ++j) if (nc + j < p.N) d[j] = (int32_t)r0[j];
-                        }
-                        if (p.dbg_out) {
-                            int32_t* d = p.dbg_out + (int64_t)m * p.N + nc;
-                            for (int j = 0; j < 32; ++j) if (nc + j < p.N) d[j] = p.has_outlier ? (int32_t)r1[j] : 0;
-                        }
+                        for (int j = 0; j < 32; j += 4)
+                            if (c * 32 + j < p.part_cols)
+                                *reinterpret_cast<float4*>(out + j) = make_float4(__uint_as_float(r0[j]), __uint_as_float(r0[j + 1]),
+                                                                                 __uint_as_float(r0[j + 2]), __uint_as_float(r0[j + 3]));
                     }
-                } else {
-                    tmem_ld_wait();
-                    if (m < p.M) {
-                        if (nc < p.p_col0) {
-                            uint16_t* out = p.dX + (int64_t)m * p.lddx + nc;
-                            if (nc + 32 <= p.n_split && (p.lddx % 8 == 0)) {
+                }
+            } else {
+#pragma unroll 1
+                for (int c = 0; c < kTileN / 32; ++c) {
+                    const int nc = n0 + c * 32;
+                    if (nc >= p.N) break;            // uniform across the warp
+                    uint32_t r0[32];
+                    tmem_ld_32x32(lane_addr + (uint32_t)(buf * kTileN + c * 32), r0);
+                    if (EPI == EPI_FWD) {
+                        uint32_t r1[32], r2[32];
+                        if (p.has_outlier) tmem_ld_32x32(lane_addr + (uint32_t)(2 * kTileN + c * 32), r1);
+                        if (p.has_lora) tmem_ld_32x32(lane_addr + (uint32_t)(3 * kTileN + c * 32), r2);
+                        tmem_ld_wait();
+                        if (m < p.M) {
+                            const float dxm = p.dx[m];
+                            float y[32];
 #pragma unroll
-                                for (int j = 0; j < 32; j += 8)
-                                    *reinterpret_cast<uint4*>(out + j) =
-                                        make_uint4(pack_bf16x2(__uint_as_float(r0[j]), __uint_as_float(r0[j + 1])),
-                                                   pack_bf16x2(__uint_as_float(r0[j + 2]), __uint_as_float(r0[j + 3])),
-                                                   pack_bf16x2(__uint_as_float(r0[j + 4]), __uint_as_float(r0[j + 5])),
-                                                   pack_bf16x2(__uint_as_float(r0[j + 6]), __uint_as_float(r0[j + 7])));
-                            } else {
-                                for (int j = 0; j < 32; ++j) if (nc + j < p.n_split) out[j] = (uint16_t)f32_to_bf16_bits(__uint_as_float(r0[j]));
+                            for (int j = 0; j < 32; ++j) {
+                                float w = (float)(int)r0[j] * sm->scale_w[buf][c * 32 + j];
+                                if (p.has_outlier) w += (float)(int)r1[j] * sm->scale_o[buf][c * 32 + j];
+                                float v = dxm * w;
+                                if (p.has_lora) v += p.lora_scale * __uint_as_float(r2[j]);
+                                y[j] = v;
                             }
-                        } else {
-                            float* out = p.P + (int64_t)m * p.ldp + (nc - p.p_col0);
-                            for (int j = 0; j < 32; ++j) if (nc + j < p.N) out[j] = __uint_as_float(r0[j]);
+                            const bool full = (nc + 32 <= p.N);
+                            if (p.y_f32) {
+                                float* out = reinterpret_cast<float*>(p.Y) + (int64_t)m * p.ldy + nc;
+                                if (full && (p.ldy % 4 == 0)) {
+#pragma unroll
+                                    for (int j = 0; j < 32; j += 4) *reinterpret_cast<float4*>(out + j) = make_float4(y[j], y[j + 1], y[j + 2], y[j + 3]);
+                                } else {
+                                    for (int j = 0; j < 32; ++j) if (nc + j < p.N) out[j] = y[j];
+                                }
+                            } else {
+                                uint16_t* out = reinterpret_cast<uint16_t*>(p.Y) + (int64_t)m * p.ldy + nc;
+                                if (full && (p.ldy % 8 == 0)) {
+#pragma unroll
+                                    for (int j = 0; j < 32; j += 8)
+                                        *reinterpret_cast<uint4*>(out + j) = make_uint4(pack_bf16x2(y[j], y[j + 1]), pack_bf16x2(y[j + 2], y[j + 3]),
+                                                                                        pack_bf16x2(y[j + 4], y[j + 5]), pack_bf16x2(y[j + 6], y[j + 7]));
+                                } else {
+                                    for (int j = 0; j < 32; ++j) if (nc + j < p.N) out[j] = (uint16_t)f32_to_bf16_bits(y[j]);
+                                }
+                            }
+                            if (p.dbg_main) {
+                                int32_t* d = p.dbg_main + (int64_t)m * p.N + nc;
+                                for (int j = 0; j < 32; ++j) if (nc + j < p.N) d[j] = (int32_t)r0[j];
+                            }
+                            if (p.dbg_out) {
+                                int32_t* d = p.dbg_out + (int64_t)m * p.N + nc;
+                                for (int j = 0; j < 32; ++j) if (nc + j < p.N) d[j] = p.has_outlier ? (int32_t)r1[j] : 0;
+                            }
+                        }
+                    } else {
+                        tmem_ld_wait();
+                        if (m < p.M) {
+                            if (nc < p.p_col0) {
+                                uint16_t* out = p.dX + (int64_t)m * p.lddx + nc;
+                                if (nc + 32 <= p.n_split && (p.lddx % 8 == 0)) {
+#pragma unroll
+                                    for (int j = 0; j < 32; j += 8)
+                                        *reinterpret_cast<uint4*>(out + j) =
+                                            make_uint4(pack_bf16x2(__uint_as_float(r0[j]), __uint_as_float(r0[j + 1])),
+                                                       pack_bf16x2(__uint_as_float(r0[j + 2]), __uint_as_float(r0[j + 3])),
+                                                       pack_bf16x2(__uint_as_float(r0[j + 4]), __uint_as_float(r0[j + 5])),
+                                                       pack_bf16x2(__uint_as_float(r0[j + 6]), __uint_as_float(r0[j + 7])));
+                                } else {
+                                    for (int j = 0; j < 32; ++j) if (nc + j < p.n_split) out[j] = (uint16_t)f32_to_bf16_bits(__uint_as_float(r0[j]));
+                                }
+                            } else {
+                                float* out = p.P + (int64_t)m * p.ldp + (nc - p.p_col0);
+                                for (int j = 0; j < 32; ++j) if (nc + j < p.N) out[j] = __uint_as_float(r0[j]);
+                            }
                         }
                     }
                 }
