@@ -131,7 +131,8 @@ quaff_status_t quaff_requant_weight_rows(const quaff_bf16* W_O, int64_t ldwo, in
  *   status_opt: optional int32[4] device word, must be zero on entry; see QUAFF_ERR_TIMEOUT
  *   ws: QUAFF_WS_FWD bytes
  * Alignment: all matrix bases 16-byte aligned; ldxq, ldxo, ldwq_main, ldwq multiples of 16;
- * ldx multiple of 8; r multiple of 8, r <= 64; nOp multiple of 32 (0 allowed).
+ * ldx multiple of 8; r multiple of 8, r <= 64; nOp multiple of 32 (0 allowed); with r > 0, K and N
+ * multiples of 8 (A and B are read in place by TMA).
  */
 quaff_status_t quaff_qlinear_fwd(int M, int K, int N,
                                  const int8_t* Xq, int64_t ldxq, const int8_t* xq_O, int64_t ldxo, int nOp,
@@ -156,6 +157,7 @@ quaff_status_t quaff_qlinear_fwd(int M, int K, int N,
  *   dX = dXhat + G A^T                                               [M][K] bf16, lddx (nullable: skipped)
  *   dA = X^T G  [K][r] f32 ;  dB = lora_scale * T^T dY  [r][N] f32   (nullable pair; accumulate != 0 adds)
  *   dY [M][N] bf16, lddy (lddy % 8 == 0);  T [M][r] bf16 from the forward
+ *   Wq, wq_O: 16-byte aligned, ldwq_main and ldwq multiples of 16 (as in the forward)
  *   ws: QUAFF_WS_BWD bytes;  status_opt as in the forward.
  */
 quaff_status_t quaff_qlinear_bwd(int M, int K, int N,

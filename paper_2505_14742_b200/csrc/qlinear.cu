@@ -44,22 +44,64 @@ quaff_status_t make_tmap_2d(CUtensorMap* map, const void* base, int elem_bytes, 
 static cudaEvent_t g_time_start[2] = {nullptr, nullptr};
 static cudaEvent_t g_time_stop[2] = {nullptr, nullptr};
 
-template <int EPI>
+// Tile-processing units (CTAs, or CTA pairs) that can be resident at once.
+template <int EPI, int CTAS, int TN>
+static int gemm_units(int dev) {
+    static int cached[64] = {0};
+    if (cached[dev]) return cached[dev];
+    int units = sm_count() / CTAS;
+    if (CTAS == 2) {
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(sm_count() / 2 * 2);
+        cfg.blockDim = dim3(kGemmThreads);
+        cfg.dynamicSmemBytes = GemmCfg<EPI, CTAS, TN>::kSmemBytes;
+        cudaLaunchAttribute attr;
+        attr.id = cudaLaunchAttributeClusterDimension;
+        attr.val.clusterDim.x = 2; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
+        cfg.attrs = &attr;
+        cfg.numAttrs = 1;
+        int nclusters = 0;
+        if (cudaOccupancyMaxActiveClusters(&nclusters, umma_gemm_kernel<EPI, CTAS, TN>, &cfg) == cudaSuccess && nclusters > 0)
+            units = min(units, nclusters);
+        else
+            cudaGetLastError();
+    }
+    cached[dev] = max(units, 1);
+    return cached[dev];
+}
+
+template <int EPI, int CTAS, int TN>
 static quaff_status_t launch_gemm(const GemmParams& p, cudaStream_t st) {
+    using Cfg = GemmCfg<EPI, CTAS, TN>;
     static bool configured[64] = {false};
     int dev = 0;
     cudaGetDevice(&dev);
-    if (dev >= 0 && dev < 64 && !configured[dev]) {
-        if (cudaFuncSetAttribute(umma_gemm_kernel<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kGemmSmemBytes) != cudaSuccess)
+    if (dev < 0 || dev >= 64) return QUAFF_ERR_CUDA;
+    if (!configured[dev]) {
+        if (cudaFuncSetAttribute(umma_gemm_kernel<EPI, CTAS, TN>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg::kSmemBytes) != cudaSuccess)
             return QUAFF_ERR_CUDA;
         configured[dev] = true;
     }
     const int ntiles = p.tiles_m * p.tiles_n;
     if (ntiles == 0) return QUAFF_OK;
-    const int grid = min(ntiles, sm_count());
+    const int units = min(ntiles, gemm_units<EPI, CTAS, TN>(dev));
     const bool timed = EPI < 2 && g_time_start[EPI % 2] && g_time_stop[EPI % 2];
     if (timed) cudaEventRecord(g_time_start[EPI % 2], st);
-    umma_gemm_kernel<EPI><<<grid, kGemmThreads, kGemmSmemBytes, st>>>(p);
+    if (CTAS == 1) {
+        umma_gemm_kernel<EPI, CTAS, TN><<<units, kGemmThreads, Cfg::kSmemBytes, st>>>(p);
+    } else {
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(units * 2);
+        cfg.blockDim = dim3(kGemmThreads);
+        cfg.dynamicSmemBytes = Cfg::kSmemBytes;
+        cfg.stream = st;
+        cudaLaunchAttribute attr;
+        attr.id = cudaLaunchAttributeClusterDimension;
+        attr.val.clusterDim.x = 2; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
+        cfg.attrs = &attr;
+        cfg.numAttrs = 1;
+        cudaLaunchKernelEx(&cfg, umma_gemm_kernel<EPI, CTAS, TN>, p);
+    }
     const quaff_status_t rc = launch_status();
     if (timed) {
         cudaEventRecord(g_time_stop[EPI % 2], st);
@@ -100,40 +142,52 @@ __global__ void reduce_parts_kernel(const float* __restrict__ part, int S, int C
     dst[idx] = accumulate ? dst[idx] + sum : sum;
 }
 
-// Dequantized, transposed weight for the grad-input GEMM (contraction over n must be contiguous):
-//   rows 0..K-1              : Wext[k][n]          = bf16(Wq[n][k]   * dW[n])
-//   rows K..Kpad-1           : 0   (Kpad = K rounded up to the tile width, so the rows below start a tile)
-//   rows Kpad..Kpad+nOp-1    : Wext[Kpad+i][n]     = bf16(Wq[n][O_i] * dW[n])   (i < nO, else 0)
-//   rows Kpad+nOp..Kpad+2nOp : Wext[Kpad+nOp+i][n] = bf16(wq_O[n][i] * dw_O[n])
-__global__ void __launch_bounds__(256) expand_weight_kernel(const int8_t* __restrict__ Wq, int64_t ldwq_main,
-                                                           const float* __restrict__ dW,
-                                                           const int8_t* __restrict__ wq_O, int64_t ldwq,
-                                                           const float* __restrict__ dw_O,
-                                                           const int32_t* __restrict__ O_idx, int nO, int nOp, int K,
-                                                           int Kpad, int N, uint16_t* __restrict__ Wext, int64_t ldw) {
-    __shared__ uint16_t tile[32][33];
-    const int e0 = blockIdx.x * 32, n0 = blockIdx.y * 32;
-    const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;   // 32 x 8
-    const int Kext = Kpad + 2 * nOp;
-    // load: thread (tx = ext row offset, ty.. = n offset)
-    const int e = e0 + tx;
-    const int8_t* src = nullptr;
-    int64_t lds = 0;
-    const float* sc = nullptr;
-    if (e < K) { src = Wq + e; lds = ldwq_main; sc = dW; }
-    else if (e >= Kpad && e < Kpad + nOp) { const int i = e - Kpad; if (i < nO) { src = Wq + O_idx[i]; lds = ldwq_main; sc = dW; } }
-    else if (e >= Kpad + nOp && e < Kext) { src = wq_O + (e - Kpad - nOp); lds = ldwq; sc = dw_O; }
-    for (int yy = ty; yy < 32; yy += 8) {
-        const int n = n0 + yy;
-        uint16_t v = 0;
-        if (src && n < N) v = (uint16_t)f32_to_bf16_bits(__fmul_rn((float)src[(int64_t)n * lds], sc[n]));
-        tile[tx][yy] = v;
+// Dequantized weight for the grad-input GEMM, in the stored orientation [N][.] (the contraction index n
+// is the row, so the GEMM reads it as an MN-major operand; nothing is transposed):
+//   columns 0..K-1              : Wd[n][k]          = bf16(Wq[n][k]   * dW[n])
+//   columns K..Kpad-1           : 0   (Kpad = K rounded up to the tile width, so the columns below start a tile)
+//   columns Kpad..Kpad+nOp-1    : Wd[n][Kpad+i]     = bf16(Wq[n][O_i] * dW[n])   (i < nO, else 0)
+//   columns Kpad+nOp..Kpad+2nOp : Wd[n][Kpad+nOp+i] = bf16(wq_O[n][i] * dw_O[n])
+// One thread converts 16 consecutive columns of one row (one 128-bit load of codes, two 128-bit stores).
+__global__ void __launch_bounds__(256) dequant_weight_kernel(const int8_t* __restrict__ Wq, int64_t ldwq_main,
+                                                            const float* __restrict__ dW,
+                                                            const int8_t* __restrict__ wq_O, int64_t ldwq,
+                                                            const float* __restrict__ dw_O,
+                                                            const int32_t* __restrict__ O_idx, int nO, int nOp, int K,
+                                                            int Kpad, uint16_t* __restrict__ Wd, int64_t ldwd) {
+    const int n = blockIdx.x;
+    const int c = blockIdx.y * blockDim.x + threadIdx.x;
+    const int k0 = c * 16;
+    if (k0 >= Kpad + 2 * nOp) return;
+    float v[16];
+    if (k0 < Kpad) {
+        const float sc = __ldg(dW + n);
+        const int8_t* src = Wq + (int64_t)n * ldwq_main + k0;
+        if (k0 + 16 <= K) {
+            const uint4 raw = __ldg(reinterpret_cast<const uint4*>(src));
+            const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+#pragma unroll
+            for (int e = 0; e < 16; ++e) v[e] = __fmul_rn((float)(int8_t)((w[e >> 2] >> ((e & 3) * 8)) & 0xFFu), sc);
+        } else {
+#pragma unroll
+            for (int e = 0; e < 16; ++e) v[e] = (k0 + e < K) ? __fmul_rn((float)src[e], sc) : 0.0f;
+        }
+    } else if (k0 < Kpad + nOp) {
+        const float sc = __ldg(dW + n);
+        const int i0 = k0 - Kpad;
+#pragma unroll
+        for (int e = 0; e < 16; ++e)
+            v[e] = (i0 + e < nO) ? __fmul_rn((float)Wq[(int64_t)n * ldwq_main + O_idx[i0 + e]], sc) : 0.0f;
+    } else {
+        const float sc = __ldg(dw_O + n);
+        const uint4 raw = __ldg(reinterpret_cast<const uint4*>(wq_O + (int64_t)n * ldwq + (k0 - Kpad - nOp)));
+        const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+#pragma unroll
+        for (int e = 0; e < 16; ++e) v[e] = __fmul_rn((float)(int8_t)((w[e >> 2] >> ((e & 3) * 8)) & 0xFFu), sc);
     }
-    __syncthreads();
-    for (int yy = ty; yy < 32; yy += 8) {
-        const int er = e0 + yy, n = n0 + tx;
-        if (er < Kext && n < N) Wext[(int64_t)er * ldw + n] = tile[yy][tx];
-    }
+    uint4* out = reinterpret_cast<uint4*>(Wd + (int64_t)n * ldwd + k0);
+    out[0] = make_uint4(pack_bf16x2(v[0], v[1]), pack_bf16x2(v[2], v[3]), pack_bf16x2(v[4], v[5]), pack_bf16x2(v[6], v[7]));
+    out[1] = make_uint4(pack_bf16x2(v[8], v[9]), pack_bf16x2(v[10], v[11]), pack_bf16x2(v[12], v[13]), pack_bf16x2(v[14], v[15]));
 }
 
 // dX[m][O_i] = bf16((P[m][i] + P[m][nOp+i]) / s_i + sum_j G[m][j] A[O_i][j])
@@ -171,7 +225,10 @@ static size_t split_part_bytes(int rows_out, int kc, int r) {
     return (size_t)split_plan(rows_out, kc).S * rows_out * max(r, 1) * 4;
 }
 
-static void fill_phase(GemmPhase& ph, int is_i8, int kext, int acc_slot, int fresh, int tn_limit, int n_mma, int b_box_rows) {
+// One phase of a tile's contraction.  kext = contraction length in elements; box_k = contraction rows
+// of an MN-major box (64 for a full k-block, less for a short LoRA contraction); ctas = CTAs per tile.
+static void fill_phase(GemmPhase& ph, int is_i8, int kext, int acc_slot, int fresh, int tn_limit, int n_mma, int ctas,
+                       int a_mn, int b_mn, int box_k, int b_per_tn) {
     const int kbox = is_i8 ? 128 : 64, kins = is_i8 ? 32 : 16;
     ph.nblk = ceil_div(kext, kbox);
     ph.is_i8 = is_i8;
@@ -179,11 +236,16 @@ static void fill_phase(GemmPhase& ph, int is_i8, int kext, int acc_slot, int fre
     ph.acc_slot = acc_slot;
     ph.fresh = fresh;
     ph.tn_limit = tn_limit;
-    ph.mn_major = 0;
+    ph.a_mn = a_mn;
+    ph.b_mn = b_mn;
     ph.n_mma = n_mma;
-    ph.tx_bytes = (uint32_t)(kOperandBytes + b_box_rows * 128);
+    const int b_cols = n_mma / ctas;                       // B extent per CTA
+    ph.b_boxes = b_mn ? ceil_div(b_cols, 64) : 1;
+    const uint32_t a_bytes = a_mn ? 2u * box_k * 128u : (uint32_t)kABytes;
+    const uint32_t b_bytes = b_mn ? (uint32_t)ph.b_boxes * box_k * 128u : (uint32_t)b_cols * 128u;
+    ph.tx_bytes = a_bytes + b_bytes;
     ph.kblk_per_tn = 0;
-    ph.b_rows_per_tn = kTileN;
+    ph.b_per_tn = b_per_tn;
 }
 
 // part[s][row][j] (f32, row pitch r) = sum over the s-th slice of the contraction of A(row, :) * B(j, :).
@@ -200,46 +262,57 @@ static quaff_status_t skinny_gemm(int mn_major, const void* A, int64_t lda, cons
     if (!mn_major) {
         if ((rc = make_tmap_2d(&ph.map_a, A, 2, rows_out, kc, lda, kTileM, 64)) != QUAFF_OK) return rc;
         if ((rc = make_tmap_2d(&ph.map_b, B, 2, r, kc, ldb, rp, 64)) != QUAFF_OK) return rc;
-        ph.tx_bytes = (uint32_t)(kOperandBytes + rp * 128);
     } else {
         if ((rc = make_tmap_2d(&ph.map_a, A, 2, kc, rows_out, lda, 64, 64)) != QUAFF_OK) return rc;
         if ((rc = make_tmap_2d(&ph.map_b, B, 2, kc, r, ldb, 64, 64)) != QUAFF_OK) return rc;
-        ph.tx_bytes = (uint32_t)(kOperandBytes + 8192);
     }
-    ph.nblk = sp.kblk; ph.is_i8 = 0; ph.nmma_last = 4; ph.acc_slot = 0; ph.fresh = 1; ph.tn_limit = 1 << 30;
-    ph.mn_major = mn_major; ph.n_mma = rp; ph.kblk_per_tn = sp.kblk; ph.b_rows_per_tn = 0;
+    fill_phase(ph, 0, 64, 0, 1, 1 << 30, rp, 1, mn_major, mn_major, 64, 0);
+    ph.nblk = sp.kblk; ph.nmma_last = 4; ph.kblk_per_tn = sp.kblk;
     p.nphases = 1;
     p.M = rows_out; p.N = rp;
     p.tiles_m = ceil_div(rows_out, kTileM); p.tiles_n = sp.S;
     p.status = status;
     p.part = part; p.part_ld = r; p.part_cols = r;
     *S_out = sp.S;
-    return launch_gemm<EPI_PART>(p, st);
+    return launch_gemm<EPI_PART, 1, 128>(p, st);
 }
 
-struct FwdWorkspace { size_t off_bt, off_at, off_part, total; };
+struct FwdWorkspace { size_t off_at, off_part, total; };
 static FwdWorkspace fwd_workspace(int M, int K, int N, int r) {
     FwdWorkspace w;
     const int rp = pad16(max(r, 1));
     size_t off = 0;
-    w.off_bt = off;   off += round_up((size_t)N * rp * 2, 256);          // B^T, K-major LoRA-up operand
     w.off_at = off;   off += round_up((size_t)rp * K * 2, 256);          // A^T, K-major LoRA-down operand
     w.off_part = off; off += round_up(split_part_bytes(M, K, r), 256);   // split-K partials of T = X A
     w.total = off;
     return w;
 }
 
+// Output-column tile of the grad-input GEMM: a 256-wide MMA runs at nearly twice the rate of a 128-wide
+// one (measured), 128 fills the machine better when there are few tiles.  Cost model: waves x tile
+// width, 128-wide tiles 1.8x dearer per column.
+static int bwd_tile_n(int M, int K, int nOp) {
+    const int units = kPlanSMs / 2;
+    const int tm = ceil_div(M, 2 * kTileM);
+    const double c256 = (double)ceil_div(tm * (ceil_div(K, 256) + (nOp > 0)), units) * 256.0;
+    const double c128 = (double)ceil_div(tm * (ceil_div(K, 128) + (nOp > 0)), units) * 128.0 * 1.8;
+    return c256 <= c128 ? 256 : 128;
+}
+
 struct BwdWorkspace {
-    size_t off_wext, off_g, off_p, off_part, total;
-    int64_t ldw;  // row pitch of Wext in elements
+    size_t off_wd, off_g, off_p, off_part, total;
+    int tile_n;       // output-column tile of the grad-input GEMM
+    int Kpad;         // K rounded up to tile_n
+    int64_t ldwd;     // row pitch of Wd in elements
 };
 
 static BwdWorkspace bwd_workspace(int M, int K, int N, int nOp, int r) {
     BwdWorkspace w;
-    w.ldw = (int64_t)round_up((size_t)N, 8);
+    w.tile_n = bwd_tile_n(M, K, nOp);
+    w.Kpad = ceil_div(K, w.tile_n) * w.tile_n;
+    w.ldwd = (int64_t)w.Kpad + 2 * nOp;
     size_t off = 0;
-    const size_t kpad = round_up((size_t)K, kTileN);
-    w.off_wext = off; off += round_up((kpad + 2 * (size_t)nOp) * w.ldw * 2, 256);
+    w.off_wd = off;   off += round_up((size_t)N * (size_t)w.ldwd * 2, 256);
     w.off_g = off;    off += round_up((size_t)M * (size_t)max(r, 1) * 2, 256);
     w.off_p = off;    off += round_up((size_t)M * (size_t)max(2 * nOp, 1) * 4, 256);
     w.off_part = off;
@@ -299,10 +372,10 @@ extern "C" quaff_status_t quaff_qlinear_fwd(int M, int K, int N, const int8_t* X
     QUAFF_RETURN_IF(r > 0 && (!X || !A || !B || !T_out || ldx < K), QUAFF_ERR_INVALID_ARG);
     QUAFF_RETURN_IF(y_dtype != QUAFF_BF16 && y_dtype != QUAFF_F32, QUAFF_ERR_INVALID_ARG);
     QUAFF_RETURN_IF((nOp % 32) || (r % 8) || r > 64, QUAFF_ERR_UNSUPPORTED_SHAPE);
-    QUAFF_RETURN_IF(r > 0 && (K % 8), QUAFF_ERR_UNSUPPORTED_SHAPE);
+    QUAFF_RETURN_IF(r > 0 && ((K % 8) || (N % 8)), QUAFF_ERR_UNSUPPORTED_SHAPE);
     QUAFF_RETURN_IF(!aligned16(Xq) || !aligned16(Wq) || (ldxq % 16) || (ldwq_main % 16), QUAFF_ERR_ALIGNMENT);
     QUAFF_RETURN_IF(nOp > 0 && (!aligned16(xq_O) || !aligned16(wq_O) || (ldxo % 16) || (ldwq % 16)), QUAFF_ERR_ALIGNMENT);
-    QUAFF_RETURN_IF(r > 0 && (!aligned16(X) || !aligned16(T_out) || (ldx % 8)), QUAFF_ERR_ALIGNMENT);
+    QUAFF_RETURN_IF(r > 0 && (!aligned16(X) || !aligned16(T_out) || !aligned16(B) || (ldx % 8)), QUAFF_ERR_ALIGNMENT);
     QUAFF_RETURN_IF(!aligned16(Y), QUAFF_ERR_ALIGNMENT);
     const FwdWorkspace w = fwd_workspace(M, K, N, r);
     QUAFF_RETURN_IF(r > 0 && (!ws || !aligned16(ws) || ws_bytes < w.total), QUAFF_ERR_WORKSPACE_TOO_SMALL);
@@ -310,9 +383,9 @@ extern "C" quaff_status_t quaff_qlinear_fwd(int M, int K, int N, const int8_t* X
     cudaStream_t st = (cudaStream_t)stream;
     const int rp = pad16(r);
     unsigned char* base = reinterpret_cast<unsigned char*>(ws);
-    uint16_t* Bt = reinterpret_cast<uint16_t*>(base + w.off_bt);
     uint16_t* At = reinterpret_cast<uint16_t*>(base + w.off_at);
     float* part = reinterpret_cast<float*>(base + w.off_part);
+    constexpr int TN = 128, CTAS = 2;
 
     GemmParams p;
     memset(&p, 0, sizeof(p));
@@ -321,40 +394,38 @@ extern "C" quaff_status_t quaff_qlinear_fwd(int M, int K, int N, const int8_t* X
     {   // main: acc1 = Xq Wq^T over K
         GemmPhase& ph = p.ph[np++];
         if ((rc = make_tmap_2d(&ph.map_a, Xq, 1, M, K, ldxq, kTileM, 128)) != QUAFF_OK) return rc;
-        if ((rc = make_tmap_2d(&ph.map_b, Wq, 1, N, K, ldwq_main, kTileN, 128)) != QUAFF_OK) return rc;
-        fill_phase(ph, 1, K, 0, 1, 1 << 30, kTileN, kTileN);
+        if ((rc = make_tmap_2d(&ph.map_b, Wq, 1, N, K, ldwq_main, TN / CTAS, 128)) != QUAFF_OK) return rc;
+        fill_phase(ph, 1, K, 0, 1, 1 << 30, TN, CTAS, 0, 0, 64, TN);
     }
     if (nOp > 0) {   // outlier: acc2 = xq_O wq_O^T over nOp
         GemmPhase& ph = p.ph[np++];
         if ((rc = make_tmap_2d(&ph.map_a, xq_O, 1, M, nOp, ldxo, kTileM, 128)) != QUAFF_OK) return rc;
-        if ((rc = make_tmap_2d(&ph.map_b, wq_O, 1, N, nOp, ldwq, kTileN, 128)) != QUAFF_OK) return rc;
-        fill_phase(ph, 1, nOp, 1, 1, 1 << 30, kTileN, kTileN);
+        if ((rc = make_tmap_2d(&ph.map_b, wq_O, 1, N, nOp, ldwq, TN / CTAS, 128)) != QUAFF_OK) return rc;
+        fill_phase(ph, 1, nOp, 1, 1, 1 << 30, TN, CTAS, 0, 0, 64, TN);
     }
     if (r > 0) {
         // LoRA down-projection T = bf16(X A): split-K tensor-core GEMM over K, then a reduction to bf16
         transpose_pad_kernel<<<ceil_div(K * rp, 256), 256, 0, st>>>(A, K, r, At, K);   // At[j][k] = A[k][j]
         if ((rc = launch_status()) != QUAFF_OK) return rc;
-        transpose_pad_kernel<<<ceil_div(N * rp, 256), 256, 0, st>>>(B, r, N, Bt, rp);  // Bt[n][j] = B[j][n]
-        if ((rc = launch_status()) != QUAFF_OK) return rc;
         int S = 1;
         if ((rc = skinny_gemm(0, X, ldx, At, K, M, K, r, part, status_opt, st, &S)) != QUAFF_OK) return rc;
         reduce_parts_bf16_kernel<<<ceil_div(M * r, 256), 256, 0, st>>>(part, S, M, r, 1.0f, T_out);
         if ((rc = launch_status()) != QUAFF_OK) return rc;
-        // LoRA up: acc3 = T Bt^T over r
+        // LoRA up: acc3 = T B over r; B [r][N] is read in place as an MN-major operand (rows = contraction)
         GemmPhase& ph = p.ph[np++];
         if ((rc = make_tmap_2d(&ph.map_a, T_out, 2, M, r, r, kTileM, 64)) != QUAFF_OK) return rc;
-        if ((rc = make_tmap_2d(&ph.map_b, Bt, 2, N, rp, rp, kTileN, 64)) != QUAFF_OK) return rc;
-        fill_phase(ph, 0, rp, 2, 1, 1 << 30, kTileN, kTileN);
+        if ((rc = make_tmap_2d(&ph.map_b, B, 2, r, N, N, rp, 64)) != QUAFF_OK) return rc;
+        fill_phase(ph, 0, rp, 2, 1, 1 << 30, TN, CTAS, 0, 1, rp, TN);
     }
     p.nphases = np;
     p.M = M; p.N = N;
-    p.tiles_m = ceil_div(M, kTileM); p.tiles_n = ceil_div(N, kTileN);
+    p.tiles_m = ceil_div(M, kTileM * CTAS); p.tiles_n = ceil_div(N, TN);
     p.status = status_opt;
     p.dx = dx; p.dW = dW; p.dw_O = dw_O; p.lora_scale = lora_scale;
     p.has_outlier = nOp > 0; p.has_lora = r > 0;
     p.Y = Y; p.ldy = ldy; p.y_f32 = (y_dtype == QUAFF_F32);
     p.dbg_main = dbg_acc_main; p.dbg_out = dbg_acc_out;
-    return launch_gemm<EPI_FWD>(p, st);
+    return launch_gemm<EPI_FWD, CTAS, TN>(p, st);
 }
 
 extern "C" quaff_status_t quaff_qlinear_bwd(int M, int K, int N, const quaff_bf16* dY, int64_t lddy, const int8_t* Wq,
@@ -374,6 +445,8 @@ extern "C" quaff_status_t quaff_qlinear_bwd(int M, int K, int N, const quaff_bf1
     QUAFF_RETURN_IF((nOp % 32) || (r % 8) || r > 64, QUAFF_ERR_UNSUPPORTED_SHAPE);
     QUAFF_RETURN_IF(r > 0 && (N % 8), QUAFF_ERR_UNSUPPORTED_SHAPE);
     QUAFF_RETURN_IF(!aligned16(dY) || (lddy % 8), QUAFF_ERR_ALIGNMENT);
+    QUAFF_RETURN_IF(!aligned16(Wq) || (ldwq_main % 16), QUAFF_ERR_ALIGNMENT);
+    QUAFF_RETURN_IF(nOp > 0 && (!aligned16(wq_O) || (ldwq % 16)), QUAFF_ERR_ALIGNMENT);
     QUAFF_RETURN_IF(dX && (!aligned16(dX) || (lddx % 8)), QUAFF_ERR_ALIGNMENT);
     QUAFF_RETURN_IF(r > 0 && (!aligned16(A) || !aligned16(B)), QUAFF_ERR_ALIGNMENT);
     QUAFF_RETURN_IF(r > 0 && dA && (!aligned16(X) || !aligned16(T) || (ldx % 8)), QUAFF_ERR_ALIGNMENT);
@@ -382,7 +455,7 @@ extern "C" quaff_status_t quaff_qlinear_bwd(int M, int K, int N, const quaff_bf1
     if (M == 0) return QUAFF_OK;
     cudaStream_t st = (cudaStream_t)stream;
     unsigned char* base = reinterpret_cast<unsigned char*>(ws);
-    uint16_t* Wext = reinterpret_cast<uint16_t*>(base + w.off_wext);
+    uint16_t* Wd = reinterpret_cast<uint16_t*>(base + w.off_wd);
     uint16_t* G = reinterpret_cast<uint16_t*>(base + w.off_g);
     float* P = reinterpret_cast<float*>(base + w.off_p);
     float* part = reinterpret_cast<float*>(base + w.off_part);
@@ -395,25 +468,27 @@ extern "C" quaff_status_t quaff_qlinear_bwd(int M, int K, int N, const quaff_bf1
         if ((rc = launch_status()) != QUAFF_OK) return rc;
     }
     if (dX) {
-        const int Kpad = ceil_div(K, kTileN) * kTileN;
+        constexpr int CTAS = 2;
+        const int TN = w.tile_n, Kpad = w.Kpad;
         const int Kext = nOp > 0 ? Kpad + 2 * nOp : K;
-        expand_weight_kernel<<<dim3(ceil_div(Kext, 32), ceil_div(N, 32)), 256, 0, st>>>(Wq, ldwq_main, dW, wq_O, ldwq, dw_O,
-                                                                                      O_idx, nO, nOp, K, Kpad, N, Wext, w.ldw);
+        const int chunks = (Kpad + 2 * nOp) / 16;
+        dequant_weight_kernel<<<dim3(N, ceil_div(chunks, 256)), 256, 0, st>>>(Wq, ldwq_main, dW, wq_O, ldwq, dw_O, O_idx, nO, nOp, K,
+                                                                            Kpad, Wd, w.ldwd);
         if ((rc = launch_status()) != QUAFF_OK) return rc;
         GemmParams p;
         memset(&p, 0, sizeof(p));
         int np = 0;
-        {   // main: dY Wext^T over N
+        {   // main: dY Wd over N; Wd [N][Kext] is MN-major for this contraction (rows = n)
             GemmPhase& ph = p.ph[np++];
             if ((rc = make_tmap_2d(&ph.map_a, dY, 2, M, N, lddy, kTileM, 64)) != QUAFF_OK) return rc;
-            if ((rc = make_tmap_2d(&ph.map_b, Wext, 2, Kext, N, w.ldw, kTileN, 64)) != QUAFF_OK) return rc;
-            fill_phase(ph, 0, N, 0, 1, 1 << 30, kTileN, kTileN);
+            if ((rc = make_tmap_2d(&ph.map_b, Wd, 2, N, Kext, w.ldwd, 64, 64)) != QUAFF_OK) return rc;
+            fill_phase(ph, 0, N, 0, 1, 1 << 30, TN, CTAS, 0, 1, 64, TN);
         }
         if (r > 0) {   // + G A^T over r, only for the real dX columns
             GemmPhase& ph = p.ph[np++];
             if ((rc = make_tmap_2d(&ph.map_a, G, 2, M, r, r, kTileM, 64)) != QUAFF_OK) return rc;
-            if ((rc = make_tmap_2d(&ph.map_b, A, 2, K, r, r, kTileN, 64)) != QUAFF_OK) return rc;
-            fill_phase(ph, 0, pad16(r), 0, 0, ceil_div(K, kTileN), kTileN, kTileN);
+            if ((rc = make_tmap_2d(&ph.map_b, A, 2, K, r, r, TN / CTAS, 64)) != QUAFF_OK) return rc;
+            fill_phase(ph, 0, pad16(r), 0, 0, ceil_div(K, TN), TN, CTAS, 0, 0, 64, TN);
         }
         p.nphases = np;
         p.M = M;
@@ -421,11 +496,12 @@ extern "C" quaff_status_t quaff_qlinear_bwd(int M, int K, int N, const quaff_bf1
         p.n_split = K;
         p.p_col0 = Kpad;
         p.N = Kext;
-        p.tiles_m = ceil_div(M, kTileM);
-        p.tiles_n = ceil_div(p.N, kTileN);
+        p.tiles_m = ceil_div(M, kTileM * CTAS);
+        p.tiles_n = ceil_div(p.N, TN);
         p.status = status_opt;
         p.dX = dX; p.lddx = lddx; p.P = P; p.ldp = 2 * nOp;
-        if ((rc = launch_gemm<EPI_BWD>(p, st)) != QUAFF_OK) return rc;
+        rc = TN == 256 ? launch_gemm<EPI_BWD, CTAS, 256>(p, st) : launch_gemm<EPI_BWD, CTAS, 128>(p, st);
+        if (rc != QUAFF_OK) return rc;
         if (nO > 0) {
             bwd_fixup_kernel<<<ceil_div(M * nO, 256), 256, 0, st>>>(P, 2 * nOp, M, nO, nOp, O_idx, s_O, G, A, r, dX, lddx);
             if ((rc = launch_status()) != QUAFF_OK) return rc;

@@ -5,20 +5,33 @@
 //   warp 1      : TMEM allocation + MMA issue (one elected lane) - tcgen05.mma, accumulators in TMEM
 //   warps 2..5  : epilogue - tcgen05.ld of the finished accumulators, dequantization / conversion, stores
 //
-// An output tile is 128 rows x up to 128 columns.  Its contraction is a list of up to three PHASES,
+// Template parameters: EPI (which epilogue), CTAS (1, or 2 = a CTA pair on two SMs that shares one
+// 256-row output tile through tcgen05 cta_group::2) and TN (output columns per tile, 128 or 256).
+//
+// CTA pair (CTAS = 2, a cluster of two): each CTA loads its own 128 rows of A and its own half
+// (TN / 2 output columns) of B into its own shared memory, at the same offsets in both CTAs.  The
+// TMA loads of both CTAs signal the "full" barrier of the leader (cluster rank 0), whose MMA warp
+// issues every tcgen05.mma for the pair; the accumulator rows 0..127 land in the leader's TMEM and
+// rows 128..255 in its peer's.  tcgen05.commit multicasts the "stage free" and "accumulator ready"
+// arrivals to both CTAs; the peer's epilogue warps report "accumulator drained" to the leader with a
+// remote mbarrier arrive.  Per output element each SM reads half as many operand bytes as it would
+// alone, which is what lets the stage ring cover the latency of the loads.  No TMA multicast anywhere.
+//
+// An output tile is (128 * CTAS) rows x TN columns.  Its contraction is a list of up to three PHASES,
 // each a run of k-blocks with its own pair of tensor maps, operand type and accumulator:
 //   forward : main INT8 (over K) -> slot 0 | outlier INT8 (over nOp) -> slot 1 | LoRA bf16 (over r) -> slot 2
 //   backward: main bf16 (over N) -> slot 0 | LoRA bf16 (over r) -> slot 0 (accumulating)
 //   skinny  : one bf16 phase over a slice of the contraction (split-K); partial sums go to a workspace
-// Every k-block is one stage: an A tile (128 rows) and a B tile (up to 128 rows) of 128 bytes per row.
-// Operands are either K-major (rows = output index, the 128 bytes run along the contraction) or
-// MN-major (rows = contraction index, the 128 bytes run along the output index; used where the
-// contraction is the slow axis of the caller's matrix, i.e. X^T G and T^T dY).
+// Every k-block is one stage: 128 bytes of contraction per row (128 INT8 or 64 bf16 elements).
+// Each operand is either K-major (rows = output index, the 128 bytes run along the contraction) or
+// MN-major (rows = contraction index, the 128 bytes run along 64 output indices; used where the
+// contraction is the slow axis of the caller's matrix: the dequantized weight and LoRA B in their
+// stored orientation, X^T G and T^T dY).
 // Tails need no special case: TMA zero-fills out-of-range rows and columns, and the epilogue masks stores.
 //
-// TMEM (512 columns): slot 0 is double-buffered at columns [0,128) and [128,256) so the main
-// contraction of tile t+1 overlaps the epilogue of tile t; slots 1 and 2 live at [256,384) and
-// [384,512) and are written only after the epilogue of the previous tile has drained them.
+// TMEM (512 columns): slot 0 is double-buffered at columns [0,TN) and [TN,2TN) so the main
+// contraction of tile t+1 overlaps the epilogue of tile t; with TN = 128, slots 1 and 2 live at
+// [256,384) and [384,512) and are written only after the epilogue of the previous tile has drained them.
 //
 // The producer and the MMA issuer are single threads; their per-k-block instruction count bounds the
 // tensor-pipe utilisation, so everything that does not change inside a phase is hoisted out of the
@@ -32,13 +45,13 @@
 
 namespace quaff {
 
-constexpr int kTileM = 128;
-constexpr int kTileN = 128;
-constexpr int kStages = 6;
-constexpr int kOperandBytes = 128 * 128;          // one operand tile: 128 rows x 128 bytes
-constexpr int kStageBytes = 2 * kOperandBytes;
+constexpr int kTileM = 128;                       // accumulator rows per CTA
+constexpr int kABytes = 128 * 128;                // A region of a stage: 128 rows x 128 bytes
+constexpr int kAtomBytes = 64 * 128;              // one MN-major box: 64 contraction rows x 128 bytes
 constexpr int kGemmThreads = 192;
 constexpr int kMaxPhases = 3;
+constexpr int kMaxStages = 12;
+constexpr int kSmemLimit = 232448;                // opt-in dynamic shared memory per CTA on sm_100
 
 struct GemmPhase {
     CUtensorMap map_a;   // K-major: [rows = output rows][cols = contraction]; MN-major: [rows = contraction][cols = output rows]
@@ -49,11 +62,12 @@ struct GemmPhase {
     int acc_slot;        // 0 main (double-buffered), 1, 2 auxiliary
     int fresh;           // 1: the first MMA of the phase overwrites the accumulator
     int tn_limit;        // the phase runs only for column tiles tn < tn_limit
-    int mn_major;        // 0: both operands K-major; 1: both MN-major
-    int n_mma;           // N of the MMA instruction (multiple of 16, <= 128)
-    uint32_t tx_bytes;   // bytes that land in one stage
+    int a_mn, b_mn;      // operand is MN-major (1) or K-major (0)
+    int n_mma;           // N of the MMA instruction (multiple of 16, <= 256); each CTA of a pair supplies n_mma / CTAS columns of B
+    int b_boxes;         // MN-major B: boxes of 64 output columns per CTA
+    uint32_t tx_bytes;   // bytes that land in one stage of ONE CTA
     int kblk_per_tn;     // split-K: first k-block of a tile is tn * kblk_per_tn (0 otherwise)
-    int b_rows_per_tn;   // B row offset per tn (128 for an ordinary GEMM, 0 for split-K)
+    int b_per_tn;        // B offset (rows if K-major, columns if MN-major) per tn: the tile width, or 0 for split-K
 };
 
 enum { EPI_FWD = 0, EPI_BWD = 1, EPI_PART = 2 };
@@ -90,17 +104,24 @@ struct GemmParams {
 };
 
 struct GemmSmem {
-    uint64_t full[kStages];
-    uint64_t empty[kStages];
+    uint64_t full[kMaxStages];
+    uint64_t empty[kMaxStages];
     uint64_t tmem_full;
     uint64_t tmem_empty;
     uint32_t tmem_base;
     int abort_flag;
-    float scale_w[2][kTileN];
-    float scale_o[2][kTileN];
 };
 
-constexpr size_t kGemmSmemBytes = 1024 + (size_t)kStages * kStageBytes + sizeof(GemmSmem);
+template <int EPI, int CTAS, int TN>
+struct GemmCfg {
+    static constexpr int kBBytes = (TN / CTAS) * 128;                // B region of a stage, per CTA
+    static constexpr int kStageBytes = kABytes + kBBytes;
+    static constexpr int kScaleBytes = (EPI == EPI_FWD) ? 2 * 2 * TN * 4 : 0;   // [2 buffers][dW | dw_O][TN]
+    static constexpr int kFixed = 1024 + (int)sizeof(GemmSmem) + kScaleBytes;
+    static constexpr int kStagesFit = (kSmemLimit - kFixed) / kStageBytes;
+    static constexpr int kStages = kStagesFit < kMaxStages ? kStagesFit : kMaxStages;
+    static constexpr size_t kSmemBytes = (size_t)kFixed + (size_t)kStages * kStageBytes;
+};
 
 // high word of the shared-memory matrix descriptor: stride byte offset 1024 (8 rows x 128 bytes),
 // descriptor version 1, SWIZZLE_128B
@@ -110,42 +131,58 @@ __device__ __forceinline__ uint64_t make_desc(uint32_t lo, uint32_t hi) {
     return (static_cast<uint64_t>(hi) << 32) | lo;
 }
 
-template <int EPI>
+template <int EPI, int CTAS, int TN>
 __global__ void __launch_bounds__(kGemmThreads, 1) umma_gemm_kernel(const __grid_constant__ GemmParams p) {
+    using Cfg = GemmCfg<EPI, CTAS, TN>;
+    constexpr int kStages = Cfg::kStages;
+    constexpr int kStageBytes = Cfg::kStageBytes;
+    static_assert(CTAS == 1 || CTAS == 2, "one CTA or a CTA pair");
+    static_assert(TN == 128 || (TN == 256 && EPI == EPI_BWD), "three accumulators fit TMEM only at TN = 128");
+
     extern __shared__ unsigned char smem_dyn[];
     const uint32_t raw = smem_u32(smem_dyn);
     const uint32_t tiles_base = (raw + 1023u) & ~1023u;
     unsigned char* aligned = smem_dyn + (tiles_base - raw);
     GemmSmem* sm = reinterpret_cast<GemmSmem*>(aligned + (size_t)kStages * kStageBytes);
+    float* scales = reinterpret_cast<float*>(sm + 1);                 // EPI_FWD only: [2][2][TN]
     volatile int* abort_flag = &sm->abort_flag;
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
+    const uint32_t rank = CTAS == 2 ? cluster_ctarank() : 0u;        // 0 = leader of the pair
+    const int unit = CTAS == 2 ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;           // tile-processing unit (CTA or pair)
+    const int nunits = CTAS == 2 ? (int)(gridDim.x >> 1) : (int)gridDim.x;
     const int ntiles = p.tiles_m * p.tiles_n;
     const uint32_t full0 = smem_u32(&sm->full[0]);
     const uint32_t empty0 = smem_u32(&sm->empty[0]);
+    const uint32_t tmem_full_bar = smem_u32(&sm->tmem_full);
+    const uint32_t tmem_empty_bar = smem_u32(&sm->tmem_empty);
+    // barriers of the leader as seen from this CTA (its own, when it is the leader)
+    const uint32_t lead_full0 = CTAS == 2 ? mapa_shared(full0, 0) : full0;
+    const uint32_t lead_tmem_empty = CTAS == 2 ? mapa_shared(tmem_empty_bar, 0) : tmem_empty_bar;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; ++s) {
             mbar_init(full0 + 8u * s, 1);
             mbar_init(empty0 + 8u * s, 1);
         }
-        mbar_init(smem_u32(&sm->tmem_full), 1);
-        mbar_init(smem_u32(&sm->tmem_empty), 4);
+        mbar_init(tmem_full_bar, 1);
+        mbar_init(tmem_empty_bar, 4 * CTAS);
         sm->abort_flag = 0;
         fence_barrier_init();
     }
     if (warp == 1) {
-        tmem_alloc(smem_u32(&sm->tmem_base), 512);
-        tmem_relinquish();
+        tmem_alloc<CTAS>(smem_u32(&sm->tmem_base), 512);
+        tmem_relinquish<CTAS>();
     }
     tc_fence_before();
     __syncthreads();
+    if (CTAS == 2) cluster_sync();      // the peer's barriers exist before anything can signal them
     tc_fence_after();
     const uint32_t tmem_base = sm->tmem_base;
 
     if (warp == 0) {
-        // ------------------------------------------------------------------ TMA producer
+        // ------------------------------------------------------------------ TMA producer (both CTAs of a pair)
         if (elect_one()) {
             for (int i = 0; i < p.nphases; ++i) {
                 prefetch_tmap(&p.ph[i].map_a);
@@ -153,32 +190,37 @@ __global__ void __launch_bounds__(kGemmThreads, 1) umma_gemm_kernel(const __grid
             }
             uint32_t stage = 0, phase = 0;
             bool ok = true;
-            for (int tile = blockIdx.x; tile < ntiles && ok; tile += gridDim.x) {
+            for (int tile = unit; tile < ntiles && ok; tile += nunits) {
                 const int tm = tile % p.tiles_m, tn = tile / p.tiles_m;
-                const int m0 = tm * kTileM;
+                const int m0 = tm * (kTileM * CTAS) + (int)rank * kTileM;
                 for (int i = 0; i < p.nphases && ok; ++i) {
                     const GemmPhase& ph = p.ph[i];
                     if (tn >= ph.tn_limit) continue;
                     const CUtensorMap* map_a = &ph.map_a;
                     const CUtensorMap* map_b = &ph.map_b;
                     const int nblk = ph.nblk;
-                    const uint32_t tx = ph.tx_bytes;
-                    const int n0 = tn * ph.b_rows_per_tn;
+                    const uint32_t tx = ph.tx_bytes * CTAS;
+                    const int n0 = tn * ph.b_per_tn + (int)rank * (ph.n_mma / CTAS);
                     const int kstep = ph.is_i8 ? 128 : 64;
                     int kc = tn * ph.kblk_per_tn * kstep;      // contraction coordinate of the next block
-                    const bool mn = ph.mn_major != 0;
+                    const bool a_mn = ph.a_mn != 0, b_mn = ph.b_mn != 0;
+                    const int b_boxes = ph.b_boxes;
                     for (int b = 0; b < nblk; ++b, kc += kstep) {
                         if (!mbar_wait(empty0 + 8u * stage, phase ^ 1u, abort_flag)) { ok = false; break; }
-                        const uint32_t bar = full0 + 8u * stage;
+                        const uint32_t bar = lead_full0 + 8u * stage;
                         const uint32_t dst = tiles_base + stage * kStageBytes;
-                        mbar_arrive_expect_tx(bar, tx);
-                        if (!mn) {
-                            tma_load_2d(dst, map_a, kc, m0, bar);
-                            tma_load_2d(dst + kOperandBytes, map_b, kc, n0, bar);
-                        } else {   // 64 output indices x 64 contraction rows per box
-                            tma_load_2d(dst, map_a, m0, kc, bar);
-                            tma_load_2d(dst + 8192, map_a, m0 + 64, kc, bar);
-                            tma_load_2d(dst + kOperandBytes, map_b, n0, kc, bar);
+                        if (rank == 0) mbar_arrive_expect_tx(full0 + 8u * stage, tx);
+                        if (!a_mn) {
+                            tma_load_2d<CTAS>(dst, map_a, kc, m0, bar);
+                        } else {   // two boxes of 64 output rows x 64 contraction rows
+                            tma_load_2d<CTAS>(dst, map_a, m0, kc, bar);
+                            tma_load_2d<CTAS>(dst + kAtomBytes, map_a, m0 + 64, kc, bar);
+                        }
+                        if (!b_mn) {
+                            tma_load_2d<CTAS>(dst + kABytes, map_b, kc, n0, bar);
+                        } else {
+                            for (int x = 0; x < b_boxes; ++x)
+                                tma_load_2d<CTAS>(dst + kABytes + x * kAtomBytes, map_b, n0 + 64 * x, kc, bar);
                         }
                         if (++stage == kStages) { stage = 0; phase ^= 1u; }
                     }
@@ -186,47 +228,47 @@ __global__ void __launch_bounds__(kGemmThreads, 1) umma_gemm_kernel(const __grid
             }
         }
     } else if (warp == 1) {
-        // ------------------------------------------------------------------ MMA issuer
-        if (elect_one()) {
+        // ------------------------------------------------------------------ MMA issuer (the leader's, for the pair)
+        if (rank == 0 && elect_one()) {
             uint32_t stage = 0, phase = 0;
             bool ok = true;
             int t = 0;
-            const uint32_t tmem_empty_bar = smem_u32(&sm->tmem_empty);
-            const uint32_t tmem_full_bar = smem_u32(&sm->tmem_full);
-            for (int tile = blockIdx.x; tile < ntiles && ok; tile += gridDim.x, ++t) {
+            for (int tile = unit; tile < ntiles && ok; tile += nunits, ++t) {
                 const int tn = tile / p.tiles_m;
                 for (int i = 0; i < p.nphases && ok; ++i) {
                     const GemmPhase& ph = p.ph[i];
                     if (tn < ph.tn_limit) {
-                        const uint32_t acc = tmem_base + (ph.acc_slot == 0 ? (uint32_t)((t & 1) * kTileN) : (uint32_t)((ph.acc_slot + 1) * kTileN));
+                        const uint32_t acc = tmem_base + (ph.acc_slot == 0 ? (uint32_t)((t & 1) * TN) : (uint32_t)((ph.acc_slot + 1) * TN));
                         const int nblk = ph.nblk;
                         const int nmma_last = ph.nmma_last;
                         const bool i8 = ph.is_i8 != 0;
-                        const bool mn = ph.mn_major != 0;
-                        // K-major: the leading byte offset is unused (encoded 1), a 32-byte K step inside the swizzled row.
-                        // MN-major: 64-wide output atoms are 8192 bytes apart (A tile = two TMA boxes); one MMA consumes
-                        // 16 contraction rows = 2048 bytes.
-                        const uint32_t lbo = mn ? ((8192u >> 4) << 16) : (1u << 16);
-                        const uint32_t kadv = mn ? (2048u >> 4) : (32u >> 4);
-                        const uint32_t idesc = (i8 ? umma_idesc(kCFmtS32, kFmtS8, kTileM, 0) : umma_idesc(kCFmtF32, kFmtBF16, kTileM, 0)) |
-                                               ((uint32_t)(ph.n_mma >> 3) << 17) | (mn ? ((1u << 15) | (1u << 16)) : 0u);
+                        // K-major: the leading byte offset is unused (encoded 1), one MMA advances 32 bytes inside the
+                        // swizzled row.  MN-major: boxes of 64 output indices are kAtomBytes apart (leading byte
+                        // offset); one MMA consumes 16 contraction rows = 2048 bytes.
+                        const uint32_t a_lbo = ph.a_mn ? ((uint32_t)(kAtomBytes >> 4) << 16) : (1u << 16);
+                        const uint32_t b_lbo = ph.b_mn ? ((uint32_t)(kAtomBytes >> 4) << 16) : (1u << 16);
+                        const uint32_t a_kadv = ph.a_mn ? (2048u >> 4) : (32u >> 4);
+                        const uint32_t b_kadv = ph.b_mn ? (2048u >> 4) : (32u >> 4);
+                        const uint32_t idesc = (i8 ? umma_idesc(kCFmtS32, kFmtS8, kTileM * CTAS, 0) : umma_idesc(kCFmtF32, kFmtBF16, kTileM * CTAS, 0)) |
+                                               ((uint32_t)(ph.n_mma >> 3) << 17) | (ph.a_mn ? (1u << 15) : 0u) | (ph.b_mn ? (1u << 16) : 0u);
                         uint32_t accumulate = ph.fresh ? 0u : 1u;
                         for (int b = 0; b < nblk; ++b) {
                             if (!mbar_wait(full0 + 8u * stage, phase, abort_flag)) { ok = false; break; }
                             tc_fence_after();
-                            const uint32_t a_lo = (((tiles_base + stage * kStageBytes) & 0x3FFFFu) >> 4) | lbo;
-                            const uint32_t b_lo = a_lo + (kOperandBytes >> 4);
+                            const uint32_t s_lo = ((tiles_base + stage * kStageBytes) & 0x3FFFFu) >> 4;
+                            const uint32_t a_lo = s_lo | a_lbo;
+                            const uint32_t b_lo = (s_lo + (kABytes >> 4)) | b_lbo;
                             const int nmma = (b == nblk - 1) ? nmma_last : 4;
                             if (i8) {
 #pragma unroll
                                 for (int k = 0; k < 4; ++k)
-                                    if (k < nmma) { umma_i8(acc, make_desc(a_lo + k * kadv, kDescHi), make_desc(b_lo + k * kadv, kDescHi), idesc, accumulate); accumulate = 1u; }
+                                    if (k < nmma) { umma_i8<CTAS>(acc, make_desc(a_lo + k * a_kadv, kDescHi), make_desc(b_lo + k * b_kadv, kDescHi), idesc, accumulate); accumulate = 1u; }
                             } else {
 #pragma unroll
                                 for (int k = 0; k < 4; ++k)
-                                    if (k < nmma) { umma_f16(acc, make_desc(a_lo + k * kadv, kDescHi), make_desc(b_lo + k * kadv, kDescHi), idesc, accumulate); accumulate = 1u; }
+                                    if (k < nmma) { umma_f16<CTAS>(acc, make_desc(a_lo + k * a_kadv, kDescHi), make_desc(b_lo + k * b_kadv, kDescHi), idesc, accumulate); accumulate = 1u; }
                             }
-                            umma_commit(empty0 + 8u * stage);
+                            umma_commit<CTAS>(empty0 + 8u * stage);
                             if (++stage == kStages) { stage = 0; phase ^= 1u; }
                         }
                     }
@@ -235,27 +277,31 @@ __global__ void __launch_bounds__(kGemmThreads, 1) umma_gemm_kernel(const __grid
                     if (ok && i == 0 && t > 0 && !mbar_wait(tmem_empty_bar, (uint32_t)((t - 1) & 1), abort_flag)) ok = false;
                 }
                 if (!ok) break;
-                umma_commit(tmem_full_bar);
+                umma_commit<CTAS>(tmem_full_bar);
             }
         }
     } else {
-        // ------------------------------------------------------------------ epilogue (128 threads)
+        // ------------------------------------------------------------------ epilogue (128 threads per CTA)
         const int q = warp & 3;                  // TMEM lane quarter this warp may read
         const int row = q * 32 + lane;
         const int et = threadIdx.x - 64;         // 0..127
         bool ok = true;
         int t = 0;
-        for (int tile = blockIdx.x; tile < ntiles && ok; tile += gridDim.x, ++t) {
+        for (int tile = unit; tile < ntiles && ok; tile += nunits, ++t) {
             const int tm = tile % p.tiles_m, tn = tile / p.tiles_m;
-            const int m0 = tm * kTileM, n0 = tn * kTileN;
+            const int m0 = tm * (kTileM * CTAS) + (int)rank * kTileM, n0 = tn * TN;
             const int buf = t & 1;
+            float* scale_w = scales + buf * 2 * TN;
+            float* scale_o = scale_w + TN;
             if (EPI == EPI_FWD) {
-                const int n = n0 + et;
-                sm->scale_w[buf][et] = n < p.N ? p.dW[n] : 0.0f;
-                sm->scale_o[buf][et] = (n < p.N && p.has_outlier) ? p.dw_O[n] : 0.0f;
+                for (int c = et; c < TN; c += 128) {
+                    const int n = n0 + c;
+                    scale_w[c] = n < p.N ? p.dW[n] : 0.0f;
+                    scale_o[c] = (n < p.N && p.has_outlier) ? p.dw_O[n] : 0.0f;
+                }
                 named_bar_sync(1, 128);
             }
-            if (!mbar_wait(smem_u32(&sm->tmem_full), (uint32_t)(t & 1), abort_flag)) { ok = false; break; }
+            if (!mbar_wait(tmem_full_bar, (uint32_t)(t & 1), abort_flag)) { ok = false; break; }
             tc_fence_after();
             const int m = m0 + row;
             const uint32_t lane_addr = tmem_base + ((uint32_t)(q * 32) << 16);
@@ -264,7 +310,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) umma_gemm_kernel(const __grid
 #pragma unroll 1
                 for (int c = 0; c * 32 < p.part_cols; ++c) {
                     uint32_t r0[32];
-                    tmem_ld_32x32(lane_addr + (uint32_t)(buf * kTileN + c * 32), r0);
+                    tmem_ld_32x32(lane_addr + (uint32_t)(buf * TN + c * 32), r0);
                     tmem_ld_wait();
                     if (m < p.M) {
                         float* out = p.part + ((int64_t)tn * p.M + m) * p.part_ld + c * 32;
@@ -277,23 +323,23 @@ __global__ void __launch_bounds__(kGemmThreads, 1) umma_gemm_kernel(const __grid
                 }
             } else {
 #pragma unroll 1
-                for (int c = 0; c < kTileN / 32; ++c) {
+                for (int c = 0; c < TN / 32; ++c) {
                     const int nc = n0 + c * 32;
                     if (nc >= p.N) break;            // uniform across the warp
                     uint32_t r0[32];
-                    tmem_ld_32x32(lane_addr + (uint32_t)(buf * kTileN + c * 32), r0);
+                    tmem_ld_32x32(lane_addr + (uint32_t)(buf * TN + c * 32), r0);
                     if (EPI == EPI_FWD) {
                         uint32_t r1[32], r2[32];
-                        if (p.has_outlier) tmem_ld_32x32(lane_addr + (uint32_t)(2 * kTileN + c * 32), r1);
-                        if (p.has_lora) tmem_ld_32x32(lane_addr + (uint32_t)(3 * kTileN + c * 32), r2);
+                        if (p.has_outlier) tmem_ld_32x32(lane_addr + (uint32_t)(2 * TN + c * 32), r1);
+                        if (p.has_lora) tmem_ld_32x32(lane_addr + (uint32_t)(3 * TN + c * 32), r2);
                         tmem_ld_wait();
                         if (m < p.M) {
                             const float dxm = p.dx[m];
                             float y[32];
 #pragma unroll
                             for (int j = 0; j < 32; ++j) {
-                                float w = (float)(int)r0[j] * sm->scale_w[buf][c * 32 + j];
-                                if (p.has_outlier) w += (float)(int)r1[j] * sm->scale_o[buf][c * 32 + j];
+                                float w = (float)(int)r0[j] * scale_w[c * 32 + j];
+                                if (p.has_outlier) w += (float)(int)r1[j] * scale_o[c * 32 + j];
                                 float v = dxm * w;
                                 if (p.has_lora) v += p.lora_scale * __uint_as_float(r2[j]);
                                 y[j] = v;
@@ -353,7 +399,10 @@ __global__ void __launch_bounds__(kGemmThreads, 1) umma_gemm_kernel(const __grid
             }
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(&sm->tmem_empty));
+            if (lane == 0) {
+                if (CTAS == 2 && rank != 0) mbar_arrive_cluster(lead_tmem_empty);
+                else mbar_arrive(tmem_empty_bar);
+            }
         }
     }
 
@@ -365,10 +414,13 @@ __global__ void __launch_bounds__(kGemmThreads, 1) umma_gemm_kernel(const __grid
         if (threadIdx.x == 0 && p.status) atomicExch(p.status, (int)QUAFF_ERR_TIMEOUT);
         __syncthreads();
     }
+    // neither CTA of a pair may retire (or free TMEM) while its partner can still read its shared
+    // memory, write its TMEM or signal its barriers
+    if (CTAS == 2) cluster_sync();
     if (warp == 1) {
         __syncwarp();
         tc_fence_after();
-        tmem_dealloc(tmem_base, 512);
+        tmem_dealloc<CTAS>(tmem_base, 512);
     }
 }
 
