@@ -385,7 +385,10 @@ extern "C" quaff_status_t quaff_qlinear_fwd(int M, int K, int N, const int8_t* X
     unsigned char* base = reinterpret_cast<unsigned char*>(ws);
     uint16_t* At = reinterpret_cast<uint16_t*>(base + w.off_at);
     float* part = reinterpret_cast<float*>(base + w.off_part);
-    constexpr int TN = 128, CTAS = 2;
+    constexpr int CTAS = 2;
+    // Three accumulators (main, outlier, LoRA) fit TMEM only with 128-column tiles; Eq. 2 alone (no outlier
+    // set, no LoRA) takes the 256-column tile.
+    const int TN = (nOp == 0 && r == 0) ? 256 : 128;
 
     GemmParams p;
     memset(&p, 0, sizeof(p));
@@ -425,7 +428,7 @@ extern "C" quaff_status_t quaff_qlinear_fwd(int M, int K, int N, const int8_t* X
     p.has_outlier = nOp > 0; p.has_lora = r > 0;
     p.Y = Y; p.ldy = ldy; p.y_f32 = (y_dtype == QUAFF_F32);
     p.dbg_main = dbg_acc_main; p.dbg_out = dbg_acc_out;
-    return launch_gemm<EPI_FWD, CTAS, TN>(p, st);
+    return TN == 256 ? launch_gemm<EPI_FWD, CTAS, 256>(p, st) : launch_gemm<EPI_FWD, CTAS, 128>(p, st);
 }
 
 extern "C" quaff_status_t quaff_qlinear_bwd(int M, int K, int N, const quaff_bf16* dY, int64_t lddy, const int8_t* Wq,

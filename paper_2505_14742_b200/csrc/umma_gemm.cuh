@@ -32,6 +32,9 @@
 // TMEM (512 columns): slot 0 is double-buffered at columns [0,TN) and [TN,2TN) so the main
 // contraction of tile t+1 overlaps the epilogue of tile t; with TN = 128, slots 1 and 2 live at
 // [256,384) and [384,512) and are written only after the epilogue of the previous tile has drained them.
+// A 256-wide tcgen05.mma runs at nearly twice the rate of a 128-wide one (a 128-wide one is bound by
+// fetching its A operand from shared memory), but two 256-column buffers fill TMEM: TN = 256 is for
+// contractions with a single accumulator (grad-input; forward without outliers and LoRA).
 //
 // The producer and the MMA issuer are single threads; their per-k-block instruction count bounds the
 // tensor-pipe utilisation, so everything that does not change inside a phase is hoisted out of the
@@ -137,7 +140,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) umma_gemm_kernel(const __grid
     constexpr int kStages = Cfg::kStages;
     constexpr int kStageBytes = Cfg::kStageBytes;
     static_assert(CTAS == 1 || CTAS == 2, "one CTA or a CTA pair");
-    static_assert(TN == 128 || (TN == 256 && EPI == EPI_BWD), "three accumulators fit TMEM only at TN = 128");
+    static_assert(TN == 128 || TN == 256, "output-column tile");   // TN = 256: slot 0 only (no room for auxiliary accumulators)
 
     extern __shared__ unsigned char smem_dyn[];
     const uint32_t raw = smem_u32(smem_dyn);
