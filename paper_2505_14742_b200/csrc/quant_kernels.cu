@@ -27,46 +27,95 @@ int sm_count() {
 // =====================================================================================
 // Activation scaling + per-token quantization (one pass over X)
 // =====================================================================================
-// One CTA owns one token row at a time and keeps it in registers as packed bf16 between the
-// absmax reduction and the quantization, so X is read from HBM exactly once.  A thread owns up to
-// J "units" of 16 consecutive channels (two 128-bit loads, one 128-bit store of codes).  Which of
-// a thread's units contain outlier channels is the same for every row, so it is found once per
-// CTA (binary search in the sorted O) and kept in registers; those units divide the outlier
-// elements by s before both the absmax and the rounding.
+// A small CTA (64..256 threads) owns one token row at a time and keeps it in registers as packed
+// bf16 between the absmax reduction and the quantization, so X is read from HBM exactly once; the
+// next row of the CTA is already being loaded while the current one is reduced and quantized, and
+// many such CTAs are resident per SM, which is what keeps enough bytes in flight for HBM.
+// A thread owns up to J "units" of 16 consecutive channels (two 128-bit loads, one 128-bit store of
+// codes).  Which elements of a thread's units are outlier channels is the same for every row: it is
+// found once per CTA (binary search in the sorted O) and kept as a 16-bit mask per unit.  The fast
+// path treats masked elements as zero; the few outlier elements are handled one by one
+// (x / s before both the absmax and the rounding, as Eq. 5 requires) and patched into the codes.
+//
+// Rounding: adding 1.5 * 2^23 to a float of magnitude < 2^22 rounds it to an integer, ties to even,
+// and leaves that integer in the low mantissa bits; the low byte of the bit pattern is the two's
+// complement INT8 code.  |x * (127 / amax)| <= 127 (1 + 2^-23) always rounds into [-127, 127].
 
-__device__ __forceinline__ void unit_decode(const uint4& a, const uint4& b, float (&v)[16]) {
-    const uint32_t w[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
+constexpr float kRoundMagic = 12582912.0f;   // 1.5 * 2^23
+#ifndef QUAFF_QA_MAX_THREADS
+#define QUAFF_QA_MAX_THREADS 128
+#endif
+constexpr int kQuantActMaxThreads = QUAFF_QA_MAX_THREADS;   // CTA size the dispatch aims for (tuning constant)
+
+__device__ __forceinline__ uint32_t code_bits(float x, float rinv) {   // low byte = Eq. 1 code of x
+    return __float_as_uint(__fadd_rn(__fmul_rn(x, rinv), kRoundMagic));
+}
+
+// Largest 15-bit magnitude among the 8 packed bf16 of a 128-bit word, as two packed 16-bit maxima.
+// `keep` has 0x7FFF on the halves that count and 0 on outlier elements (they enter scaled, separately).
+__device__ __forceinline__ uint32_t absmax8(const uint4& a, const uint4& keep, uint32_t acc) {
+    acc = __vmaxu2(acc, a.x & keep.x);
+    acc = __vmaxu2(acc, a.y & keep.y);
+    acc = __vmaxu2(acc, a.z & keep.z);
+    acc = __vmaxu2(acc, a.w & keep.w);
+    return acc;
+}
+
+// codes of the 8 packed bf16 of a 128-bit word -> two 32-bit words of 4 codes each
+__device__ __forceinline__ uint2 codes8(const uint4& a, float rinv) {
+    const uint32_t w[4] = {a.x, a.y, a.z, a.w};
+    uint32_t c[8];
 #pragma unroll
-    for (int i = 0; i < 8; ++i) {
-        v[2 * i] = bf16_lo(w[i]);
-        v[2 * i + 1] = bf16_hi(w[i]);
+    for (int i = 0; i < 4; ++i) {
+        c[2 * i] = code_bits(__uint_as_float(w[i] << 16), rinv);
+        c[2 * i + 1] = code_bits(__uint_as_float(w[i] & 0xFFFF0000u), rinv);
+    }
+    uint2 r;
+    r.x = __byte_perm(__byte_perm(c[0], c[1], 0x0040), __byte_perm(c[2], c[3], 0x0040), 0x5410);
+    r.y = __byte_perm(__byte_perm(c[4], c[5], 0x0040), __byte_perm(c[6], c[7], 0x0040), 0x5410);
+    return r;
+}
+
+// TAIL: K is not a multiple of 16 (the last unit of a row is loaded and stored element by element)
+template <int J, bool TAIL>
+__device__ __forceinline__ void load_row(uint4 (&raw)[J][2], const uint16_t* __restrict__ xrow, int tid, int T, int K) {
+#pragma unroll
+    for (int j = 0; j < J; ++j) {
+        const int k0 = (tid + j * T) << 4;
+        if (!TAIL && k0 >= K) {
+            raw[j][0] = raw[j][1] = make_uint4(0, 0, 0, 0);
+        } else if (!TAIL || k0 + 16 <= K) {
+            const uint4* p = reinterpret_cast<const uint4*>(xrow + k0);
+            raw[j][0] = __ldg(p);
+            raw[j][1] = __ldg(p + 1);
+        } else {
+            uint32_t w[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+            for (int e = 0; e < 16; ++e)
+                if (k0 + e < K) w[e >> 1] |= (uint32_t)xrow[k0 + e] << ((e & 1) * 16);
+            raw[j][0] = make_uint4(w[0], w[1], w[2], w[3]);
+            raw[j][1] = make_uint4(w[4], w[5], w[6], w[7]);
+        }
     }
 }
 
-__device__ __forceinline__ void unit_apply_scale(float (&v)[16], int ustart, int obeg, int ocnt,
-                                                 const int* O_s, const float* s_s) {
-    for (int t = 0; t < ocnt; ++t) {
-        const int e = O_s[obeg + t] - ustart;
-        const float sv = s_s[obeg + t];
-#pragma unroll
-        for (int i = 0; i < 16; ++i)
-            if (i == e) v[i] = __fdiv_rn(v[i], sv);
-    }
-}
-
-template <int J>
-__global__ void __launch_bounds__(256) quant_act_kernel(const uint16_t* __restrict__ X, int64_t ldx, int M, int K,
+#ifndef QUAFF_QA_MIN_BLOCKS
+#define QUAFF_QA_MIN_BLOCKS 2
+#endif
+template <int J, bool TAIL>
+__global__ void __launch_bounds__(256, QUAFF_QA_MIN_BLOCKS) quant_act_kernel(const uint16_t* __restrict__ X, int64_t ldx, int M, int K,
                                                         const int32_t* __restrict__ O_idx, int nO,
                                                         const float* __restrict__ s_O,
                                                         int8_t* __restrict__ Xq, int64_t ldxq,
                                                         int8_t* __restrict__ xq_O, int64_t ldxo, int nOp,
                                                         float* __restrict__ dx) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    float* red = reinterpret_cast<float*>(smem_raw);            // [2][8]
-    int* O_s = reinterpret_cast<int*>(smem_raw + 64);           // [nO]
-    float* s_s = reinterpret_cast<float*>(smem_raw + 64) + nO;  // [nO]
-
     const int tid = threadIdx.x, T = blockDim.x;
+    float* red = reinterpret_cast<float*>(smem_raw);            // [2][8]
+    uint4* keep_s = reinterpret_cast<uint4*>(smem_raw + 64);    // [J][2][T]: magnitude masks of this thread's units
+    int* O_s = reinterpret_cast<int*>(smem_raw + 64 + (size_t)J * 2 * T * 16);   // [nO]
+    float* s_s = reinterpret_cast<float*>(O_s) + nO;                               // [nO]
+    float* xo_s = s_s + nO;                                                        // [2][nO]: scaled outlier elements of the row
+
     const int lane = tid & 31, warp = tid >> 5, nwarps = T >> 5;
     const int nunits = (K + 15) >> 4;
 
@@ -76,58 +125,53 @@ __global__ void __launch_bounds__(256) quant_act_kernel(const uint16_t* __restri
     }
     __syncthreads();
 
-    int obeg[J], ocnt[J];
+    // outlier elements of this thread's units (mask bit e = channel 16 u + e is in O) -> magnitude masks in smem
 #pragma unroll
     for (int j = 0; j < J; ++j) {
         const int u = tid + j * T;
-        obeg[j] = 0;
-        ocnt[j] = 0;
+        uint32_t mask = 0;
         if (u < nunits && nO > 0) {
-            const int lo_key = u << 4, hi_key = lo_key + 16;
+            const int lo_key = u << 4;
             int lo = 0, hi = nO;
             while (lo < hi) {  // first index with O >= lo_key
                 const int mid = (lo + hi) >> 1;
                 if (O_s[mid] < lo_key) lo = mid + 1; else hi = mid;
             }
-            const int b = lo;
-            hi = nO;
-            while (lo < hi) {  // first index with O >= hi_key
-                const int mid = (lo + hi) >> 1;
-                if (O_s[mid] < hi_key) lo = mid + 1; else hi = mid;
-            }
-            obeg[j] = b;
-            ocnt[j] = lo - b;
+            for (int t = lo; t < nO && O_s[t] < lo_key + 16; ++t) mask |= 1u << (O_s[t] - lo_key);
         }
+        uint32_t kw[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i)
+            kw[i] = ((mask >> (2 * i)) & 1u ? 0u : 0x00007FFFu) | ((mask >> (2 * i + 1)) & 1u ? 0u : 0x7FFF0000u);
+        keep_s[(j * 2 + 0) * T + tid] = make_uint4(kw[0], kw[1], kw[2], kw[3]);
+        keep_s[(j * 2 + 1) * T + tid] = make_uint4(kw[4], kw[5], kw[6], kw[7]);
     }
 
+    uint4 raw[J][2];
+    int m = blockIdx.x;
+    if (m < M) load_row<J, TAIL>(raw, X + (int64_t)m * ldx, tid, T, K);
     int parity = 0;
-    for (int m = blockIdx.x; m < M; m += gridDim.x, parity ^= 1) {
+    for (; m < M; m += gridDim.x, parity ^= 1) {
         const uint16_t* xrow = X + (int64_t)m * ldx;
-        uint4 raw[J][2];
+        // the CTA's next row is on its way while this one is processed
+        uint4 nxt[J][2];
+        const int mn = m + gridDim.x;
+        if (mn < M) load_row<J, TAIL>(nxt, X + (int64_t)mn * ldx, tid, T, K);
+
+        uint32_t mag = 0;                               // two packed 15-bit magnitudes (bf16 bits order like the values)
 #pragma unroll
         for (int j = 0; j < J; ++j) {
-            const int u = tid + j * T;
-            const int k0 = u << 4;
-            if (k0 + 16 <= K) {
-                const uint4* p = reinterpret_cast<const uint4*>(xrow + k0);
-                raw[j][0] = __ldg(p);
-                raw[j][1] = __ldg(p + 1);
-            } else {
-                uint32_t w[8] = {0, 0, 0, 0, 0, 0, 0, 0};
-                for (int e = 0; e < 16; ++e)
-                    if (k0 + e < K) w[e >> 1] |= (uint32_t)xrow[k0 + e] << ((e & 1) * 16);
-                raw[j][0] = make_uint4(w[0], w[1], w[2], w[3]);
-                raw[j][1] = make_uint4(w[4], w[5], w[6], w[7]);
-            }
+            mag = absmax8(raw[j][0], keep_s[(j * 2 + 0) * T + tid], mag);
+            mag = absmax8(raw[j][1], keep_s[(j * 2 + 1) * T + tid], mag);
         }
-        float amax = 0.0f;
-#pragma unroll
-        for (int j = 0; j < J; ++j) {
-            float v[16];
-            unit_decode(raw[j][0], raw[j][1], v);
-            if (ocnt[j]) unit_apply_scale(v, (tid + j * T) << 4, obeg[j], ocnt[j], O_s, s_s);
-#pragma unroll
-            for (int i = 0; i < 16; ++i) amax = fmaxf(amax, fabsf(v[i]));
+        float amax = __uint_as_float(max(mag & 0xFFFFu, mag >> 16) << 16);
+        // Eq. 5: the outlier channels enter the absmax as x / s.  They are spread over the CTA's threads
+        // (thread i takes channels O[i], O[i + T], ...), whoever owns the unit they sit in.
+        float* xo = xo_s + parity * nO;
+        for (int i = tid; i < nO; i += T) {
+            const float xs = __fdiv_rn(bf16_bits_to_f32(__ldg(xrow + O_s[i])), s_s[i]);
+            xo[i] = xs;
+            amax = fmaxf(amax, fabsf(xs));
         }
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
@@ -143,39 +187,48 @@ __global__ void __launch_bounds__(256) quant_act_kernel(const uint16_t* __restri
         int8_t* qrow = Xq + (int64_t)m * ldxq;
 #pragma unroll
         for (int j = 0; j < J; ++j) {
-            const int u = tid + j * T;
-            const int k0 = u << 4;
+            const int k0 = (tid + j * T) << 4;
             if (k0 >= K) continue;
-            float v[16];
-            unit_decode(raw[j][0], raw[j][1], v);
-            if (ocnt[j]) unit_apply_scale(v, k0, obeg[j], ocnt[j], O_s, s_s);
-            uint32_t c[4] = {0, 0, 0, 0};
-#pragma unroll
-            for (int i = 0; i < 16; ++i) c[i >> 2] |= ((uint32_t)quant_code(v[i], rinv) & 0xFFu) << ((i & 3) * 8);
-            if (k0 + 16 <= K) {
-                *reinterpret_cast<uint4*>(qrow + k0) = make_uint4(c[0], c[1], c[2], c[3]);
+            const uint2 c0 = codes8(raw[j][0], rinv), c1 = codes8(raw[j][1], rinv);
+            if (!TAIL || k0 + 16 <= K) {
+                *reinterpret_cast<uint4*>(qrow + k0) = make_uint4(c0.x, c0.y, c1.x, c1.y);
             } else {
+                const uint32_t c[4] = {c0.x, c0.y, c1.x, c1.y};
                 for (int e = 0; e < 16 && k0 + e < K; ++e) qrow[k0 + e] = (int8_t)((c[e >> 2] >> ((e & 3) * 8)) & 0xFFu);
             }
-            for (int t = 0; t < ocnt[j]; ++t) {  // Eq. 9: the outlier operand is a column gather of the codes
-                const int e = O_s[obeg[j] + t] - k0;
-                xq_O[(int64_t)m * ldxo + obeg[j] + t] = (int8_t)((c[e >> 2] >> ((e & 3) * 8)) & 0xFFu);
+        }
+        if (nO > 0) {
+            // outlier channels: the code of x / s replaces the one just written by the unit's owner (the
+            // barrier orders the two stores); Eq. 9: the outlier operand is a column gather of the codes
+            __syncthreads();
+            for (int i = tid; i < nO; i += T) {
+                const int8_t q = (int8_t)(code_bits(xo[i], rinv) & 0xFFu);
+                qrow[O_s[i]] = q;
+                xq_O[(int64_t)m * ldxo + i] = q;
             }
         }
         for (int i = nO + tid; i < nOp; i += T) xq_O[(int64_t)m * ldxo + i] = 0;
+#pragma unroll
+        for (int j = 0; j < J; ++j) {
+            raw[j][0] = nxt[j][0];
+            raw[j][1] = nxt[j][1];
+        }
     }
 }
 
-template <int J>
+template <int J, bool TAIL>
 static quaff_status_t launch_quant_act(int T, const uint16_t* X, int64_t ldx, int M, int K, const int32_t* O_idx, int nO,
                                        const float* s_O, int8_t* Xq, int64_t ldxq, int8_t* xq_O, int64_t ldxo, int nOp,
                                        float* dx, cudaStream_t st) {
-    const size_t smem = 64 + (size_t)nO * 8;
+    const size_t smem = 64 + (size_t)J * 2 * T * 16 + (size_t)nO * 16;
+    if (smem > 48 * 1024 &&
+        cudaFuncSetAttribute(quant_act_kernel<J, TAIL>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+        return QUAFF_ERR_UNSUPPORTED_SHAPE;
     int per_sm = 0;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, quant_act_kernel<J>, T, smem) != cudaSuccess || per_sm < 1)
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, quant_act_kernel<J, TAIL>, T, smem) != cudaSuccess || per_sm < 1)
         per_sm = 1;
     const int grid = min(M, sm_count() * per_sm);
-    quant_act_kernel<J><<<grid, T, smem, st>>>(X, ldx, M, K, O_idx, nO, s_O, Xq, ldxq, xq_O, ldxo, nOp, dx);
+    quant_act_kernel<J, TAIL><<<grid, T, smem, st>>>(X, ldx, M, K, O_idx, nO, s_O, Xq, ldxq, xq_O, ldxo, nOp, dx);
     return launch_status();
 }
 
@@ -183,16 +236,21 @@ static quaff_status_t quant_act_dispatch(const uint16_t* X, int64_t ldx, int M, 
                                          const float* s_O, int8_t* Xq, int64_t ldxq, int8_t* xq_O, int64_t ldxo,
                                          int nOp, float* dx, cudaStream_t st) {
     const int nunits = (K + 15) / 16;
-    int J = ceil_div(nunits, 256);
-    if (J > 8) return QUAFF_ERR_UNSUPPORTED_SHAPE;  // K > 32768
+    if (nunits > 8 * 256) return QUAFF_ERR_UNSUPPORTED_SHAPE;  // K > 32768
+    // units per thread: as many as keep the CTA at 128 threads or fewer (more, smaller CTAs per SM), at most 8
+    int J = 1;
+    while (J < 8 && ceil_div(nunits, J) > kQuantActMaxThreads) ++J;
+    if (J == 5) J = 6;
+    if (J == 7) J = 8;
     const int T = min(256, ceil_div(ceil_div(nunits, J), 32) * 32);
-#define QA(JJ) return launch_quant_act<JJ>(T, X, ldx, M, K, O_idx, nO, s_O, Xq, ldxq, xq_O, ldxo, nOp, dx, st)
+#define QA(JJ)                                                                                                    \
+    return (K % 16) ? launch_quant_act<JJ, true>(T, X, ldx, M, K, O_idx, nO, s_O, Xq, ldxq, xq_O, ldxo, nOp, dx, st) \
+                    : launch_quant_act<JJ, false>(T, X, ldx, M, K, O_idx, nO, s_O, Xq, ldxq, xq_O, ldxo, nOp, dx, st)
     switch (J) {
         case 1: QA(1);
         case 2: QA(2);
         case 3: QA(3);
         case 4: QA(4);
-        case 5:
         case 6: QA(6);
         default: QA(8);
     }
