@@ -280,11 +280,15 @@ __global__ void __launch_bounds__(256) momentum_kernel(const uint16_t* __restric
         const int i = c0 + lane;
         unsigned int best = 0;
         if (i < nO) {
-            const int col = O_idx[i];
-            for (int m = r0 + warp; m < r1; m += 8) {
-                const unsigned int mag = ((unsigned int)X[(int64_t)m * ldx + col] & 0x7FFFu) << 16;  // |x| as fp32 bits
-                best = max(best, mag);
+            const uint16_t* xc = X + O_idx[i];
+            int m = r0 + warp;
+            for (; m + 24 < r1; m += 32) {     // four independent gathers in flight per thread
+                const unsigned int a = __ldg(xc + (int64_t)m * ldx), b = __ldg(xc + (int64_t)(m + 8) * ldx);
+                const unsigned int c = __ldg(xc + (int64_t)(m + 16) * ldx), d = __ldg(xc + (int64_t)(m + 24) * ldx);
+                best = max(best, max(max(a & 0x7FFFu, b & 0x7FFFu), max(c & 0x7FFFu, d & 0x7FFFu)));
             }
+            for (; m < r1; m += 8) best = max(best, (unsigned int)__ldg(xc + (int64_t)m * ldx) & 0x7FFFu);
+            best <<= 16;                       // |x| as fp32 bits
         }
         red[warp][lane] = best;
         __syncthreads();
@@ -315,34 +319,55 @@ __global__ void __launch_bounds__(256) momentum_kernel(const uint16_t* __restric
 // =====================================================================================
 // Outlier weight rows: what = (s_O - 1) W_O, per-output-channel quantization
 // =====================================================================================
-// One thread per output channel n: reads down column n of W_O (coalesced across n), twice (the
-// second pass comes from L2), and writes its own row of codes wq_O[n][0..nOp).
-__global__ void __launch_bounds__(64) requant_rows_kernel(const uint16_t* __restrict__ W_O, int64_t ldwo, int nO, int N,
-                                                          const float* __restrict__ s_O, int8_t* __restrict__ wq_O,
-                                                          int64_t ldwq, int nOp, float* __restrict__ dw_O) {
-    const int n = blockIdx.x * blockDim.x + threadIdx.x;
-    if (n >= N) return;
+// A CTA of 8 warps owns 32 output channels: warp w takes the outlier rows w, w + 8, ... (a warp reads 32
+// consecutive channels of one row of W_O: coalesced), the per-channel maxima meet in shared memory, and
+// the codes go through a shared tile so that each row of wq_O leaves in 128-bit pieces.  The second
+// read of W_O comes from L1/L2.
+constexpr int kRqCols = 32, kRqRows = 128, kRqPitch = kRqRows + 16;
+__global__ void __launch_bounds__(256) requant_rows_kernel(const uint16_t* __restrict__ W_O, int64_t ldwo, int nO, int N,
+                                                           const float* __restrict__ s_O, int8_t* __restrict__ wq_O,
+                                                           int64_t ldwq, int nOp, float* __restrict__ dw_O) {
+    extern __shared__ __align__(16) unsigned char rq_smem[];
+    float* sm1_s = reinterpret_cast<float*>(rq_smem);                 // [nO]: s - 1
+    float* red = sm1_s + ((nO + 3) & ~3);                             // [8][32]
+    unsigned char* tile = reinterpret_cast<unsigned char*>(red + 8 * kRqCols);   // [32][kRqPitch] codes
+    const int tid = threadIdx.x, cx = tid & 31, ry = tid >> 5;
+    const int n = blockIdx.x * kRqCols + cx;
+    const bool live = n < N;
+    for (int i = tid; i < nO; i += 256) sm1_s[i] = __fsub_rn(__ldg(s_O + i), 1.0f);
+    __syncthreads();
     float amax = 0.0f;
-    for (int i = 0; i < nO; ++i) {
-        const float sm1 = __fsub_rn(__ldg(s_O + i), 1.0f);
-        const float w = __fmul_rn(sm1, bf16_bits_to_f32(__ldg(W_O + (int64_t)i * ldwo + n)));
-        amax = fmaxf(amax, fabsf(w));
+    if (live) {
+#pragma unroll 4
+        for (int i = ry; i < nO; i += 8)
+            amax = fmaxf(amax, fabsf(__fmul_rn(sm1_s[i], bf16_bits_to_f32(__ldg(W_O + (int64_t)i * ldwo + n)))));
     }
-    dw_O[n] = __fdiv_rn(amax, 127.0f);
-    const float rinv = amax > 0.0f ? __fdiv_rn(127.0f, amax) : 0.0f;
-    int8_t* out = wq_O + (int64_t)n * ldwq;
-    for (int i0 = 0; i0 < nOp; i0 += 16) {
-        uint32_t c[4] = {0, 0, 0, 0};
+    red[ry * kRqCols + cx] = amax;
+    __syncthreads();
 #pragma unroll
-        for (int e = 0; e < 16; ++e) {
-            const int i = i0 + e;
-            if (i < nO) {
-                const float sm1 = __fsub_rn(__ldg(s_O + i), 1.0f);
-                const float w = __fmul_rn(sm1, bf16_bits_to_f32(__ldg(W_O + (int64_t)i * ldwo + n)));
-                c[e >> 2] |= ((uint32_t)quant_code(w, rinv) & 0xFFu) << ((e & 3) * 8);
+    for (int w = 0; w < 8; ++w) amax = fmaxf(amax, red[w * kRqCols + cx]);
+    if (live && ry == 0) dw_O[n] = __fdiv_rn(amax, 127.0f);
+    const float rinv = amax > 0.0f ? __fdiv_rn(127.0f, amax) : 0.0f;
+    for (int c0 = 0; c0 < nOp; c0 += kRqRows) {
+        const int cl = min(kRqRows, nOp - c0);                        // a multiple of 16
+        if (live) {
+#pragma unroll 4
+            for (int i = c0 + ry; i < c0 + cl; i += 8) {
+                int q = 0;
+                if (i < nO) q = quant_code(__fmul_rn(sm1_s[i], bf16_bits_to_f32(__ldg(W_O + (int64_t)i * ldwo + n))), rinv);
+                tile[cx * kRqPitch + (i - c0)] = (unsigned char)(q & 0xFF);
             }
         }
-        *reinterpret_cast<uint4*>(out + i0) = make_uint4(c[0], c[1], c[2], c[3]);
+        __syncthreads();
+        const int cpr = cl >> 4;                                      // 128-bit pieces per channel row
+        for (int idx = tid; idx < kRqCols * cpr; idx += 256) {
+            const int col = idx / cpr, ch = idx - col * cpr;
+            const int nn = blockIdx.x * kRqCols + col;
+            if (nn < N)
+                *reinterpret_cast<uint4*>(wq_O + (int64_t)nn * ldwq + c0 + 16 * ch) =
+                    *reinterpret_cast<const uint4*>(tile + col * kRqPitch + 16 * ch);
+        }
+        __syncthreads();
     }
 }
 
@@ -422,7 +447,8 @@ extern "C" quaff_status_t quaff_requant_weight_rows(const quaff_bf16* W_O, int64
     QUAFF_RETURN_IF(nOp > 0 && (!wq_O || ldwq < nOp), QUAFF_ERR_INVALID_ARG);
     QUAFF_RETURN_IF(nOp % 16, QUAFF_ERR_UNSUPPORTED_SHAPE);
     QUAFF_RETURN_IF(nOp > 0 && (!aligned16(wq_O) || (ldwq % 16)), QUAFF_ERR_ALIGNMENT);
-    requant_rows_kernel<<<ceil_div(N, 64), 64, 0, (cudaStream_t)stream>>>(W_O, ldwo, nO, N, s_O, wq_O, ldwq, nOp, dw_O);
+    const size_t smem = (size_t)((nO + 3) & ~3) * 4 + 8 * kRqCols * 4 + (size_t)kRqCols * kRqPitch;
+    requant_rows_kernel<<<ceil_div(N, kRqCols), 256, smem, (cudaStream_t)stream>>>(W_O, ldwo, nO, N, s_O, wq_O, ldwq, nOp, dw_O);
     return launch_status();
 }
 
