@@ -16,7 +16,6 @@ import json
 import os
 import subprocess
 import sys
-import threading
 import time
 
 import numpy as np
@@ -41,47 +40,53 @@ def load_peaks():
 
 
 class ClockSampler:
-    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    """Samples SM clocks and throttle reasons with one `nvidia-smi -lms` process while the timed region runs."""
     Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
          "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
 
-    def __init__(self, index):
+    def __init__(self, index, period_ms=20):
         self.index = index
+        self.period_ms = period_ms
         self.rows = []
-        self._stop = threading.Event()
-        self._t = threading.Thread(target=self._run, daemon=True)
-
-    def _run(self):
-        while not self._stop.is_set():
-            try:
-                out = subprocess.run(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-i", str(self.index)],
-                                     capture_output=True, text=True, timeout=5).stdout.strip()
-                if out:
-                    self.rows.append([c.strip() for c in out.split(",")])
-            except Exception:
-                pass
-            self._stop.wait(0.1)
+        self.proc = None
 
     def __enter__(self):
-        self._t.start()
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                          "-i", str(self.index), "-lms", str(self.period_ms)],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            time.sleep(0.25)          # let the sampler start before the timed region
+        except Exception:
+            self.proc = None
         return self
 
     def __exit__(self, *a):
-        self._stop.set()
-        self._t.join(timeout=6)
+        if self.proc is None:
+            return
+        time.sleep(0.05)
+        self.proc.terminate()          # the exact process started above
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except Exception:
+            self.proc.kill()
+            out = ""
+        for line in out.strip().splitlines():
+            self.rows.append([c.strip() for c in line.split(",")])
 
     def summary(self):
-        sm, mx, reasons = [], [], set()
+        sm, mx, power, reasons = [], [], [], set()
         for r in self.rows:
             try:
-                sm.append(float(r[0])); mx.append(float(r[1]))
+                sm.append(float(r[0])); mx.append(float(r[1])); power.append(float(r[2]))
             except Exception:
                 continue
             for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), r[3:7]):
                 if v.lower().startswith("active"):
                     reasons.add(name)
-        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "reasons": sorted(reasons), "samples": len(sm)}
+        # samples taken while the GPU was working: the upper half by power draw
+        busy = [c for c, p in zip(sm, power) if power and p >= 0.5 * (min(power) + max(power))] or sm
+        return {"sm_mhz": float(np.median(busy)) if busy else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm), "power_w_max": max(power) if power else None}
 
 
 def layer_ops(M, sp, nOp):
@@ -198,11 +203,13 @@ def run_gpu(args, wl):
         host_in.append((hx, hdy))
     torch.cuda.synchronize()
 
+    from paper_2505_14742_b200.layer import StepGraph
+
     def step(i, timing=None):
         layers, xs, dys = sets[i % REPLICAS]
         for li in range(nl):
             if timing is not None:
-                ev = timing[li][i]
+                ev = timing[i % REPLICAS][li]
                 Q.quaff_debug_time_gemm(0, ev[0], ev[1])
                 Q.quaff_debug_time_gemm(1, ev[2], ev[3])
             layers[li].forward(xs[li])
@@ -217,32 +224,49 @@ def run_gpu(args, wl):
     for i in range(args.warmup):
         step(i)
     sync_all()
+
+    # One pair of CUDA events around each tensor-core GEMM of each buffer set (torch creates the event lazily
+    # at its first record(): materialise every handle now).  In graph mode they are recorded by the graph.
+    timing = [[[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(nl)] for _ in range(REPLICAS)]
+    for per_set in timing:
+        for evs in per_set:
+            for e in evs:
+                e.record()
+    # ---- the step as a CUDA graph per buffer set (default), or enqueued launch by launch (--eager)
+    launches0 = Q.quaff_debug_launch_count()
+    if args.eager:
+        step(0, timing)
+        run_step = lambda i: step(i, timing)
+    else:
+        graphs = [StepGraph(lambda rep=rep: step(rep, timing)) for rep in range(REPLICAS)]
+        run_step = lambda i: graphs[i % REPLICAS].replay()
+    launches_per_step = (Q.quaff_debug_launch_count() - launches0) // (1 if args.eager else REPLICAS)
+    for i in range(REPLICAS):
+        run_step(i)
+    sync_all()
     for layers, _, _ in sets:
         for l in layers:
             assert int(l.status[0].item()) == 0, "device-side wait timed out"
 
     # ---- device-resident timed region
-    # torch creates the CUDA event lazily at its first record(): materialise every handle before the timed region
-    timing = [[[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(args.steps)] for _ in range(nl)]
-    for per_layer_events in timing:
-        for evs in per_layer_events:
-            for e in evs:
-                e.record()
-    launches0 = Q.quaff_debug_launch_count()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     with ClockSampler(local) as clocks:
         sync_all()
         e0.record()
         for i in range(args.steps):
-            step(i, timing)
+            run_step(i)
         e1.record()
         sync_all()
-    launches = Q.quaff_debug_launch_count() - launches0
+    launches = launches_per_step * args.steps
     ms_total = e0.elapsed_time(e1)
     t = torch.tensor([ms_total], dtype=torch.float64, device="cuda")
     if world > 1:
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
     ms_per_step = float(t.item()) / args.steps
+    # GEMM durations of the latest step on each buffer set that the timed region used
+    used_sets = min(REPLICAS, args.steps)
+    gemm_ms = [[float(np.mean([timing[rep][li][a].elapsed_time(timing[rep][li][a + 1]) for rep in range(used_sets)]))
+                for a in (0, 2)] for li in range(nl)]
 
     # ---- end to end: host buffers in, host buffers out, copies inside the timed region
     h_out = []
@@ -267,9 +291,17 @@ def run_gpu(args, wl):
     for i in range(2):
         step_e2e(i)
     sync_all()
+    if args.eager:
+        run_e2e = step_e2e
+    else:
+        e2e_graphs = [StepGraph(lambda rep=rep: step_e2e(rep)) for rep in range(REPLICAS)]
+        run_e2e = lambda i: e2e_graphs[i % REPLICAS].replay()
+        for i in range(REPLICAS):
+            run_e2e(i)
+    sync_all()
     e0.record()
     for i in range(e2e_steps):
-        step_e2e(i)
+        run_e2e(i)
     e1.record()
     sync_all()
     t2 = torch.tensor([e0.elapsed_time(e1)], dtype=torch.float64, device="cuda")
@@ -288,8 +320,7 @@ def run_gpu(args, wl):
     dominant = None
     for li, sp in enumerate(wl.layers):
         nOp = synth.pad_to(sp.nO, 32)
-        f_ms = float(np.mean([ev[0].elapsed_time(ev[1]) for ev in timing[li]]))
-        b_ms = float(np.mean([ev[2].elapsed_time(ev[3]) for ev in timing[li]]))
+        f_ms, b_ms = gemm_ms[li]
         fwd_int8, fwd_lora, bwd_bf16 = layer_ops(M, sp, nOp)
         entry = {"layer": sp.name, "K": sp.K, "N": sp.N, "nO": sp.nO, "r": sp.r,
                  "fwd_gemm_ms": f_ms, "fwd_int8_tops": fwd_int8 / (f_ms * 1e-3) / 1e12,
@@ -319,7 +350,8 @@ def run_gpu(args, wl):
             "data": "synthetic",
             "config": {"workload": wl.name, "tokens_per_gpu": M,
                        "layers": [f"{l.name} {l.K}->{l.N} nO={l.nO} r={l.r}" for l in wl.layers], "gamma": wl.gamma,
-                       "l2": f"rotating {REPLICAS} full buffer sets (weights, activations, outputs); one set alone exceeds the 126 MB L2"},
+                       "l2": f"rotating {REPLICAS} full buffer sets (weights, activations, outputs); one set alone exceeds the 126 MB L2",
+                       "launch": "eager" if args.eager else "one CUDA graph replay per step"},
             "clocks": clocks.summary(),
             "e2e": {"value": world * M / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                     "ms_per_step": e2e_ms, "steps": e2e_steps},
@@ -333,12 +365,13 @@ def run_gpu(args, wl):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--steps", type=int, default=1000)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--workload", default="phi3_attn", choices=sorted(synth.WORKLOADS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--sample-tokens", type=int, default=128, help="tokens per step of the CPU oracle (reference arm); the cpu_baseline leg uses 8x this")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--eager", action="store_true", help="enqueue every launch from Python instead of replaying a CUDA graph of the step")
     args = ap.parse_args()
     wl = synth.WORKLOADS[args.workload]
     if args.impl == "reference":

@@ -204,7 +204,9 @@ quaff_status_t quaff_momentum_update_static(const quaff_bf16* X, int64_t ldx, in
  * quaff_debug_time_gemm: arm a one-shot pair of CUDA events (cudaEvent_t, created by the caller
  * with timing enabled) around the next launch of the forward (which = 0) or grad-input
  * (which = 1) tensor-core GEMM kernel: `start` is recorded on the launch stream right before the
- * kernel, `stop` right after, then the pair is disarmed.  Null events disarm.
+ * kernel, `stop` right after, then the pair is disarmed.  Null events disarm.  If the stream is being
+ * captured into a CUDA graph, the pair becomes two event-record nodes of that graph: every replay records
+ * them again, and the elapsed time between them is that of the latest replay.
  */
 uint64_t quaff_debug_launch_count(void);
 void quaff_debug_time_gemm(int which, void* start_event, void* stop_event);

@@ -86,7 +86,14 @@ static quaff_status_t launch_gemm(const GemmParams& p, cudaStream_t st) {
     if (ntiles == 0) return QUAFF_OK;
     const int units = min(ntiles, gemm_units<EPI, CTAS, TN>(dev));
     const bool timed = EPI < 2 && g_time_start[EPI % 2] && g_time_stop[EPI % 2];
-    if (timed) cudaEventRecord(g_time_start[EPI % 2], st);
+    // while the stream is being captured into a CUDA graph, the events become event-record nodes of the
+    // graph (every replay records them again); otherwise they are recorded once, now
+    unsigned int ev_flags = cudaEventRecordDefault;
+    if (timed) {
+        cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+        if (cudaStreamIsCapturing(st, &cap) == cudaSuccess && cap == cudaStreamCaptureStatusActive) ev_flags = cudaEventRecordExternal;
+        cudaEventRecordWithFlags(g_time_start[EPI % 2], st, ev_flags);
+    }
     if (CTAS == 1) {
         umma_gemm_kernel<EPI, CTAS, TN><<<units, kGemmThreads, Cfg::kSmemBytes, st>>>(p);
     } else {
@@ -104,7 +111,7 @@ static quaff_status_t launch_gemm(const GemmParams& p, cudaStream_t st) {
     }
     const quaff_status_t rc = launch_status();
     if (timed) {
-        cudaEventRecord(g_time_stop[EPI % 2], st);
+        cudaEventRecordWithFlags(g_time_stop[EPI % 2], st, ev_flags);
         g_time_start[EPI % 2] = g_time_stop[EPI % 2] = nullptr;
     }
     return rc;
@@ -190,7 +197,8 @@ __global__ void __launch_bounds__(256) dequant_weight_kernel(const int8_t* __res
     out[1] = make_uint4(pack_bf16x2(v[8], v[9]), pack_bf16x2(v[10], v[11]), pack_bf16x2(v[12], v[13]), pack_bf16x2(v[14], v[15]));
 }
 
-// dX[m][O_i] = bf16((P[m][i] + P[m][nOp+i]) / s_i + sum_j G[m][j] A[O_i][j])
+// dX[m][O_i] = bf16((P[m][i] + P[m][nOp+i]) / s_i + sum_j G[m][j] A[O_i][j]);  r is a multiple of 8:
+// the rows of G and A are read as 128-bit words of 8 bf16
 __global__ void bwd_fixup_kernel(const float* __restrict__ P, int64_t ldp, int M, int nO, int nOp,
                                  const int32_t* __restrict__ O_idx, const float* __restrict__ s_O,
                                  const uint16_t* __restrict__ G, const uint16_t* __restrict__ A, int r,
@@ -199,9 +207,19 @@ __global__ void bwd_fixup_kernel(const float* __restrict__ P, int64_t ldp, int M
     if (idx >= M * nO) return;
     const int m = idx / nO, i = idx % nO;
     const int k = O_idx[i];
-    float v = (P[(int64_t)m * ldp + i] + P[(int64_t)m * ldp + nOp + i]) / s_O[i];
+    const float v = (P[(int64_t)m * ldp + i] + P[(int64_t)m * ldp + nOp + i]) / s_O[i];
     float l = 0.0f;
-    for (int j = 0; j < r; ++j) l = fmaf(bf16_bits_to_f32(G[(int64_t)m * r + j]), bf16_bits_to_f32(A[(int64_t)k * r + j]), l);
+    const uint4* g = reinterpret_cast<const uint4*>(G + (int64_t)m * r);
+    const uint4* a = reinterpret_cast<const uint4*>(A + (int64_t)k * r);
+    for (int j = 0; j < (r >> 3); ++j) {
+        const uint4 gv = __ldg(g + j), av = __ldg(a + j);
+        const uint32_t gw[4] = {gv.x, gv.y, gv.z, gv.w}, aw[4] = {av.x, av.y, av.z, av.w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            l = fmaf(bf16_lo(gw[e]), bf16_lo(aw[e]), l);
+            l = fmaf(bf16_hi(gw[e]), bf16_hi(aw[e]), l);
+        }
+    }
     dX[(int64_t)m * lddx + k] = (uint16_t)f32_to_bf16_bits(v + l);
 }
 
