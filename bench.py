@@ -165,12 +165,10 @@ def run_reference(args, wl):
 def run_gpu(args, wl):
     import torch
     import torch.distributed as dist
-    from paper_2505_14742_b200 import binding as Q, build
+    from paper_2505_14742_b200 import binding as Q, build, dist as qdist
     from paper_2505_14742_b200.layer import QuaffLinear
 
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
+    rank, world, local = qdist.rank_world()
     torch.cuda.set_device(local)
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
@@ -195,7 +193,7 @@ def run_gpu(args, wl):
             sp = lin.spec
             layer = QuaffLinear(to_bf16(lin.W), torch.from_numpy(lin.O_idx).cuda(), to_bf16(lin.A), to_bf16(lin.B),
                                 wl.lora_alpha / sp.r, wl.gamma, M)
-            X, dY = synth.step_inputs(wl, li, rep + 1000 * rank, lin)
+            X, dY = synth.step_inputs(wl, li, qdist.batch_index(rep, rank), lin)
             layers.append(layer)
             xs.append(to_bf16(X)); dys.append(to_bf16(dY))
             hx.append(torch.from_numpy(X.view(np.int16)).pin_memory()); hdy.append(torch.from_numpy(dY.view(np.int16)).pin_memory())
@@ -258,11 +256,7 @@ def run_gpu(args, wl):
         e1.record()
         sync_all()
     launches = launches_per_step * args.steps
-    ms_total = e0.elapsed_time(e1)
-    t = torch.tensor([ms_total], dtype=torch.float64, device="cuda")
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms_per_step = float(t.item()) / args.steps
+    ms_per_step = qdist.max_over_ranks(e0.elapsed_time(e1), "cuda") / args.steps
     # GEMM durations of the latest step on each buffer set that the timed region used
     used_sets = min(REPLICAS, args.steps)
     gemm_ms = [[float(np.mean([timing[rep][li][a].elapsed_time(timing[rep][li][a + 1]) for rep in range(used_sets)]))
@@ -304,10 +298,7 @@ def run_gpu(args, wl):
         run_e2e(i)
     e1.record()
     sync_all()
-    t2 = torch.tensor([e0.elapsed_time(e1)], dtype=torch.float64, device="cuda")
-    if world > 1:
-        dist.all_reduce(t2, op=dist.ReduceOp.MAX)
-    e2e_ms = float(t2.item()) / e2e_steps
+    e2e_ms = qdist.max_over_ranks(e0.elapsed_time(e1), "cuda") / e2e_steps
 
     if rank != 0:
         if world > 1:
@@ -344,7 +335,7 @@ def run_gpu(args, wl):
                 "avg_launch_ms": ms}
 
     cpu = cpu_baseline(wl, min(wl.M, 8 * args.sample_tokens)) if not args.no_cpu_baseline else None
-    line = {"metric": METRIC, "value": world * M / (ms_per_step * 1e-3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+    line = {"metric": METRIC, "value": qdist.whole_job_rate(M, world, ms_per_step), "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "int8 forward (int32 accumulate), bf16 backward (f32 accumulate)",
             "data": "synthetic",
@@ -353,7 +344,7 @@ def run_gpu(args, wl):
                        "l2": f"rotating {REPLICAS} full buffer sets (weights, activations, outputs); one set alone exceeds the 126 MB L2",
                        "launch": "eager" if args.eager else "one CUDA graph replay per step"},
             "clocks": clocks.summary(),
-            "e2e": {"value": world * M / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+            "e2e": {"value": qdist.whole_job_rate(M, world, e2e_ms), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                     "ms_per_step": e2e_ms, "steps": e2e_steps},
             "gpu_launches": int(launches),
             "roofline": roofline, "layers": per_layer, "cpu_baseline": cpu}

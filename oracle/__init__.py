@@ -162,6 +162,22 @@ def qlinear_fwd(Xq, xq_O, dx, Wq, dW, wq_O, dw_O, X, A, B, lora_scale: float):
     return Y, T[:, :r], a1, a2
 
 
+def lora_down(X, A):
+    """T[M,r] = bf16(X A) (bf16 bits) of the whole batch: the forward routine run with no output
+    channels, so that only its LoRA down-projection step executes."""
+    X = _c(X, np.uint16)
+    M, K = X.shape
+    r = A.shape[1]
+    z8 = np.zeros((1, 1), np.int8)
+    zf = np.zeros(1, np.float32)
+    T = np.zeros((M, r), np.uint16)
+    _load().qo_qlinear_fwd(I32(M), I32(K), I32(0), _p(_c(np.zeros((M, 1), np.int8), np.int8)), I64(1), _p(z8), I64(1), I32(0),
+                           _p(_c(np.zeros(M, np.float32), np.float32)), _p(z8), I64(1), _p(zf), _p(z8), I64(1), _p(zf),
+                           _p(X), I64(K), _p(_c(A, np.uint16)), _p(np.zeros((r, 1), np.uint16)), I32(r), F32(1.0),
+                           _p(T), _p(np.zeros(1, np.float64)), _p(None), _p(None))
+    return T
+
+
 def qlinear_bwd(dY, Wq, dW, wq_O, dw_O, O_idx, s_O, X, T, A, B, lora_scale: float,
                 want_dX: bool = True, want_dAB: bool = True):
     """Returns (dX[M,K] f64 | None, dA[K,r] f64 | None, dB[r,N] f64 | None, G[M,r] bf16 bits)."""

@@ -3,6 +3,7 @@
 ``synth``    seeded synthetic workloads (numpy only)
 ``build``    builds libquaff.so in-tree with nvcc
 ``binding``  ctypes binding with the C ABI's names (needs torch + a CUDA device to run)
-``layer``    per-layer buffer owner that chains the entry points into one training step
+``layer``    per-layer buffer owner that chains the entry points into one training step (+ CUDA graph of a step)
+``dist``     multi-GPU plumbing of the benchmark (token-sharded replicas, no data-path collective)
 """
-__all__ = ["synth", "build", "binding", "layer"]
+__all__ = ["synth", "build", "binding", "layer", "dist"]

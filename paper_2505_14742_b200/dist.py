@@ -1,0 +1,35 @@
+"""Multi-GPU plumbing of the benchmark: one process per GPU, token-sharded replicas.
+
+Per-token quantization makes the rows of a batch independent and the weight is frozen and replicated,
+so the path shards over tokens with no collective on the data path: every rank runs the same layers on
+its own batch.  What the ranks share is only the clock: a step takes as long as its slowest rank.
+"""
+from __future__ import annotations
+
+import os
+
+
+def rank_world():
+    """(rank, world size, local rank) from the launcher's environment (torchrun), or a single process."""
+    return int(os.environ.get("RANK", "0")), int(os.environ.get("WORLD_SIZE", "1")), int(os.environ.get("LOCAL_RANK", "0"))
+
+
+def batch_index(step: int, rank: int) -> int:
+    """Index of the synthetic batch that `rank` processes at `step`: ranks never share a batch."""
+    return step + 1000 * rank
+
+
+def max_over_ranks(value: float, device=None) -> float:
+    """The largest `value` over all ranks (the job's time for a step); the value itself in a single process."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return float(value)
+    t = torch.tensor([value], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_rate(units_per_rank: int, world: int, ms_per_step: float) -> float:
+    """Units per second of the whole job: all ranks' units over the slowest rank's time."""
+    return world * units_per_rank / (ms_per_step * 1e-3)
