@@ -6,6 +6,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <utility>
+
 #include "../../include/quaff.h"
 
 namespace quaff {
@@ -29,6 +31,34 @@ inline quaff_status_t launch_status() {
 }
 
 int sm_count();  // SMs of the current device (cached)
+
+// Every kernel of this library is launched with programmatic stream serialization: it may be scheduled
+// while its predecessor in the stream is still running, and it orders itself behind that predecessor with
+// griddepcontrol.wait (pdl_wait) before its first access to global memory.  The launch latency, the CTA
+// start-up and the prologue (barrier set-up, TMEM allocation) of a kernel then overlap the tail of the
+// one before; the data dependencies are exactly those of a plain in-order stream.
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, int cluster_x,
+                              Args&&... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[2];
+    int n = 0;
+    attr[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[n].val.programmaticStreamSerializationAllowed = 1;
+    ++n;
+    if (cluster_x > 1) {
+        attr[n].id = cudaLaunchAttributeClusterDimension;
+        attr[n].val.clusterDim.x = cluster_x; attr[n].val.clusterDim.y = 1; attr[n].val.clusterDim.z = 1;
+        ++n;
+    }
+    cfg.attrs = attr;
+    cfg.numAttrs = n;
+    return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
+}
 
 // cuTensorMapEncodeTiled through the runtime's driver entry point (no link against libcuda).
 // 2-D row-major tensor [rows][cols] with a row pitch of ld elements; box = box_rows x box_cols.
@@ -56,6 +86,12 @@ __device__ __forceinline__ int quant_code(float x, float rinv) {
     int q = __float2int_rn(__fmul_rn(x, rinv));
     return max(-127, min(127, q));
 }
+
+// ------------------------------------------------------------------ PTX: programmatic dependent launch
+// First statements of every kernel: let the next kernel in the stream be scheduled early, then wait until
+// everything before this kernel in the stream has completed and its memory is visible.
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
 // ------------------------------------------------------------------ PTX: mbarrier
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }

@@ -94,21 +94,7 @@ static quaff_status_t launch_gemm(const GemmParams& p, cudaStream_t st) {
         if (cudaStreamIsCapturing(st, &cap) == cudaSuccess && cap == cudaStreamCaptureStatusActive) ev_flags = cudaEventRecordExternal;
         cudaEventRecordWithFlags(g_time_start[EPI % 2], st, ev_flags);
     }
-    if (CTAS == 1) {
-        umma_gemm_kernel<EPI, CTAS, TN><<<units, kGemmThreads, Cfg::kSmemBytes, st>>>(p);
-    } else {
-        cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3(units * 2);
-        cfg.blockDim = dim3(kGemmThreads);
-        cfg.dynamicSmemBytes = Cfg::kSmemBytes;
-        cfg.stream = st;
-        cudaLaunchAttribute attr;
-        attr.id = cudaLaunchAttributeClusterDimension;
-        attr.val.clusterDim.x = 2; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
-        cfg.attrs = &attr;
-        cfg.numAttrs = 1;
-        cudaLaunchKernelEx(&cfg, umma_gemm_kernel<EPI, CTAS, TN>, p);
-    }
+    launch_pdl(umma_gemm_kernel<EPI, CTAS, TN>, dim3(units * CTAS), dim3(kGemmThreads), Cfg::kSmemBytes, st, CTAS, p);
     const quaff_status_t rc = launch_status();
     if (timed) {
         cudaEventRecordWithFlags(g_time_stop[EPI % 2], st, ev_flags);
@@ -120,6 +106,8 @@ static quaff_status_t launch_gemm(const GemmParams& p, cudaStream_t st) {
 // ------------------------------------------------------------------ small kernels
 // dst[c][j] = src[j][c] for j < rows, 0 for rows <= j < rows_pad   (src is [rows][cols], dst is [cols][rows_pad])
 __global__ void transpose_pad_kernel(const uint16_t* __restrict__ src, int rows, int cols, uint16_t* __restrict__ dst, int rows_pad) {
+    pdl_launch_dependents();
+    pdl_wait();
     const int idx = blockIdx.x * blockDim.x + threadIdx.x;
     if (idx >= cols * rows_pad) return;
     const int c = idx / rows_pad, j = idx % rows_pad;
@@ -129,6 +117,8 @@ __global__ void transpose_pad_kernel(const uint16_t* __restrict__ src, int rows,
 // out[m][j] = bf16(scale * sum_s part[s][m][j])
 __global__ void reduce_parts_bf16_kernel(const float* __restrict__ part, int S, int rows, int r, float scale,
                                          uint16_t* __restrict__ out) {
+    pdl_launch_dependents();
+    pdl_wait();
     const int idx = blockIdx.x * blockDim.x + threadIdx.x;
     if (idx >= rows * r) return;
     float sum = 0.0f;
@@ -139,6 +129,8 @@ __global__ void reduce_parts_bf16_kernel(const float* __restrict__ part, int S, 
 // dst = (accumulate ? dst : 0) + scale * sum_s part[s][c][j];  dst index c*r + j, or j*C + c when transposed
 __global__ void reduce_parts_kernel(const float* __restrict__ part, int S, int C, int r, float scale, int transposed,
                                     int accumulate, float* __restrict__ dst) {
+    pdl_launch_dependents();
+    pdl_wait();
     const int idx = blockIdx.x * blockDim.x + threadIdx.x;
     if (idx >= C * r) return;
     int c, j;
@@ -162,6 +154,8 @@ __global__ void __launch_bounds__(256) dequant_weight_kernel(const int8_t* __res
                                                             const float* __restrict__ dw_O,
                                                             const int32_t* __restrict__ O_idx, int nO, int nOp, int K,
                                                             int Kpad, uint16_t* __restrict__ Wd, int64_t ldwd) {
+    pdl_launch_dependents();
+    pdl_wait();
     const int n = blockIdx.x;
     const int c = blockIdx.y * blockDim.x + threadIdx.x;
     const int k0 = c * 16;
@@ -203,6 +197,8 @@ __global__ void bwd_fixup_kernel(const float* __restrict__ P, int64_t ldp, int M
                                  const int32_t* __restrict__ O_idx, const float* __restrict__ s_O,
                                  const uint16_t* __restrict__ G, const uint16_t* __restrict__ A, int r,
                                  uint16_t* __restrict__ dX, int64_t lddx) {
+    pdl_launch_dependents();
+    pdl_wait();
     const int idx = blockIdx.x * blockDim.x + threadIdx.x;
     if (idx >= M * nO) return;
     const int m = idx / nO, i = idx % nO;
@@ -426,11 +422,11 @@ extern "C" quaff_status_t quaff_qlinear_fwd(int M, int K, int N, const int8_t* X
     }
     if (r > 0) {
         // LoRA down-projection T = bf16(X A): split-K tensor-core GEMM over K, then a reduction to bf16
-        transpose_pad_kernel<<<ceil_div(K * rp, 256), 256, 0, st>>>(A, K, r, At, K);   // At[j][k] = A[k][j]
+        launch_pdl(transpose_pad_kernel, dim3(ceil_div(K * rp, 256)), dim3(256), 0, st, 1, A, K, r, At, K);   // At[j][k] = A[k][j]
         if ((rc = launch_status()) != QUAFF_OK) return rc;
         int S = 1;
         if ((rc = skinny_gemm(0, X, ldx, At, K, M, K, r, part, status_opt, st, &S)) != QUAFF_OK) return rc;
-        reduce_parts_bf16_kernel<<<ceil_div(M * r, 256), 256, 0, st>>>(part, S, M, r, 1.0f, T_out);
+        launch_pdl(reduce_parts_bf16_kernel, dim3(ceil_div(M * r, 256)), dim3(256), 0, st, 1, part, S, M, r, 1.0f, T_out);
         if ((rc = launch_status()) != QUAFF_OK) return rc;
         // LoRA up: acc3 = T B over r; B [r][N] is read in place as an MN-major operand (rows = contraction)
         GemmPhase& ph = p.ph[np++];
@@ -485,7 +481,7 @@ extern "C" quaff_status_t quaff_qlinear_bwd(int M, int K, int N, const quaff_bf1
 
     if (r > 0) {   // G = bf16(lora_scale * dY B^T): B [r][N] is already K-major for this contraction over N
         if ((rc = skinny_gemm(0, dY, lddy, B, N, M, N, r, part, status_opt, st, &S)) != QUAFF_OK) return rc;
-        reduce_parts_bf16_kernel<<<ceil_div(M * r, 256), 256, 0, st>>>(part, S, M, r, lora_scale, G);
+        launch_pdl(reduce_parts_bf16_kernel, dim3(ceil_div(M * r, 256)), dim3(256), 0, st, 1, part, S, M, r, lora_scale, G);
         if ((rc = launch_status()) != QUAFF_OK) return rc;
     }
     if (dX) {
@@ -493,7 +489,7 @@ extern "C" quaff_status_t quaff_qlinear_bwd(int M, int K, int N, const quaff_bf1
         const int TN = w.tile_n, Kpad = w.Kpad;
         const int Kext = nOp > 0 ? Kpad + 2 * nOp : K;
         const int chunks = (Kpad + 2 * nOp) / 16;
-        dequant_weight_kernel<<<dim3(N, ceil_div(chunks, 256)), 256, 0, st>>>(Wq, ldwq_main, dW, wq_O, ldwq, dw_O, O_idx, nO, nOp, K,
+        launch_pdl(dequant_weight_kernel, dim3(N, ceil_div(chunks, 256)), dim3(256), 0, st, 1, Wq, ldwq_main, dW, wq_O, ldwq, dw_O, O_idx, nO, nOp, K,
                                                                             Kpad, Wd, w.ldwd);
         if ((rc = launch_status()) != QUAFF_OK) return rc;
         GemmParams p;
@@ -524,7 +520,7 @@ extern "C" quaff_status_t quaff_qlinear_bwd(int M, int K, int N, const quaff_bf1
         rc = TN == 256 ? launch_gemm<EPI_BWD, CTAS, 256>(p, st) : launch_gemm<EPI_BWD, CTAS, 128>(p, st);
         if (rc != QUAFF_OK) return rc;
         if (nO > 0) {
-            bwd_fixup_kernel<<<ceil_div(M * nO, 256), 256, 0, st>>>(P, 2 * nOp, M, nO, nOp, O_idx, s_O, G, A, r, dX, lddx);
+            launch_pdl(bwd_fixup_kernel, dim3(ceil_div(M * nO, 256)), dim3(256), 0, st, 1, P, (int64_t)(2 * nOp), M, nO, nOp, O_idx, s_O, G, A, r, dX, lddx);
             if ((rc = launch_status()) != QUAFF_OK) return rc;
         }
     }
@@ -532,10 +528,10 @@ extern "C" quaff_status_t quaff_qlinear_bwd(int M, int K, int N, const quaff_bf1
         // dA = X^T G and dB^T = dY^T T: the contraction runs over the tokens, the slow axis of X, G, dY and T,
         // so both operands are MN-major
         if ((rc = skinny_gemm(1, X, ldx, G, r, K, M, r, part, status_opt, st, &S)) != QUAFF_OK) return rc;
-        reduce_parts_kernel<<<ceil_div(K * r, 256), 256, 0, st>>>(part, S, K, r, 1.0f, 0, accumulate, dA);
+        launch_pdl(reduce_parts_kernel, dim3(ceil_div(K * r, 256)), dim3(256), 0, st, 1, part, S, K, r, 1.0f, 0, accumulate, dA);
         if ((rc = launch_status()) != QUAFF_OK) return rc;
         if ((rc = skinny_gemm(1, dY, lddy, T, r, N, M, r, part, status_opt, st, &S)) != QUAFF_OK) return rc;
-        reduce_parts_kernel<<<ceil_div(N * r, 256), 256, 0, st>>>(part, S, N, r, lora_scale, 1, accumulate, dB);
+        launch_pdl(reduce_parts_kernel, dim3(ceil_div(N * r, 256)), dim3(256), 0, st, 1, part, S, N, r, lora_scale, 1, accumulate, dB);
         if ((rc = launch_status()) != QUAFF_OK) return rc;
     }
     return QUAFF_OK;

@@ -108,6 +108,8 @@ __global__ void __launch_bounds__(256, QUAFF_QA_MIN_BLOCKS) quant_act_kernel(con
                                                         int8_t* __restrict__ Xq, int64_t ldxq,
                                                         int8_t* __restrict__ xq_O, int64_t ldxo, int nOp,
                                                         float* __restrict__ dx) {
+    pdl_launch_dependents();
+    pdl_wait();
     extern __shared__ __align__(16) unsigned char smem_raw[];
     const int tid = threadIdx.x, T = blockDim.x;
     float* red = reinterpret_cast<float*>(smem_raw);            // [2][8]
@@ -228,7 +230,7 @@ static quaff_status_t launch_quant_act(int T, const uint16_t* X, int64_t ldx, in
     if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, quant_act_kernel<J, TAIL>, T, smem) != cudaSuccess || per_sm < 1)
         per_sm = 1;
     const int grid = min(M, sm_count() * per_sm);
-    quant_act_kernel<J, TAIL><<<grid, T, smem, st>>>(X, ldx, M, K, O_idx, nO, s_O, Xq, ldxq, xq_O, ldxo, nOp, dx);
+    launch_pdl(quant_act_kernel<J, TAIL>, dim3(grid), dim3(T), smem, st, 1, X, ldx, M, K, O_idx, nO, s_O, Xq, ldxq, xq_O, ldxo, nOp, dx);
     return launch_status();
 }
 
@@ -269,6 +271,8 @@ __global__ void __launch_bounds__(256) momentum_kernel(const uint16_t* __restric
                                                        const float* __restrict__ wmax_O, float gamma,
                                                        float* __restrict__ s_O, float* __restrict__ colmax_opt,
                                                        float* __restrict__ beta_opt, unsigned int* __restrict__ ws) {
+    pdl_launch_dependents();
+    pdl_wait();
     __shared__ unsigned int red[8][32];
     __shared__ int is_last;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -327,6 +331,8 @@ constexpr int kRqCols = 32, kRqRows = 128, kRqPitch = kRqRows + 16;
 __global__ void __launch_bounds__(256) requant_rows_kernel(const uint16_t* __restrict__ W_O, int64_t ldwo, int nO, int N,
                                                            const float* __restrict__ s_O, int8_t* __restrict__ wq_O,
                                                            int64_t ldwq, int nOp, float* __restrict__ dw_O) {
+    pdl_launch_dependents();
+    pdl_wait();
     extern __shared__ __align__(16) unsigned char rq_smem[];
     float* sm1_s = reinterpret_cast<float*>(rq_smem);                 // [nO]: s - 1
     float* red = sm1_s + ((nO + 3) & ~3);                             // [8][32]
@@ -378,6 +384,8 @@ __global__ void __launch_bounds__(256) gather_outlier_rows_kernel(const uint16_t
                                                                  const int32_t* __restrict__ O_idx,
                                                                  uint16_t* __restrict__ W_O, int64_t ldwo,
                                                                  float* __restrict__ wmax_O) {
+    pdl_launch_dependents();
+    pdl_wait();
     __shared__ unsigned int red[8];
     const int i = blockIdx.x;
     const int col = O_idx[i];
@@ -434,8 +442,8 @@ extern "C" quaff_status_t quaff_momentum_update(const quaff_bf16* X, int64_t ldx
     cudaStream_t st = (cudaStream_t)stream;
     if (cudaMemsetAsync(ws, 0, (size_t)(nO + 1) * 4, st) != cudaSuccess) return QUAFF_ERR_CUDA;
     const int grid = max(1, min(ceil_div(M, 16), sm_count() * 2));
-    momentum_kernel<<<grid, 256, 0, st>>>(X, ldx, M, O_idx, nO, wmax_O, gamma, s_O, colmax_O_opt, beta_O_opt,
-                                          reinterpret_cast<unsigned int*>(ws));
+    launch_pdl(momentum_kernel, dim3(grid), dim3(256), 0, st, 1, X, ldx, M, O_idx, nO, wmax_O, gamma, s_O, colmax_O_opt, beta_O_opt,
+               reinterpret_cast<unsigned int*>(ws));
     return launch_status();
 }
 
@@ -448,7 +456,7 @@ extern "C" quaff_status_t quaff_requant_weight_rows(const quaff_bf16* W_O, int64
     QUAFF_RETURN_IF(nOp % 16, QUAFF_ERR_UNSUPPORTED_SHAPE);
     QUAFF_RETURN_IF(nOp > 0 && (!aligned16(wq_O) || (ldwq % 16)), QUAFF_ERR_ALIGNMENT);
     const size_t smem = (size_t)((nO + 3) & ~3) * 4 + 8 * kRqCols * 4 + (size_t)kRqCols * kRqPitch;
-    requant_rows_kernel<<<ceil_div(N, kRqCols), 256, smem, (cudaStream_t)stream>>>(W_O, ldwo, nO, N, s_O, wq_O, ldwq, nOp, dw_O);
+    launch_pdl(requant_rows_kernel, dim3(ceil_div(N, kRqCols)), dim3(256), smem, (cudaStream_t)stream, 1, W_O, ldwo, nO, N, s_O, wq_O, ldwq, nOp, dw_O);
     return launch_status();
 }
 
@@ -464,7 +472,7 @@ extern "C" quaff_status_t quaff_prepare_weight(const quaff_bf16* Wt, int64_t ldw
     quaff_status_t rc = quant_act_dispatch(Wt, ldw, N, K, nullptr, 0, nullptr, Wq, ldwq, nullptr, 0, 0, dW, st);
     if (rc != QUAFF_OK) return rc;
     if (nO > 0) {
-        gather_outlier_rows_kernel<<<nO, 256, 0, st>>>(Wt, ldw, N, O_idx, W_O, ldwo, wmax_O);
+        launch_pdl(gather_outlier_rows_kernel, dim3(nO), dim3(256), 0, st, 1, Wt, ldw, N, O_idx, W_O, ldwo, wmax_O);
         rc = launch_status();
     }
     return rc;
@@ -496,6 +504,6 @@ extern "C" quaff_status_t quaff_momentum_update_static(const quaff_bf16* X, int6
     // the array keeps the previous call's maxima and ticket count: both must start at zero
     if (cudaMemsetAsync(scratch, 0, (size_t)(nO + 1) * sizeof(unsigned int), st) != cudaSuccess) return QUAFF_ERR_CUDA;
     const int grid = max(1, min(ceil_div(M, 16), sm_count() * 2));
-    momentum_kernel<<<grid, 256, 0, st>>>(X, ldx, M, O_idx, nO, wmax_O, gamma, s_O, colmax_O_opt, beta_O_opt, scratch);
+    launch_pdl(momentum_kernel, dim3(grid), dim3(256), 0, st, 1, X, ldx, M, O_idx, nO, wmax_O, gamma, s_O, colmax_O_opt, beta_O_opt, scratch);
     return launch_status();
 }

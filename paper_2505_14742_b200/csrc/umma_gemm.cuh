@@ -178,11 +178,13 @@ __global__ void __launch_bounds__(kGemmThreads, 1) umma_gemm_kernel(const __grid
         tmem_alloc<CTAS>(smem_u32(&sm->tmem_base), 512);
         tmem_relinquish<CTAS>();
     }
+    pdl_launch_dependents();
     tc_fence_before();
     __syncthreads();
     if (CTAS == 2) cluster_sync();      // the peer's barriers exist before anything can signal them
     tc_fence_after();
     const uint32_t tmem_base = sm->tmem_base;
+    pdl_wait();                         // everything above overlapped the previous kernel; global memory only from here on
 
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer (both CTAs of a pair)
