@@ -11,7 +11,7 @@
  *
  * Conventions
  *  - Every pointer is a DEVICE pointer unless its comment says "host".  The caller owns every
- *    buffer; the library allocates nothing and keeps no state between calls.
+ *    buffer; the library allocates no memory and keeps no numerical state between calls.
  *  - All work is enqueued on the given stream; no call synchronises the device.
  *  - Matrices are row-major with leading dimensions given in ELEMENTS.
  *  - bf16 data are raw 16-bit patterns (quaff_bf16); INT8 codes are symmetric in [-127, 127].
@@ -117,6 +117,18 @@ quaff_status_t quaff_requant_weight_rows(const quaff_bf16* W_O, int64_t ldwo, in
                                          float* dw_O, quaff_stream_t stream);
 
 /*
+ * LoRA down-projection on its own: T_out [M][r] bf16 (dense) = bf16(X A), fp32 accumulation.  The paper's
+ * LoRA adapter reads the unquantized X, so this step depends on nothing the other entry points compute: a
+ * caller may run it on a second stream beside quaff_momentum_update / quaff_quant_act and hand the result to
+ * quaff_qlinear_fwd (X = NULL there).   X [M][K] bf16, ldx (ldx % 8 == 0);  A [K][r] bf16 dense;
+ * r a multiple of 8, <= 64; K a multiple of 8;  ws: QUAFF_WS_FWD bytes (its own, not shared with a call
+ * that runs concurrently);  status_opt as in the forward.
+ */
+quaff_status_t quaff_lora_down(const quaff_bf16* X, int64_t ldx, int M, int K, const quaff_bf16* A, int r,
+                               quaff_bf16* T_out, int32_t* status_opt, void* ws, size_t ws_bytes,
+                               quaff_stream_t stream);
+
+/*
  * Forward (Eq. 9) with the LoRA branch fused into the epilogue:
  *   acc1 = Xq Wq^T  (INT8 x INT8 -> INT32 over K),  acc2 = xq_O wq_O^T  (over nOp)
  *   T    = bf16(X A)                                                     [M][r], LoRA down-projection
@@ -125,7 +137,8 @@ quaff_status_t quaff_requant_weight_rows(const quaff_bf16* W_O, int64_t ldwo, in
  *   Wq [N][K], ldwq_main;  dW [N]                             frozen (quaff_prepare_weight)
  *   wq_O [N][nOp], ldwq;  dw_O [N]                            from quaff_requant_weight_rows
  *   X [M][K] bf16, ldx;  A [K][r] bf16;  B [r][N] bf16        LoRA (dense, ld = r and N); r == 0 disables
- *   T_out [M][r] bf16 (out, dense; kept for the backward)
+ *   T_out [M][r] bf16 (out, dense; kept for the backward).  With X = NULL (and r > 0), T_out is an INPUT:
+ *   T from an earlier quaff_lora_down on the same X and A; A and ws may then be NULL
  *   Y [M][N], ldy, y_dtype QUAFF_BF16 or QUAFF_F32 (out)
  *   dbg_acc_main, dbg_acc_out: optional dense [M][N] int32 dumps of acc1 / acc2 (parity checks)
  *   status_opt: optional int32[4] device word, must be zero on entry; see QUAFF_ERR_TIMEOUT
@@ -159,6 +172,11 @@ quaff_status_t quaff_qlinear_fwd(int M, int K, int N,
  *   dY [M][N] bf16, lddy (lddy % 8 == 0);  T [M][r] bf16 from the forward
  *   Wq, wq_O: 16-byte aligned, ldwq_main and ldwq multiples of 16 (as in the forward)
  *   ws: QUAFF_WS_BWD bytes;  status_opt as in the forward.
+ * Independent parts of the backward (weight dequantization, G, dB; later dA and the outlier fix-up) are forked
+ * onto two library-owned side streams per device and joined back into `stream` before the call returns its
+ * last launch: for the caller everything is still ordered on `stream`.  The side streams are created by the
+ * first backward call on a device (make that call outside any stream capture); under capture the forks become
+ * parallel branches of the captured graph.
  */
 quaff_status_t quaff_qlinear_bwd(int M, int K, int N,
                                  const quaff_bf16* dY, int64_t lddy,

@@ -24,7 +24,7 @@ QUAFF_ERR_TIMEOUT = 6
 QUAFF_BF16, QUAFF_F32 = 0, 1
 QUAFF_WS_PREPARE, QUAFF_WS_MOMENTUM, QUAFF_WS_FWD, QUAFF_WS_BWD = 0, 1, 2, 3
 
-EXPORTS = ("quaff_status_string", "quaff_workspace_bytes", "quaff_debug_launch_count", "quaff_debug_time_gemm", "quaff_prepare_weight", "quaff_momentum_update",
+EXPORTS = ("quaff_status_string", "quaff_workspace_bytes", "quaff_debug_launch_count", "quaff_debug_time_gemm", "quaff_prepare_weight", "quaff_momentum_update", "quaff_lora_down",
            "quaff_momentum_update_static", "quaff_quant_act", "quaff_requant_weight_rows", "quaff_qlinear_fwd", "quaff_qlinear_bwd")
 
 _lib = None
@@ -64,6 +64,8 @@ def lib() -> ctypes.CDLL:
         L.quaff_quant_act.argtypes = [_vp, _i64, _i32, _i32, _vp, _i32, _vp, _vp, _i64, _vp, _i64, _i32, _vp, _vp]
         L.quaff_requant_weight_rows.restype = _i32
         L.quaff_requant_weight_rows.argtypes = [_vp, _i64, _i32, _i32, _vp, _vp, _i64, _i32, _vp, _vp]
+        L.quaff_lora_down.restype = _i32
+        L.quaff_lora_down.argtypes = [_vp, _i64, _i32, _i32, _vp, _i32, _vp, _vp, _vp, _sz, _vp]
         L.quaff_qlinear_fwd.restype = _i32
         L.quaff_qlinear_fwd.argtypes = [_i32, _i32, _i32, _vp, _i64, _vp, _i64, _i32, _vp, _vp, _i64, _vp, _vp, _i64, _vp,
                                         _vp, _i64, _vp, _vp, _i32, _f32, _vp, _vp, _i32, _i64, _vp, _vp, _vp, _vp, _sz, _vp]
@@ -161,12 +163,18 @@ def quaff_requant_weight_rows(W_O, s_O, wq_O, dw_O) -> None:
            "quaff_requant_weight_rows")
 
 
+def quaff_lora_down(X, A, T_out, ws, status=None) -> None:
+    M, K = X.shape
+    _check(lib().quaff_lora_down(_ptr(X), _ld(X), M, K, _ptr(A), A.shape[1], _ptr(T_out), _ptr(status), _ptr(ws),
+                                 ws.numel() * ws.element_size(), _stream()), "quaff_lora_down")
+
+
 def quaff_qlinear_fwd(Xq, xq_O, dx, Wq, dW, wq_O, dw_O, X, A, B, lora_scale: float, T_out, Y, ws,
                       dbg_acc_main=None, dbg_acc_out=None, status=None) -> None:
     M, K = Xq.shape
     N = Wq.shape[0]
     nOp = 0 if xq_O is None else xq_O.shape[1]
-    r = 0 if A is None else A.shape[1]
+    r = 0 if B is None else B.shape[0]
     y_dtype = QUAFF_F32 if Y.dtype == torch.float32 else QUAFF_BF16
     _check(lib().quaff_qlinear_fwd(M, K, N, _ptr(Xq), _ld(Xq), _ptr(xq_O), _ld(xq_O) if xq_O is not None else 0, nOp,
                                    _ptr(dx), _ptr(Wq), _ld(Wq), _ptr(dW), _ptr(wq_O),

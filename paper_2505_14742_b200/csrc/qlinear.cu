@@ -41,6 +41,42 @@ quaff_status_t make_tmap_2d(CUtensorMap* map, const void* base, int elem_bytes, 
     return rc == CUDA_SUCCESS ? QUAFF_OK : QUAFF_ERR_CUDA;
 }
 
+// Side streams of the backward: work that does not depend on each other (the dequantization of the weight,
+// G = dY B^T, dB = T^T dY; later the outlier fix-up and dA = X^T G) is forked from the caller's stream onto
+// these and joined back with events, so the small kernels overlap instead of queueing.  One set per device,
+// created at the first backward call on that device; under stream capture the forks become parallel
+// branches of the graph.
+struct SideStreams {
+    cudaStream_t s[2];
+    cudaEvent_t fork[2], join[2];
+    bool ok;
+};
+static SideStreams* side_streams() {
+    static SideStreams per_dev[64];
+    static bool tried[64] = {false};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    SideStreams& ss = per_dev[dev];
+    if (!tried[dev]) {
+        tried[dev] = true;
+        ss.ok = true;
+        for (int i = 0; i < 2; ++i) {
+            ss.ok = ss.ok && cudaStreamCreateWithFlags(&ss.s[i], cudaStreamNonBlocking) == cudaSuccess;
+            ss.ok = ss.ok && cudaEventCreateWithFlags(&ss.fork[i], cudaEventDisableTiming) == cudaSuccess;
+            ss.ok = ss.ok && cudaEventCreateWithFlags(&ss.join[i], cudaEventDisableTiming) == cudaSuccess;
+        }
+        if (!ss.ok) cudaGetLastError();
+    }
+    return ss.ok ? &ss : nullptr;
+}
+// side stream i continues from the current end of `st` / `st` continues after side stream i
+static bool fork_to(SideStreams* ss, int i, cudaStream_t st) {
+    return cudaEventRecord(ss->fork[i], st) == cudaSuccess && cudaStreamWaitEvent(ss->s[i], ss->fork[i], 0) == cudaSuccess;
+}
+static bool join_from(SideStreams* ss, int i, cudaStream_t st) {
+    return cudaEventRecord(ss->join[i], ss->s[i]) == cudaSuccess && cudaStreamWaitEvent(st, ss->join[i], 0) == cudaSuccess;
+}
+
 static cudaEvent_t g_time_start[2] = {nullptr, nullptr};
 static cudaEvent_t g_time_stop[2] = {nullptr, nullptr};
 
@@ -314,7 +350,7 @@ static int bwd_tile_n(int M, int K, int nOp) {
 }
 
 struct BwdWorkspace {
-    size_t off_wd, off_g, off_p, off_part, total;
+    size_t off_wd, off_g, off_p, off_part, off_part_a, off_part_b, total;
     int tile_n;       // output-column tile of the grad-input GEMM
     int Kpad;         // K rounded up to tile_n
     int64_t ldwd;     // row pitch of Wd in elements
@@ -329,18 +365,45 @@ static BwdWorkspace bwd_workspace(int M, int K, int N, int nOp, int r) {
     w.off_wd = off;   off += round_up((size_t)N * (size_t)w.ldwd * 2, 256);
     w.off_g = off;    off += round_up((size_t)M * (size_t)max(r, 1) * 2, 256);
     w.off_p = off;    off += round_up((size_t)M * (size_t)max(2 * nOp, 1) * 4, 256);
-    w.off_part = off;
-    size_t pmax = split_part_bytes(M, N, r);                 // G = dY B^T
-    pmax = max(pmax, split_part_bytes(K, M, r));             // dA = X^T G
-    pmax = max(pmax, split_part_bytes(N, M, r));             // dB^T = dY^T T
-    off += round_up(pmax, 256);
+    // split-K partials: one buffer per skinny GEMM (they run concurrently)
+    w.off_part = off;   off += round_up(split_part_bytes(M, N, r), 256);   // G = dY B^T
+    w.off_part_a = off; off += round_up(split_part_bytes(K, M, r), 256);   // dA = X^T G
+    w.off_part_b = off; off += round_up(split_part_bytes(N, M, r), 256);   // dB^T = dY^T T
     w.total = off;
     return w;
+}
+
+// T = bf16(X A): At = A^T (K-major operand), split-K tensor-core GEMM over K, reduction to bf16
+static quaff_status_t lora_down(const quaff_bf16* X, int64_t ldx, int M, int K, const quaff_bf16* A, int r, quaff_bf16* T_out,
+                                const FwdWorkspace& w, void* ws, int32_t* status_opt, cudaStream_t st) {
+    unsigned char* base = reinterpret_cast<unsigned char*>(ws);
+    uint16_t* At = reinterpret_cast<uint16_t*>(base + w.off_at);
+    float* part = reinterpret_cast<float*>(base + w.off_part);
+    const int rp = pad16(r);
+    quaff_status_t rc;
+    launch_pdl(transpose_pad_kernel, dim3(ceil_div(K * rp, 256)), dim3(256), 0, st, 1, A, K, r, At, K);   // At[j][k] = A[k][j]
+    if ((rc = launch_status()) != QUAFF_OK) return rc;
+    int S = 1;
+    if ((rc = skinny_gemm(0, X, ldx, At, K, M, K, r, part, status_opt, st, &S)) != QUAFF_OK) return rc;
+    launch_pdl(reduce_parts_bf16_kernel, dim3(ceil_div(M * r, 256)), dim3(256), 0, st, 1, part, S, M, r, 1.0f, T_out);
+    return launch_status();
 }
 
 }  // namespace quaff
 
 using namespace quaff;
+
+extern "C" quaff_status_t quaff_lora_down(const quaff_bf16* X, int64_t ldx, int M, int K, const quaff_bf16* A, int r,
+                                          quaff_bf16* T_out, int32_t* status_opt, void* ws, size_t ws_bytes,
+                                          quaff_stream_t stream) {
+    QUAFF_RETURN_IF(M < 0 || K <= 0 || r <= 0 || !X || !A || !T_out || ldx < K, QUAFF_ERR_INVALID_ARG);
+    QUAFF_RETURN_IF((r % 8) || r > 64 || (K % 8), QUAFF_ERR_UNSUPPORTED_SHAPE);
+    QUAFF_RETURN_IF(!aligned16(X) || !aligned16(T_out) || (ldx % 8), QUAFF_ERR_ALIGNMENT);
+    const FwdWorkspace w = fwd_workspace(M, K, 0, r);
+    QUAFF_RETURN_IF(!ws || !aligned16(ws) || ws_bytes < w.total, QUAFF_ERR_WORKSPACE_TOO_SMALL);
+    if (M == 0) return QUAFF_OK;
+    return lora_down(X, ldx, M, K, A, r, T_out, w, ws, status_opt, (cudaStream_t)stream);
+}
 
 extern "C" uint64_t quaff_debug_launch_count(void) { return g_launch_count; }
 
@@ -383,22 +446,22 @@ extern "C" quaff_status_t quaff_qlinear_fwd(int M, int K, int N, const int8_t* X
     QUAFF_RETURN_IF(M < 0 || K <= 0 || N <= 0 || nOp < 0 || r < 0, QUAFF_ERR_INVALID_ARG);
     QUAFF_RETURN_IF(!Xq || !dx || !Wq || !dW || !Y || ldxq < K || ldwq_main < K || ldy < N, QUAFF_ERR_INVALID_ARG);
     QUAFF_RETURN_IF(nOp > 0 && (!xq_O || !wq_O || !dw_O || ldxo < nOp || ldwq < nOp), QUAFF_ERR_INVALID_ARG);
-    QUAFF_RETURN_IF(r > 0 && (!X || !A || !B || !T_out || ldx < K), QUAFF_ERR_INVALID_ARG);
+    const bool have_T = r > 0 && !X;      // T_out already holds T = bf16(X A) (quaff_lora_down)
+    QUAFF_RETURN_IF(r > 0 && (!B || !T_out), QUAFF_ERR_INVALID_ARG);
+    QUAFF_RETURN_IF(r > 0 && !have_T && (!A || ldx < K), QUAFF_ERR_INVALID_ARG);
     QUAFF_RETURN_IF(y_dtype != QUAFF_BF16 && y_dtype != QUAFF_F32, QUAFF_ERR_INVALID_ARG);
     QUAFF_RETURN_IF((nOp % 32) || (r % 8) || r > 64, QUAFF_ERR_UNSUPPORTED_SHAPE);
     QUAFF_RETURN_IF(r > 0 && ((K % 8) || (N % 8)), QUAFF_ERR_UNSUPPORTED_SHAPE);
     QUAFF_RETURN_IF(!aligned16(Xq) || !aligned16(Wq) || (ldxq % 16) || (ldwq_main % 16), QUAFF_ERR_ALIGNMENT);
     QUAFF_RETURN_IF(nOp > 0 && (!aligned16(xq_O) || !aligned16(wq_O) || (ldxo % 16) || (ldwq % 16)), QUAFF_ERR_ALIGNMENT);
-    QUAFF_RETURN_IF(r > 0 && (!aligned16(X) || !aligned16(T_out) || !aligned16(B) || (ldx % 8)), QUAFF_ERR_ALIGNMENT);
+    QUAFF_RETURN_IF(r > 0 && (!aligned16(T_out) || !aligned16(B)), QUAFF_ERR_ALIGNMENT);
+    QUAFF_RETURN_IF(r > 0 && !have_T && (!aligned16(X) || (ldx % 8)), QUAFF_ERR_ALIGNMENT);
     QUAFF_RETURN_IF(!aligned16(Y), QUAFF_ERR_ALIGNMENT);
     const FwdWorkspace w = fwd_workspace(M, K, N, r);
-    QUAFF_RETURN_IF(r > 0 && (!ws || !aligned16(ws) || ws_bytes < w.total), QUAFF_ERR_WORKSPACE_TOO_SMALL);
+    QUAFF_RETURN_IF(r > 0 && !have_T && (!ws || !aligned16(ws) || ws_bytes < w.total), QUAFF_ERR_WORKSPACE_TOO_SMALL);
     if (M == 0) return QUAFF_OK;
     cudaStream_t st = (cudaStream_t)stream;
     const int rp = pad16(r);
-    unsigned char* base = reinterpret_cast<unsigned char*>(ws);
-    uint16_t* At = reinterpret_cast<uint16_t*>(base + w.off_at);
-    float* part = reinterpret_cast<float*>(base + w.off_part);
     constexpr int CTAS = 2;
     // Three accumulators (main, outlier, LoRA) fit TMEM only with 128-column tiles; Eq. 2 alone (no outlier
     // set, no LoRA) takes the 256-column tile.
@@ -421,13 +484,8 @@ extern "C" quaff_status_t quaff_qlinear_fwd(int M, int K, int N, const int8_t* X
         fill_phase(ph, 1, nOp, 1, 1, 1 << 30, TN, CTAS, 0, 0, 64, TN);
     }
     if (r > 0) {
-        // LoRA down-projection T = bf16(X A): split-K tensor-core GEMM over K, then a reduction to bf16
-        launch_pdl(transpose_pad_kernel, dim3(ceil_div(K * rp, 256)), dim3(256), 0, st, 1, A, K, r, At, K);   // At[j][k] = A[k][j]
-        if ((rc = launch_status()) != QUAFF_OK) return rc;
-        int S = 1;
-        if ((rc = skinny_gemm(0, X, ldx, At, K, M, K, r, part, status_opt, st, &S)) != QUAFF_OK) return rc;
-        launch_pdl(reduce_parts_bf16_kernel, dim3(ceil_div(M * r, 256)), dim3(256), 0, st, 1, part, S, M, r, 1.0f, T_out);
-        if ((rc = launch_status()) != QUAFF_OK) return rc;
+        // LoRA down-projection T = bf16(X A), unless the caller has run it already
+        if (!have_T && (rc = lora_down(X, ldx, M, K, A, r, T_out, w, ws, status_opt, st)) != QUAFF_OK) return rc;
         // LoRA up: acc3 = T B over r; B [r][N] is read in place as an MN-major operand (rows = contraction)
         GemmPhase& ph = p.ph[np++];
         if ((rc = make_tmap_2d(&ph.map_a, T_out, 2, M, r, r, kTileM, 64)) != QUAFF_OK) return rc;
@@ -476,22 +534,41 @@ extern "C" quaff_status_t quaff_qlinear_bwd(int M, int K, int N, const quaff_bf1
     uint16_t* G = reinterpret_cast<uint16_t*>(base + w.off_g);
     float* P = reinterpret_cast<float*>(base + w.off_p);
     float* part = reinterpret_cast<float*>(base + w.off_part);
+    float* part_a = reinterpret_cast<float*>(base + w.off_part_a);
+    float* part_b = reinterpret_cast<float*>(base + w.off_part_b);
     quaff_status_t rc;
     int S = 1;
+    const bool want_dAB = r > 0 && dA && dB;
+    // Dependencies:  dB = T^T dY needs nothing computed here;  the weight dequantization neither;
+    // G = dY B^T feeds the grad-input GEMM and dA = X^T G;  the outlier fix-up follows the GEMM.
+    SideStreams* ss = side_streams();
+    cudaStream_t s_deq = ss ? ss->s[0] : st;       // dequantization, later dA
+    cudaStream_t s_db = ss ? ss->s[1] : st;        // dB
+    bool forked0 = false, forked1 = false;
 
+    if (want_dAB) {   // dB^T = dY^T T: the contraction runs over the tokens, the slow axis of dY and T: MN-major operands
+        if (ss && !(forked1 = fork_to(ss, 1, st))) return QUAFF_ERR_CUDA;
+        if ((rc = skinny_gemm(1, dY, lddy, T, r, N, M, r, part_b, status_opt, s_db, &S)) != QUAFF_OK) return rc;
+        launch_pdl(reduce_parts_kernel, dim3(ceil_div(N * r, 256)), dim3(256), 0, s_db, 1, part_b, S, N, r, lora_scale, 1, accumulate, dB);
+        if ((rc = launch_status()) != QUAFF_OK) return rc;
+    }
+    constexpr int CTAS = 2;
+    const int TN = w.tile_n, Kpad = w.Kpad;
+    const int Kext = nOp > 0 ? Kpad + 2 * nOp : K;
+    if (dX) {
+        if (ss && !(forked0 = fork_to(ss, 0, st))) return QUAFF_ERR_CUDA;
+        const int chunks = (Kpad + 2 * nOp) / 16;
+        launch_pdl(dequant_weight_kernel, dim3(N, ceil_div(chunks, 256)), dim3(256), 0, s_deq, 1, Wq, ldwq_main, dW, wq_O, ldwq, dw_O, O_idx,
+                   nO, nOp, K, Kpad, Wd, w.ldwd);
+        if ((rc = launch_status()) != QUAFF_OK) return rc;
+    }
     if (r > 0) {   // G = bf16(lora_scale * dY B^T): B [r][N] is already K-major for this contraction over N
         if ((rc = skinny_gemm(0, dY, lddy, B, N, M, N, r, part, status_opt, st, &S)) != QUAFF_OK) return rc;
         launch_pdl(reduce_parts_bf16_kernel, dim3(ceil_div(M * r, 256)), dim3(256), 0, st, 1, part, S, M, r, lora_scale, G);
         if ((rc = launch_status()) != QUAFF_OK) return rc;
     }
     if (dX) {
-        constexpr int CTAS = 2;
-        const int TN = w.tile_n, Kpad = w.Kpad;
-        const int Kext = nOp > 0 ? Kpad + 2 * nOp : K;
-        const int chunks = (Kpad + 2 * nOp) / 16;
-        launch_pdl(dequant_weight_kernel, dim3(N, ceil_div(chunks, 256)), dim3(256), 0, st, 1, Wq, ldwq_main, dW, wq_O, ldwq, dw_O, O_idx, nO, nOp, K,
-                                                                            Kpad, Wd, w.ldwd);
-        if ((rc = launch_status()) != QUAFF_OK) return rc;
+        if (forked0 && !join_from(ss, 0, st)) return QUAFF_ERR_CUDA;     // the dequantized weight is ready
         GemmParams p;
         memset(&p, 0, sizeof(p));
         int np = 0;
@@ -519,20 +596,27 @@ extern "C" quaff_status_t quaff_qlinear_bwd(int M, int K, int N, const quaff_bf1
         p.dX = dX; p.lddx = lddx; p.P = P; p.ldp = 2 * nOp;
         rc = TN == 256 ? launch_gemm<EPI_BWD, CTAS, 256>(p, st) : launch_gemm<EPI_BWD, CTAS, 128>(p, st);
         if (rc != QUAFF_OK) return rc;
-        if (nO > 0) {
-            launch_pdl(bwd_fixup_kernel, dim3(ceil_div(M * nO, 256)), dim3(256), 0, st, 1, P, (int64_t)(2 * nOp), M, nO, nOp, O_idx, s_O, G, A, r, dX, lddx);
-            if ((rc = launch_status()) != QUAFF_OK) return rc;
+    }
+    if (want_dAB) {   // dA = X^T G (MN-major operands), beside the outlier fix-up
+        cudaStream_t s_da = st;
+        bool forked_da = false;
+        if (ss && dX && nO > 0) {
+            if (!(forked_da = fork_to(ss, 0, st))) return QUAFF_ERR_CUDA;
+            s_da = ss->s[0];
         }
-    }
-    if (r > 0 && dA && dB) {
-        // dA = X^T G and dB^T = dY^T T: the contraction runs over the tokens, the slow axis of X, G, dY and T,
-        // so both operands are MN-major
-        if ((rc = skinny_gemm(1, X, ldx, G, r, K, M, r, part, status_opt, st, &S)) != QUAFF_OK) return rc;
-        launch_pdl(reduce_parts_kernel, dim3(ceil_div(K * r, 256)), dim3(256), 0, st, 1, part, S, K, r, 1.0f, 0, accumulate, dA);
+        if ((rc = skinny_gemm(1, X, ldx, G, r, K, M, r, part_a, status_opt, s_da, &S)) != QUAFF_OK) return rc;
+        launch_pdl(reduce_parts_kernel, dim3(ceil_div(K * r, 256)), dim3(256), 0, s_da, 1, part_a, S, K, r, 1.0f, 0, accumulate, dA);
         if ((rc = launch_status()) != QUAFF_OK) return rc;
-        if ((rc = skinny_gemm(1, dY, lddy, T, r, N, M, r, part, status_opt, st, &S)) != QUAFF_OK) return rc;
-        launch_pdl(reduce_parts_kernel, dim3(ceil_div(N * r, 256)), dim3(256), 0, st, 1, part, S, N, r, lora_scale, 1, accumulate, dB);
+        forked0 = forked_da;
+    } else {
+        forked0 = false;
+    }
+    if (dX && nO > 0) {
+        launch_pdl(bwd_fixup_kernel, dim3(ceil_div(M * nO, 256)), dim3(256), 0, st, 1, P, (int64_t)(2 * nOp), M, nO, nOp, O_idx, s_O, G, A, r,
+                   dX, lddx);
         if ((rc = launch_status()) != QUAFF_OK) return rc;
     }
+    if (forked0 && !join_from(ss, 0, st)) return QUAFF_ERR_CUDA;
+    if (forked1 && !join_from(ss, 1, st)) return QUAFF_ERR_CUDA;
     return QUAFF_OK;
 }

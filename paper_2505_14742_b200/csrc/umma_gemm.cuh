@@ -121,8 +121,12 @@ struct GemmCfg {
     static constexpr int kStageBytes = kABytes + kBBytes;
     static constexpr int kScaleBytes = (EPI == EPI_FWD) ? 2 * 2 * TN * 4 : 0;   // [2 buffers][dW | dw_O][TN]
     static constexpr int kFixed = 1024 + (int)sizeof(GemmSmem) + kScaleBytes;
+    // The skinny split-K GEMMs run a handful of k-blocks per CTA: a short ring and half of TMEM leave room
+    // for a second such CTA (or other kernels) on the same SM, so that independent ones overlap.
+    static constexpr int kStageCap = (EPI == EPI_PART) ? 4 : kMaxStages;
+    static constexpr int kTmemCols = (EPI == EPI_PART) ? 2 * TN : 512;
     static constexpr int kStagesFit = (kSmemLimit - kFixed) / kStageBytes;
-    static constexpr int kStages = kStagesFit < kMaxStages ? kStagesFit : kMaxStages;
+    static constexpr int kStages = kStagesFit < kStageCap ? kStagesFit : kStageCap;
     static constexpr size_t kSmemBytes = (size_t)kFixed + (size_t)kStages * kStageBytes;
 };
 
@@ -175,7 +179,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) umma_gemm_kernel(const __grid
         fence_barrier_init();
     }
     if (warp == 1) {
-        tmem_alloc<CTAS>(smem_u32(&sm->tmem_base), 512);
+        tmem_alloc<CTAS>(smem_u32(&sm->tmem_base), Cfg::kTmemCols);
         tmem_relinquish<CTAS>();
     }
     pdl_launch_dependents();
@@ -425,7 +429,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) umma_gemm_kernel(const __grid
     if (warp == 1) {
         __syncwarp();
         tc_fence_after();
-        tmem_dealloc<CTAS>(tmem_base, 512);
+        tmem_dealloc<CTAS>(tmem_base, Cfg::kTmemCols);
     }
 }
 

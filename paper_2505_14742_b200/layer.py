@@ -61,6 +61,9 @@ class QuaffLinear:
                        Q.workspace_bytes(Q.QUAFF_WS_FWD, M, K, N, nOp, r),
                        Q.workspace_bytes(Q.QUAFF_WS_BWD, M, K, N, nOp, r), 256)
         self.ws = torch.empty(ws_bytes, dtype=torch.uint8, device=dev)
+        # the LoRA down-projection runs beside the quantization chain, on its own stream and workspace
+        self.ws_lora = torch.empty(max(Q.workspace_bytes(Q.QUAFF_WS_FWD, M, K, N, nOp, r), 256), dtype=torch.uint8, device=dev) if r else None
+        self.side = torch.cuda.Stream(device=dev) if r else None
         Q.quaff_prepare_weight(Wt, O_idx, self.Wq, self.dW, self.W_O, self.wmax_O)
 
     def forward(self, X: torch.Tensor) -> torch.Tensor:
@@ -69,11 +72,18 @@ class QuaffLinear:
         Xq, dx, Y = self.Xq[:M], self.dx[:M], self.Y[:M]
         xq_O = self.xq_O[:M] if self.nOp else None
         T = self.T[:M] if self.r else None
+        main = torch.cuda.current_stream()
+        if self.r:     # T = X A needs only X: fork it off
+            self.side.wait_stream(main)
+            with torch.cuda.stream(self.side):
+                Q.quaff_lora_down(X, self.A, T, self.ws_lora, self.status)
         if self.nO:
             Q.quaff_momentum_update(X, self.O_idx, self.wmax_O, self.gamma, self.s_O, self.ws, self.colmax_O, self.beta_O)
             Q.quaff_requant_weight_rows(self.W_O, self.s_O, self.wq_O, self.dw_O)
         Q.quaff_quant_act(X, self.O_idx, self.s_O, Xq, xq_O, dx)
-        Q.quaff_qlinear_fwd(Xq, xq_O, dx, self.Wq, self.dW, self.wq_O, self.dw_O, X, self.A, self.B, self.lora_scale,
+        if self.r:
+            main.wait_stream(self.side)
+        Q.quaff_qlinear_fwd(Xq, xq_O, dx, self.Wq, self.dW, self.wq_O, self.dw_O, None, None, self.B, self.lora_scale,
                             T, Y, self.ws,
                             self.acc_main[:M] if self.acc_main is not None else None,
                             self.acc_out[:M] if self.acc_out is not None else None, self.status)
