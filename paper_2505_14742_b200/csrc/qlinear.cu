@@ -569,6 +569,9 @@ extern "C" quaff_status_t quaff_qlinear_bwd(int M, int K, int N, const quaff_bf1
     }
     if (dX) {
         if (forked0 && !join_from(ss, 0, st)) return QUAFF_ERR_CUDA;     // the dequantized weight is ready
+        // dB is joined here too: the persistent GEMM wants every SM, a straggler beside it only delays its CTAs
+        if (forked1 && !join_from(ss, 1, st)) return QUAFF_ERR_CUDA;
+        forked1 = false;
         GemmParams p;
         memset(&p, 0, sizeof(p));
         int np = 0;
