@@ -353,8 +353,63 @@ def run_gpu(args, wl):
         dist.destroy_process_group()
 
 
+def run_micro(args):
+    """--micro NAME: one HBM-bound kernel alone on rows of a given shape, L2 flushed (read-only sweep of a
+    512 MB buffer) before every launch, CUDA events around each launch; prints its own JSON line.  Used for
+    the per-kernel rooflines and as the small command of the ncu captures."""
+    import torch
+    from paper_2505_14742_b200 import binding as Q, build
+    build.build_library()
+    Q.lib()
+    torch.cuda.set_device(0)
+    M, K, N, nO = args.micro_shape
+    nOp = synth.pad_to(nO, 32)
+    g = torch.Generator(device="cuda").manual_seed(1234)
+    X = torch.randn((M, K), device="cuda", generator=g).to(torch.bfloat16)
+    O = torch.sort(torch.randperm(K, device="cuda", generator=g)[:nO])[0].to(torch.int32)
+    X[:, O.long()] *= 50.0
+    s = 1.0 + 10.0 * torch.rand(nO, device="cuda", generator=g)
+    flush = torch.empty(512 << 20, dtype=torch.uint8, device="cuda")
+    if args.micro == "quant_act":
+        Xq = torch.empty((M, K), dtype=torch.int8, device="cuda")
+        xqo = torch.empty((M, nOp), dtype=torch.int8, device="cuda")
+        dx = torch.empty(M, device="cuda")
+        fn = lambda: Q.quaff_quant_act(X, O, s, Xq, xqo, dx)
+        nbytes = M * K * 3 + M * nOp + 4 * M
+    elif args.micro == "momentum":
+        wmax = 0.05 + 0.05 * torch.rand(nO, device="cuda", generator=g)
+        ws = torch.empty(Q.workspace_bytes(Q.QUAFF_WS_MOMENTUM, M, K, N, nOp, 0), dtype=torch.uint8, device="cuda")
+        fn = lambda: Q.quaff_momentum_update(X, O, wmax, 0.2, s, ws)
+        nbytes = 32 * M * nO            # one 32-byte sector per gathered element
+    else:
+        W_O = (0.02 * torch.randn((nO, N), device="cuda", generator=g)).to(torch.bfloat16)
+        wq = torch.empty((N, nOp), dtype=torch.int8, device="cuda")
+        dw = torch.empty(N, device="cuda")
+        fn = lambda: Q.quaff_requant_weight_rows(W_O, s, wq, dw)
+        nbytes = 2 * nO * N + nOp * N + 4 * N
+    times = []
+    for i in range(args.warmup + args.steps):
+        flush.sum()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(); fn(); e1.record()
+        torch.cuda.synchronize()
+        if i >= args.warmup:
+            times.append(e0.elapsed_time(e1))
+    ms = float(np.median(times))
+    peaks = load_peaks()
+    gbs = nbytes / (ms * 1e-3) / 1e9
+    print(json.dumps({"micro": args.micro, "shape": {"M": M, "K": K, "N": N, "nO": nO}, "ms_per_launch": ms, "launches": len(times),
+                      "roofline": {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                                   "frac": gbs / peaks["hbm_gbs"], "algorithmic_bytes": nbytes,
+                                   "peak_source": f"{peaks['source']} copy bandwidth"}}), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
+    ap.add_argument("--micro", default=None, choices=["quant_act", "momentum", "requant"],
+                    help="time one HBM-bound kernel alone instead of the step")
+    ap.add_argument("--micro-shape", type=lambda v: tuple(int(x) for x in v.split(",")), default=(8192, 11008, 4096, 55),
+                    help="M,K,N,nO of --micro (default: the LLaMA-2-7B down_proj rows)")
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=1000)
     ap.add_argument("--warmup", type=int, default=5)
@@ -365,6 +420,10 @@ def main():
     ap.add_argument("--eager", action="store_true", help="enqueue every launch from Python instead of replaying a CUDA graph of the step")
     args = ap.parse_args()
     wl = synth.WORKLOADS[args.workload]
+    if args.micro:
+        if args.steps == 1000:
+            args.steps = 30
+        return run_micro(args)
     if args.impl == "reference":
         run_reference(args, wl)
     else:
