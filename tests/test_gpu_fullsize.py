@@ -114,3 +114,56 @@ def test_phi3_attn_o_proj_full_size():
 
 def test_llama7b_down_proj_full_size():
     _run_layer(synth.WORKLOADS["llama7b_block"], 6, steps=1, nsample=24, check_acc=True, full_grads=False)
+
+
+def test_phi3_mlp_late_outliers_momentum_adaptation():
+    """Configuration 'phi3_mlp': two members of O are dormant (magnitude 1) until step 100.  The scale state is
+    carried over 112 steps through the momentum / requant / quant_act entry points and compared bit-exactly with
+    the oracle at every step (cheap: O(M nO) per step); around the wake-up (steps 99-102, 111) the activation
+    codes and the re-quantized rows are compared in full as well, and the late channels' scale must have left 1."""
+    import torch
+    from paper_2505_14742_b200 import binding as Q, build
+    build.build_library()
+    wl = synth.WORKLOADS["phi3_mlp"]
+    li = 1                                              # down_proj 8192 -> 3072, nO = 82 incl. 2 late
+    lin = synth.layer_inputs(wl, li)
+    sp = lin.spec
+    M, K, N = 512, sp.K, sp.N                           # a 512-token slice of the 4096: the state logic does not depend on M
+    nOp = synth.pad_to(sp.nO, 32)
+    Wq, dW, W_O, wmax = oracle.prepare_weight(lin.W, lin.O_idx)
+    O_d, wmax_d, W_O_d = dev(lin.O_idx), dev(wmax), dev_bf16(W_O)
+    s_d = torch.ones(sp.nO, dtype=torch.float32, device="cuda")
+    ws = torch.empty(Q.workspace_bytes(Q.QUAFF_WS_MOMENTUM, M, K, N, nOp, 0), dtype=torch.uint8, device="cuda")
+    Xq = torch.empty((M, K), dtype=torch.int8, device="cuda")
+    xqo = torch.empty((M, nOp), dtype=torch.int8, device="cuda")
+    dx = torch.empty(M, dtype=torch.float32, device="cuda")
+    wq = torch.empty((N, nOp), dtype=torch.int8, device="cuda")
+    dw = torch.empty(N, dtype=torch.float32, device="cuda")
+    s = np.ones(sp.nO, np.float32)
+    for step in range(112):
+        mag = synth.outlier_magnitude(wl.seed, li, step, lin.base, sp.late)
+        X = synth.activations(wl.seed, li, step, M, K, lin.O_idx, mag)
+        Xd = dev_bf16(X)
+        Q.quaff_momentum_update(Xd, O_d, wmax_d, wl.gamma, s_d, ws)
+        s, _, _ = oracle.momentum_update(X, lin.O_idx, wmax, wl.gamma, s)
+        assert np.array_equal(host(s_d), s), f"s_O, step {step}"
+        if step in (0, 99, 100, 101, 102, 111):
+            Q.quaff_requant_weight_rows(W_O_d, s_d, wq, dw)
+            Q.quaff_quant_act(Xd, O_d, s_d, Xq, xqo, dx)
+            torch.cuda.synchronize()
+            oXq, oxqo, odx = oracle.quant_act(X, lin.O_idx, s, nOp)
+            owq, odw = oracle.requant_weight_rows(W_O, s, nOp)
+            assert np.array_equal(host(Xq), oXq) and np.array_equal(host(xqo), oxqo) and np.array_equal(host(dx), odx), step
+            assert np.array_equal(host(wq), owq) and np.array_equal(host(dw), odw), step
+        if step == 99:
+            assert np.all(s[-sp.late:] < 12.0), "dormant channels: beta = sqrt(max|x| / max|w|) of an ordinary N(0,1) channel, about 7"
+        if step == 111:
+            assert np.all(s[-sp.late:] > 25.0), "the late outlier channels (20-100x) have been picked up by the momentum update"
+
+
+@pytest.mark.parametrize("M,K,N,r,frac", [(512, 2048, 4096, 8, 0.05), (2048, 8192, 2048, 32, 0.01), (32768, 2048, 2048, 64, 0.005)])
+def test_shape_sweep_points(M, K, N, r, frac):
+    """Points of the shape sweep (tokens x K x N x rank x outlier fraction), one step each; 5 % of 2048 channels is
+    nO = 102 (the 128-column forward with nOp = 128)."""
+    wl = synth.sweep_point(M, K, N, r, frac)
+    _run_layer(wl, 0, steps=1, nsample=16, check_acc=True, full_grads=False)
