@@ -134,7 +134,7 @@ def cpu_baseline(wl, sample_tokens=16, reps=1):
     lins, state = oracle_setup(wl, sample_tokens)
     best = min(oracle_sample_step(wl, sample_tokens, lins, state) for _ in range(reps))
     return {"value": sample_tokens / best, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
-            "sample": f"{sample_tokens} of {wl.M} tokens through all {len(wl.layers)} layers, fwd+bwd, {best:.2f} s"}
+            "sample": f"{sample_tokens} of {wl.M} tokens through all {len(wl.layers)} layers, fwd+bwd; best of {reps} runs, {best:.2f} s each"}
 
 
 def run_reference(args, wl):
@@ -363,7 +363,7 @@ def run_gpu(args, wl):
                                + (" x2 (nominal int8:bf16 ratio)" if kind == "fwd_int8_gemm" else ""),
                 "avg_launch_ms": ms}
 
-    cpu = cpu_baseline(wl, min(wl.M, 8 * args.sample_tokens)) if not args.no_cpu_baseline else None
+    cpu = cpu_baseline(wl, min(wl.M, 8 * args.sample_tokens), reps=5) if not args.no_cpu_baseline else None
     line = {"metric": METRIC, "value": qdist.whole_job_rate(M, world, ms_per_step), "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "int8 forward (int32 accumulate), bf16 backward (f32 accumulate)",
