@@ -206,3 +206,21 @@ def qlinear_bwd(dY, Wq, dW, wq_O, dw_O, O_idx, s_O, X, T, A, B, lora_scale: floa
                            _p(X), I64(K), _p(T_), _p(A_), _p(B_), I32(r), F32(lora_scale),
                            _p(dX), _p(dA), _p(dB), _p(G))
     return dX, dA, dB, G[:, :r]
+
+
+def outlier_count(X: np.ndarray, thr: int, xi: np.ndarray) -> np.ndarray:
+    """Eq. 6 for one calibration sample X[M,K] (bf16 bits): returns xi + indicator (xi is not modified)."""
+    X = _c(X, np.uint16)
+    M, K = X.shape
+    out = _c(xi, np.int32).copy()
+    _load().qo_outlier_count(_p(X), I64(K), I32(M), I32(K), I32(int(thr)), _p(out))
+    return out
+
+
+def select_outliers(xi: np.ndarray, nO: int) -> np.ndarray:
+    """The nO channels with the largest xi (ties: lower index first), sorted ascending (int32)."""
+    xi = _c(xi, np.int32)
+    O = np.empty(nO, np.int32)
+    _load().qo_select_outliers(_p(xi), I32(xi.shape[0]), I32(nO), _p(O))
+    return O
+

@@ -358,3 +358,46 @@ void qo_qlinear_bwd(int M, int K, int N,
     }
     free(G);
 }
+
+/* ---------------------------------------------------------------- calibration, Eq. 6
+ * One calibration sample X^i [M][K]:  xi[o] += 1  if  max_m |X[m][o]| > thr * mean(|X|).
+ * So that the indicator is one well-defined integer decision, |x| is taken in units of 2^-16,
+ * truncated (anything below 2^-16 counts as 0) and saturating at 2^32 - 1:
+ *     a(x) = min(floor(|x| * 65536), 2^32 - 1)
+ * and the comparison is made without any division:  a(max_o) * (M * K)  >  thr * sum_{m,k} a(X[m][k]).
+ */
+static uint64_t abs_fix16(uint16_t b) {
+    double f = floor(fabs((double)bf2f(b)) * 65536.0); /* exact: bf16 -> double, scaling by a power of two */
+    return f >= 4294967295.0 ? 4294967295ull : (uint64_t)f;
+}
+
+void qo_outlier_count(const uint16_t* X, int64_t ldx, int M, int K, int thr, int32_t* xi) {
+    unsigned __int128 sum = 0;
+    for (int m = 0; m < M; ++m)
+        for (int k = 0; k < K; ++k) sum += abs_fix16(X[(int64_t)m * ldx + k]);
+    const unsigned __int128 count = (unsigned __int128)M * (unsigned __int128)K;
+    for (int k = 0; k < K; ++k) {
+        uint64_t mx = 0;
+        for (int m = 0; m < M; ++m) {
+            uint64_t a = abs_fix16(X[(int64_t)m * ldx + k]);
+            if (a > mx) mx = a;
+        }
+        if ((unsigned __int128)mx * count > (unsigned __int128)thr * sum) xi[k] += 1;
+    }
+}
+
+/* The nO channels with the largest xi (ties: the lower channel index first), as a sorted index set. */
+void qo_select_outliers(const int32_t* xi, int K, int nO, int32_t* O_idx) {
+    char* taken = (char*)calloc((size_t)(K > 0 ? K : 1), 1);
+    for (int i = 0; i < nO; ++i) {
+        int best = -1;
+        for (int k = 0; k < K; ++k)
+            if (!taken[k] && (best < 0 || xi[k] > xi[best])) best = k; /* strict >: the first (lowest) index wins ties */
+        taken[best] = 1;
+    }
+    int n = 0;
+    for (int k = 0; k < K; ++k)
+        if (taken[k]) O_idx[n++] = k;
+    free(taken);
+}
+

@@ -409,3 +409,63 @@ def test_synthetic_workload_shapes_and_outliers():
     assert np.array_equal(X, X2)
     X3, _ = synth.step_inputs(wl, 0, 1, lin)
     assert not np.array_equal(X, X3)
+
+
+# ----------------------------------------------------------------------------- calibration, Eq. 6
+def _xi_brute(x_f32, thr):
+    """Eq. 6 from its definition in Python integers / Fractions (independent of the C code): |x| in units of 2^-16."""
+    from fractions import Fraction
+    M, K = x_f32.shape
+    a = [[min(int(Fraction(abs(float(v))) * 65536), 2 ** 32 - 1) for v in row] for row in x_f32]
+    total = sum(sum(r) for r in a)
+    return np.array([1 if max(a[m][k] for m in range(M)) * M * K > thr * total else 0 for k in range(K)], np.int32)
+
+
+def test_outlier_count_boundary_is_strict():
+    # one token, channels [1, 1, 1, x], thr = 2: channel 3 counts iff x > 2 (3 + x) / 4  <=>  x > 3
+    for x, hit in ((3.0, 0), (3.015625, 1), (2.984375, 0)):
+        X = synth.f32_to_bf16_bits(np.array([[1.0, 1.0, 1.0, x]], np.float32))
+        xi = oracle.outlier_count(X, 2, np.zeros(4, np.int32))
+        assert xi.tolist() == [0, 0, 0, hit], (x, xi)
+
+
+def test_outlier_count_fixed_point_truncation_and_accumulation():
+    # 2^-17 is below the 2^-16 unit and counts as 0; 2^-10 is 64 units
+    X = synth.f32_to_bf16_bits(np.array([[2.0 ** -17, 2.0 ** -10]], np.float32))
+    xi = oracle.outlier_count(X, 1, np.array([5, 7], np.int32))       # 64 * 2 > 1 * 64 ; 0 * 2 > 64 is false
+    assert xi.tolist() == [5, 8]
+    xi = oracle.outlier_count(X, 2, xi)                                 # 64 * 2 > 2 * 64 is false (strict)
+    assert xi.tolist() == [5, 8]
+
+
+def test_outlier_count_matches_brute_force_and_finds_planted_channels():
+    rng = np.random.default_rng(11)
+    for M, K in ((3, 5), (7, 16), (16, 33)):
+        x = rng.standard_normal((M, K)).astype(np.float32)
+        x[:, rng.integers(K)] *= 300.0
+        xb = synth.f32_to_bf16_bits(x)
+        xf = synth.bf16_bits_to_f32(xb)
+        for thr in (1, 3, 100):
+            assert np.array_equal(oracle.outlier_count(xb, thr, np.zeros(K, np.int32)), _xi_brute(xf, thr))
+    # the paper's threshold (100 x mean|X|) on the synthetic activations: the planted outlier set is what comes out
+    wl = synth.WORKLOADS["tiny"]
+    lin = synth.layer_inputs(wl, 0)
+    xi = np.zeros(lin.spec.K, np.int32)
+    for step in range(8):
+        X, _ = synth.step_inputs(wl, 0, step, lin)
+        xi = oracle.outlier_count(X, 100, xi)
+    # (the threshold is 100 x the mean over ALL channels, outliers included: here about 150, so only the stronger
+    # half of the planted channels - magnitude 30..80 times a 3-sigma peak - can cross it)
+    assert xi[np.setdiff1d(np.arange(lin.spec.K), lin.O_idx)].max() == 0     # an N(0,1) channel never reaches 100 x mean
+    strong = lin.O_idx[lin.base >= 65.0]
+    assert len(strong) > 0 and np.all(xi[strong] >= 6), (lin.base, xi[lin.O_idx])
+    n_found = int((xi > 0).sum())
+    assert set(oracle.select_outliers(xi, n_found).tolist()) <= set(lin.O_idx.tolist())
+
+
+def test_select_outliers_ties_and_order():
+    xi = np.array([2, 5, 5, 0, 5, 1], np.int32)
+    assert oracle.select_outliers(xi, 2).tolist() == [1, 2]        # three channels tie at 5: the lower indices win
+    assert oracle.select_outliers(xi, 4).tolist() == [0, 1, 2, 4]   # sorted ascending
+    assert oracle.select_outliers(xi, 0).tolist() == []
+    assert oracle.select_outliers(xi, 6).tolist() == [0, 1, 2, 3, 4, 5]
