@@ -405,6 +405,11 @@ def run_micro(args):
         dx = torch.empty(M, device="cuda")
         fn = lambda: Q.quaff_quant_act(X, O, s, Xq, xqo, dx)
         nbytes = M * K * 3 + M * nOp + 4 * M
+    elif args.micro == "outlier_count":
+        xi = torch.zeros(K, dtype=torch.int32, device="cuda")
+        ws = torch.empty(Q.workspace_bytes(Q.QUAFF_WS_CALIBRATE, M, K, 0, 0, 0), dtype=torch.uint8, device="cuda")
+        fn = lambda: Q.quaff_outlier_count(X, 100, xi, ws)
+        nbytes = 2 * M * K              # one pass over the sample
     elif args.micro == "momentum":
         wmax = 0.05 + 0.05 * torch.rand(nO, device="cuda", generator=g)
         ws = torch.empty(Q.workspace_bytes(Q.QUAFF_WS_MOMENTUM, M, K, N, nOp, 0), dtype=torch.uint8, device="cuda")
@@ -435,7 +440,7 @@ def run_micro(args):
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--micro", default=None, choices=["quant_act", "momentum", "requant"],
+    ap.add_argument("--micro", default=None, choices=["quant_act", "momentum", "requant", "outlier_count"],
                     help="time one HBM-bound kernel alone instead of the step")
     ap.add_argument("--micro-shape", type=lambda v: tuple(int(x) for x in v.split(",")), default=(8192, 11008, 4096, 55),
                     help="M,K,N,nO of --micro (default: the LLaMA-2-7B down_proj rows)")

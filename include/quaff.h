@@ -51,13 +51,33 @@ enum { /* `which` of quaff_workspace_bytes */
     QUAFF_WS_PREPARE = 0,
     QUAFF_WS_MOMENTUM = 1,
     QUAFF_WS_FWD = 2,
-    QUAFF_WS_BWD = 3
+    QUAFF_WS_BWD = 3,
+    QUAFF_WS_CALIBRATE = 4   /* quaff_outlier_count and quaff_select_outliers (depends on K only) */
 };
 
 const char* quaff_status_string(quaff_status_t s);
 
 /* Bytes of scratch that entry point `which` needs for these sizes (a multiple of 256; may be 0). */
 size_t quaff_workspace_bytes(int which, int M, int K, int N, int nOp, int r);
+
+/*
+ * Calibration before fine-tuning (Sec. 3.3, Eq. 6), one call per calibration sample X^i [M][K]:
+ *   xi[o] += 1   if   max_m |X[m][o]| > thr * mean(|X|)          (the paper uses thr = 100)
+ * The indicator is one exact integer decision: |x| is taken in units of 2^-16, truncated and saturating
+ * at 2^32 - 1, a(x) = min(floor(|x| 2^16), 2^32 - 1), and the test is a(max_o) * (M K) > thr * sum a(X).
+ *   X [M][K] bf16, ldx (ldx % 8 == 0);  thr >= 0;  xi [K] int32 (in/out: the caller zeroes it before the first sample)
+ *   ws: QUAFF_WS_CALIBRATE bytes
+ */
+quaff_status_t quaff_outlier_count(const quaff_bf16* X, int64_t ldx, int M, int K, int thr, int32_t* xi,
+                                   void* ws, size_t ws_bytes, quaff_stream_t stream);
+
+/*
+ * The outlier set O from the counts of Eq. 6 ("selecting outlier channels o based on xi_o"): the nO channels
+ * with the largest xi, ties going to the lower channel index, written as a sorted index set.
+ *   xi [K] int32 (in);  O_idx [nO] int32 (out, ascending);  nO <= K is the layer's budget;  ws: QUAFF_WS_CALIBRATE bytes
+ */
+quaff_status_t quaff_select_outliers(const int32_t* xi, int K, int nO, int32_t* O_idx, void* ws, size_t ws_bytes,
+                                     quaff_stream_t stream);
 
 /*
  * One-time weight preprocessing (Sec. 3.3, "weights preprocessing"; Eq. 1 per output channel).

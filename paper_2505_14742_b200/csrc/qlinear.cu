@@ -432,6 +432,7 @@ extern "C" size_t quaff_workspace_bytes(int which, int M, int K, int N, int nOp,
         case QUAFF_WS_MOMENTUM: return round_up((size_t)(nOp + 1) * 4, 256);
         case QUAFF_WS_FWD: return fwd_workspace(M, K, N, r).total;
         case QUAFF_WS_BWD: return bwd_workspace(M, K, N, nOp, r).total;
+        case QUAFF_WS_CALIBRATE: return round_up((size_t)max(K, 0) * 4, 256) + 256;   // column maxima / flags, sum, ticket
     }
     return 0;
 }
