@@ -64,6 +64,7 @@ class QuaffLinear:
         # the LoRA down-projection runs beside the quantization chain, on its own stream and workspace
         self.ws_lora = torch.empty(max(Q.workspace_bytes(Q.QUAFF_WS_FWD, M, K, N, nOp, r), 256), dtype=torch.uint8, device=dev) if r else None
         self.side = torch.cuda.Stream(device=dev) if r else None
+        self.side2 = torch.cuda.Stream(device=dev) if nO else None
         Q.quaff_prepare_weight(Wt, O_idx, self.Wq, self.dW, self.W_O, self.wmax_O)
 
     def forward(self, X: torch.Tensor) -> torch.Tensor:
@@ -79,8 +80,13 @@ class QuaffLinear:
                 Q.quaff_lora_down(X, self.A, T, self.ws_lora, self.status)
         if self.nO:
             Q.quaff_momentum_update(X, self.O_idx, self.wmax_O, self.gamma, self.s_O, self.ws, self.colmax_O, self.beta_O)
-            Q.quaff_requant_weight_rows(self.W_O, self.s_O, self.wq_O, self.dw_O)
+            # the outlier rows of the weight and the activations both need only s_O: side by side
+            self.side2.wait_stream(main)
+            with torch.cuda.stream(self.side2):
+                Q.quaff_requant_weight_rows(self.W_O, self.s_O, self.wq_O, self.dw_O)
         Q.quaff_quant_act(X, self.O_idx, self.s_O, Xq, xq_O, dx)
+        if self.nO:
+            main.wait_stream(self.side2)
         if self.r:
             main.wait_stream(self.side)
         Q.quaff_qlinear_fwd(Xq, xq_O, dx, self.Wq, self.dW, self.wq_O, self.dw_O, None, None, self.B, self.lora_scale,
