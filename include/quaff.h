@@ -158,7 +158,7 @@ quaff_status_t quaff_lora_down(const quaff_bf16* X, int64_t ldx, int M, int K, c
  *   wq_O [N][nOp], ldwq;  dw_O [N]                            from quaff_requant_weight_rows
  *   X [M][K] bf16, ldx;  A [K][r] bf16;  B [r][N] bf16        LoRA (dense, ld = r and N); r == 0 disables
  *   T_out [M][r] bf16 (out, dense; kept for the backward).  With X = NULL (and r > 0), T_out is an INPUT:
- *   T from an earlier quaff_lora_down on the same X and A; A and ws may then be NULL
+ *   T from an earlier quaff_lora_down on the same X and A; A may then be NULL (ws is still needed)
  *   Y [M][N], ldy, y_dtype QUAFF_BF16 or QUAFF_F32 (out)
  *   dbg_acc_main, dbg_acc_out: optional dense [M][N] int32 dumps of acc1 / acc2 (parity checks)
  *   status_opt: optional int32[4] device word, must be zero on entry; see QUAFF_ERR_TIMEOUT

@@ -4,7 +4,7 @@
 #include <stdlib.h>
 #include <string.h>
 
-#include "umma_gemm.cuh"
+#include "fwd192.cuh"
 
 namespace quaff {
 
@@ -139,6 +139,50 @@ static quaff_status_t launch_gemm(const GemmParams& p, cudaStream_t st) {
     return rc;
 }
 
+static quaff_status_t launch_fwd192(const Fwd192Params& p, cudaStream_t st) {
+    static bool configured[64] = {false};
+    static int units_of[64] = {0};
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (dev < 0 || dev >= 64) return QUAFF_ERR_CUDA;
+    if (!configured[dev]) {
+        if (cudaFuncSetAttribute(fwd192_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kF192SmemBytes) != cudaSuccess)
+            return QUAFF_ERR_CUDA;
+        int units = sm_count() / 2;
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(units * 2);
+        cfg.blockDim = dim3(kGemmThreads);
+        cfg.dynamicSmemBytes = kF192SmemBytes;
+        cudaLaunchAttribute attr;
+        attr.id = cudaLaunchAttributeClusterDimension;
+        attr.val.clusterDim.x = 2; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
+        cfg.attrs = &attr;
+        cfg.numAttrs = 1;
+        int nclusters = 0;
+        if (cudaOccupancyMaxActiveClusters(&nclusters, fwd192_kernel, &cfg) == cudaSuccess && nclusters > 0) units = min(units, nclusters);
+        else cudaGetLastError();
+        units_of[dev] = max(units, 1);
+        configured[dev] = true;
+    }
+    const int ntiles = p.tiles_m * p.tiles_n;
+    if (ntiles == 0) return QUAFF_OK;
+    const int units = min(ntiles, units_of[dev]);
+    const bool timed = g_time_start[0] && g_time_stop[0];
+    unsigned int ev_flags = cudaEventRecordDefault;
+    if (timed) {
+        cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+        if (cudaStreamIsCapturing(st, &cap) == cudaSuccess && cap == cudaStreamCaptureStatusActive) ev_flags = cudaEventRecordExternal;
+        cudaEventRecordWithFlags(g_time_start[0], st, ev_flags);
+    }
+    launch_pdl(fwd192_kernel, dim3(units * 2), dim3(kGemmThreads), kF192SmemBytes, st, 2, p);
+    const quaff_status_t rc = launch_status();
+    if (timed) {
+        cudaEventRecordWithFlags(g_time_stop[0], st, ev_flags);
+        g_time_start[0] = g_time_stop[0] = nullptr;
+    }
+    return rc;
+}
+
 // ------------------------------------------------------------------ small kernels
 // dst[c][j] = src[j][c] for j < rows, 0 for rows <= j < rows_pad   (src is [rows][cols], dst is [cols][rows_pad])
 __global__ void transpose_pad_kernel(const uint16_t* __restrict__ src, int rows, int cols, uint16_t* __restrict__ dst, int rows_pad) {
@@ -257,6 +301,7 @@ __global__ void bwd_fixup_kernel(const float* __restrict__ P, int64_t ldp, int M
 
 static int pad16(int r) { return (r + 15) / 16 * 16; }
 
+constexpr int kFwd192MinK = 4096;   // shortest main contraction for which the 192-column forward wins
 constexpr int kPlanSMs = 148;   // split-K plans (and so workspace sizes) are fixed for the B200's 148 SMs
 
 // Split-K plan of a skinny GEMM with `rows_out` output rows and a contraction of `kc` elements (bf16,
@@ -327,11 +372,12 @@ static quaff_status_t skinny_gemm(int mn_major, const void* A, int64_t lda, cons
     return launch_gemm<EPI_PART, 1, 128>(p, st);
 }
 
-struct FwdWorkspace { size_t off_at, off_part, total; };
+struct FwdWorkspace { size_t off_bt, off_at, off_part, total; };
 static FwdWorkspace fwd_workspace(int M, int K, int N, int r) {
     FwdWorkspace w;
     const int rp = pad16(max(r, 1));
     size_t off = 0;
+    w.off_bt = off;   off += round_up((size_t)max(N, 1) * rp * 2, 256);  // B^T, K-major LoRA-up operand of the 192-column forward
     w.off_at = off;   off += round_up((size_t)rp * K * 2, 256);          // A^T, K-major LoRA-down operand
     w.off_part = off; off += round_up(split_part_bytes(M, K, r), 256);   // split-K partials of T = X A
     w.total = off;
@@ -459,13 +505,46 @@ extern "C" quaff_status_t quaff_qlinear_fwd(int M, int K, int N, const int8_t* X
     QUAFF_RETURN_IF(r > 0 && !have_T && (!aligned16(X) || (ldx % 8)), QUAFF_ERR_ALIGNMENT);
     QUAFF_RETURN_IF(!aligned16(Y), QUAFF_ERR_ALIGNMENT);
     const FwdWorkspace w = fwd_workspace(M, K, N, r);
-    QUAFF_RETURN_IF(r > 0 && !have_T && (!ws || !aligned16(ws) || ws_bytes < w.total), QUAFF_ERR_WORKSPACE_TOO_SMALL);
+    QUAFF_RETURN_IF(r > 0 && (!ws || !aligned16(ws) || ws_bytes < w.total), QUAFF_ERR_WORKSPACE_TOO_SMALL);
     if (M == 0) return QUAFF_OK;
     cudaStream_t st = (cudaStream_t)stream;
     const int rp = pad16(r);
     constexpr int CTAS = 2;
-    // Three accumulators (main, outlier, LoRA) fit TMEM only with 128-column tiles; Eq. 2 alone (no outlier
-    // set, no LoRA) takes the 256-column tile.
+    // Eq. 2 alone (no outlier set, no LoRA) takes 256-column tiles.  With the two short contractions: 192-column
+    // tiles with the short accumulators in rounds of 64 columns (fwd192.cuh) where the main contraction is long
+    // enough to pay for the rounds (measured: K >= 4096; a tcgen05.mma costs about 60 + N/2 clocks, so wider is
+    // cheaper per column, but each tile carries six extra ring stages and three more epilogue hand-shakes) and an
+    // outlier round is one k-block (nOp <= 128); otherwise 128-column tiles with all three accumulators in TMEM.
+    if ((nOp > 0 || r > 0) && nOp <= 128 && K >= kFwd192MinK) {
+        Fwd192Params q;
+        memset(&q, 0, sizeof(q));
+        quaff_status_t rc;
+        if ((rc = make_tmap_2d(&q.map_xq, Xq, 1, M, K, ldxq, kTileM, 128)) != QUAFF_OK) return rc;
+        if ((rc = make_tmap_2d(&q.map_wq, Wq, 1, N, K, ldwq_main, kF192TN / 2, 128)) != QUAFF_OK) return rc;
+        q.nblk = ceil_div(K, 128);
+        q.nmma_last = ceil_div(K - (q.nblk - 1) * 128, 32);
+        if (nOp > 0) {
+            if ((rc = make_tmap_2d(&q.map_xo, xq_O, 1, M, nOp, ldxo, kTileM, 128)) != QUAFF_OK) return rc;
+            if ((rc = make_tmap_2d(&q.map_wo, wq_O, 1, N, nOp, ldwq, kF192Round / 2, 128)) != QUAFF_OK) return rc;
+            q.nmma_o = nOp / 32;
+        }
+        if (r > 0) {
+            if (!have_T && (rc = lora_down(X, ldx, M, K, A, r, T_out, w, ws, status_opt, st)) != QUAFF_OK) return rc;
+            uint16_t* Bt = reinterpret_cast<uint16_t*>(reinterpret_cast<unsigned char*>(ws) + w.off_bt);
+            launch_pdl(transpose_pad_kernel, dim3(ceil_div(N * rp, 256)), dim3(256), 0, st, 1, B, r, N, Bt, rp);   // Bt[n][j] = B[j][n]
+            if ((rc = launch_status()) != QUAFF_OK) return rc;
+            if ((rc = make_tmap_2d(&q.map_t, T_out, 2, M, r, r, kTileM, 64)) != QUAFF_OK) return rc;
+            if ((rc = make_tmap_2d(&q.map_bt, Bt, 2, N, rp, rp, kF192Round / 2, 64)) != QUAFF_OK) return rc;
+            q.nmma_l = rp / 16;
+        }
+        q.M = M; q.N = N;
+        q.tiles_m = ceil_div(M, 2 * kTileM); q.tiles_n = ceil_div(N, kF192TN);
+        q.status = status_opt;
+        q.dx = dx; q.dW = dW; q.dw_O = dw_O; q.lora_scale = lora_scale;
+        q.Y = Y; q.ldy = ldy; q.y_f32 = (y_dtype == QUAFF_F32);
+        q.dbg_main = dbg_acc_main; q.dbg_out = dbg_acc_out;
+        return launch_fwd192(q, st);
+    }
     const int TN = (nOp == 0 && r == 0) ? 256 : 128;
 
     GemmParams p;

@@ -32,9 +32,11 @@
 // TMEM (512 columns): slot 0 is double-buffered at columns [0,TN) and [TN,2TN) so the main
 // contraction of tile t+1 overlaps the epilogue of tile t; with TN = 128, slots 1 and 2 live at
 // [256,384) and [384,512) and are written only after the epilogue of the previous tile has drained them.
-// A 256-wide tcgen05.mma runs at nearly twice the rate of a 128-wide one (a 128-wide one is bound by
-// fetching its A operand from shared memory), but two 256-column buffers fill TMEM: TN = 256 is for
-// contractions with a single accumulator (grad-input; forward without outliers and LoRA).
+// Measured on B200, a tcgen05.mma of a CTA pair (M = 256, 32 bytes of contraction) costs about 60 + N/2
+// clocks (N = 128: 125, 192: 165, 256: 190): the wider the tile, the cheaper the column.  Two 256-column
+// buffers fill TMEM, so TN = 256 is for contractions with a single accumulator (grad-input; forward
+// without outliers and LoRA); the forward with its three accumulators runs TN = 128 here or the
+// 192-column kernel of fwd192.cuh.
 //
 // The producer and the MMA issuer are single threads; their per-k-block instruction count bounds the
 // tensor-pipe utilisation, so everything that does not change inside a phase is hoisted out of the
