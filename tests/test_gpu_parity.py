@@ -145,7 +145,8 @@ FWD_SHAPES = [(1, 128, 16, 0, 0), (128, 128, 128, 32, 16), (200, 320, 136, 5, 8)
               (300, 1024, 392, 150, 16), (513, 640, 520, 128, 8),   # nOp > 128 or K < 4096: 128-column tiles, all accumulators in TMEM
               # K >= 4096: 192-column tiles with the short accumulators in rounds (ragged N, LoRA only, outliers only, r = 8)
               (130, 4096, 296, 33, 64), (257, 4224, 136, 0, 32), (100, 4096, 200, 3, 0), (300, 8192, 1032, 100, 16),
-              (520, 4096, 392, 40, 8), (1, 4096, 64, 5, 16)]
+              (520, 4096, 392, 40, 8), (1, 4096, 64, 5, 16),
+              (200, 11008, 520, 1100, 16)]   # the paper's 10 % budget of down_proj: nO = 1100 outlier channels
 
 
 @pytest.mark.parametrize("M,K,N,nO,r", FWD_SHAPES)
@@ -181,7 +182,8 @@ def test_qlinear_fwd(Q, M, K, N, nO, r, y_f32):
 # ----------------------------------------------------------------------------- S6-S8 backward
 BWD_SHAPES = [(1, 128, 64, 0, 0), (128, 128, 128, 32, 16), (200, 320, 136, 5, 8), (256, 512, 512, 8, 8),
               (384, 640, 1024, 40, 16), (130, 300 // 4 * 4 + 4, 2048, 33, 64), (100, 256, 256, 3, 0),
-              (520, 1032, 3072, 32, 16), (300, 2056, 520, 70, 32)]
+              (520, 1032, 3072, 32, 16), (300, 2056, 520, 70, 32),
+              (200, 11008, 520, 1100, 16)]   # 10 % outlier budget: 2 x 1120 columns of outlier partial products
 
 
 @pytest.mark.parametrize("M,K,N,nO,r", BWD_SHAPES)
