@@ -410,6 +410,14 @@ def run_micro(args):
         ws = torch.empty(Q.workspace_bytes(Q.QUAFF_WS_CALIBRATE, M, K, 0, 0, 0), dtype=torch.uint8, device="cuda")
         fn = lambda: Q.quaff_outlier_count(X, 100, xi, ws)
         nbytes = 2 * M * K              # one pass over the sample
+    elif args.micro == "lora_down":
+        r = 64
+        A = (0.02 * torch.randn((K, r), device="cuda", generator=g)).to(torch.bfloat16)
+        T = torch.empty((M, r), dtype=torch.bfloat16, device="cuda")
+        st = torch.zeros(4, dtype=torch.int32, device="cuda")
+        ws = torch.empty(Q.workspace_bytes(Q.QUAFF_WS_FWD, M, K, N, nOp, r), dtype=torch.uint8, device="cuda")
+        fn = lambda: Q.quaff_lora_down(X, A, T, ws, st)
+        nbytes = 2 * M * K + 2 * K * r + 2 * M * r
     elif args.micro == "momentum":
         wmax = 0.05 + 0.05 * torch.rand(nO, device="cuda", generator=g)
         ws = torch.empty(Q.workspace_bytes(Q.QUAFF_WS_MOMENTUM, M, K, N, nOp, 0), dtype=torch.uint8, device="cuda")
@@ -440,7 +448,7 @@ def run_micro(args):
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--micro", default=None, choices=["quant_act", "momentum", "requant", "outlier_count"],
+    ap.add_argument("--micro", default=None, choices=["quant_act", "momentum", "requant", "outlier_count", "lora_down"],
                     help="time one HBM-bound kernel alone instead of the step")
     ap.add_argument("--micro-shape", type=lambda v: tuple(int(x) for x in v.split(",")), default=(8192, 11008, 4096, 55),
                     help="M,K,N,nO of --micro (default: the LLaMA-2-7B down_proj rows)")

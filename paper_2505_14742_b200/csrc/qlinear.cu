@@ -305,12 +305,13 @@ constexpr int kFwd192MinK = 4096;   // shortest main contraction for which the 1
 constexpr int kPlanSMs = 148;   // split-K plans (and so workspace sizes) are fixed for the B200's 148 SMs
 
 // Split-K plan of a skinny GEMM with `rows_out` output rows and a contraction of `kc` elements (bf16,
-// 64 per k-block): enough splits to give every SM a tile, at least two k-blocks per split.
+// 64 per k-block): as many splits as still run in ONE wave (a second, partial wave of split tiles costs more
+// than shorter splits save), at least two k-blocks per split.
 struct SplitPlan { int S, kblk; };
 static SplitPlan split_plan(int rows_out, int kc) {
     const int tiles = ceil_div(rows_out, kTileM);
     const int nblk = max(1, ceil_div(kc, 64));
-    int S = max(1, min(ceil_div(kPlanSMs, tiles), ceil_div(nblk, 2)));
+    int S = max(1, min(max(1, kPlanSMs / tiles), ceil_div(nblk, 2)));
     SplitPlan p;
     p.kblk = ceil_div(nblk, S);
     p.S = ceil_div(nblk, p.kblk);
