@@ -194,31 +194,55 @@ __global__ void transpose_pad_kernel(const uint16_t* __restrict__ src, int rows,
     dst[idx] = j < rows ? src[(int64_t)j * cols + c] : (uint16_t)0;
 }
 
-// out[m][j] = bf16(scale * sum_s part[s][m][j])
+// out[m][j] = bf16(scale * sum_s part[s][m][j]);  a thread sums 8 consecutive j (r is a multiple of 8)
 __global__ void reduce_parts_bf16_kernel(const float* __restrict__ part, int S, int rows, int r, float scale,
                                          uint16_t* __restrict__ out) {
     pdl_launch_dependents();
     pdl_wait();
-    const int idx = blockIdx.x * blockDim.x + threadIdx.x;
-    if (idx >= rows * r) return;
-    float sum = 0.0f;
-    for (int s = 0; s < S; ++s) sum += part[(int64_t)s * rows * r + idx];
-    out[idx] = (uint16_t)f32_to_bf16_bits(scale * sum);
+    const int64_t idx = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) * 8;
+    const int64_t total = (int64_t)rows * r;
+    if (idx >= total) return;
+    float acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+    for (int s = 0; s < S; ++s) {
+        const float4* src = reinterpret_cast<const float4*>(part + s * total + idx);
+        const float4 a = __ldg(src), b = __ldg(src + 1);
+        acc[0] += a.x; acc[1] += a.y; acc[2] += a.z; acc[3] += a.w;
+        acc[4] += b.x; acc[5] += b.y; acc[6] += b.z; acc[7] += b.w;
+    }
+    *reinterpret_cast<uint4*>(out + idx) = make_uint4(pack_bf16x2(scale * acc[0], scale * acc[1]), pack_bf16x2(scale * acc[2], scale * acc[3]),
+                                                      pack_bf16x2(scale * acc[4], scale * acc[5]), pack_bf16x2(scale * acc[6], scale * acc[7]));
 }
 
-// dst = (accumulate ? dst : 0) + scale * sum_s part[s][c][j];  dst index c*r + j, or j*C + c when transposed
+// dst = (accumulate ? dst : 0) + scale * sum_s part[s][c][j];  dst index c*r + j, or j*C + c when transposed.
+// A thread sums 4 consecutive j of one c (r is a multiple of 8); consecutive threads take consecutive c when the
+// output is transposed (coalesced stores along c) and consecutive j-quads otherwise.
 __global__ void reduce_parts_kernel(const float* __restrict__ part, int S, int C, int r, float scale, int transposed,
                                     int accumulate, float* __restrict__ dst) {
     pdl_launch_dependents();
     pdl_wait();
     const int idx = blockIdx.x * blockDim.x + threadIdx.x;
-    if (idx >= C * r) return;
-    int c, j;
-    if (transposed) { j = idx / C; c = idx % C; } else { c = idx / r; j = idx % r; }
-    float sum = 0.0f;
-    for (int s = 0; s < S; ++s) sum += part[((int64_t)s * C + c) * r + j];
-    sum *= scale;
-    dst[idx] = accumulate ? dst[idx] + sum : sum;
+    const int rq = r >> 2;
+    if (idx >= C * rq) return;
+    int c, jq;
+    if (transposed) { jq = idx / C; c = idx % C; } else { c = idx / rq; jq = idx % rq; }
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int s = 0; s < S; ++s) {
+        const float4 a = __ldg(reinterpret_cast<const float4*>(part + ((int64_t)s * C + c) * r + 4 * jq));
+        acc.x += a.x; acc.y += a.y; acc.z += a.z; acc.w += a.w;
+    }
+    const float v[4] = {acc.x * scale, acc.y * scale, acc.z * scale, acc.w * scale};
+    if (!transposed) {
+        float4* d = reinterpret_cast<float4*>(dst + (int64_t)c * r + 4 * jq);
+        float4 o = make_float4(v[0], v[1], v[2], v[3]);
+        if (accumulate) { const float4 old = *d; o.x += old.x; o.y += old.y; o.z += old.z; o.w += old.w; }
+        *d = o;
+    } else {
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            float* d = dst + (int64_t)(4 * jq + e) * C + c;
+            *d = accumulate ? *d + v[e] : v[e];
+        }
+    }
 }
 
 // Dequantized weight for the grad-input GEMM, in the stored orientation [N][.] (the contraction index n
@@ -432,7 +456,7 @@ static quaff_status_t lora_down(const quaff_bf16* X, int64_t ldx, int M, int K, 
     if ((rc = launch_status()) != QUAFF_OK) return rc;
     int S = 1;
     if ((rc = skinny_gemm(0, X, ldx, At, K, M, K, r, part, status_opt, st, &S)) != QUAFF_OK) return rc;
-    launch_pdl(reduce_parts_bf16_kernel, dim3(ceil_div(M * r, 256)), dim3(256), 0, st, 1, part, S, M, r, 1.0f, T_out);
+    launch_pdl(reduce_parts_bf16_kernel, dim3(ceil_div(M * r / 8, 256)), dim3(256), 0, st, 1, part, S, M, r, 1.0f, T_out);
     return launch_status();
 }
 
@@ -605,7 +629,7 @@ extern "C" quaff_status_t quaff_qlinear_bwd(int M, int K, int N, const quaff_bf1
     QUAFF_RETURN_IF(nOp > 0 && (!aligned16(wq_O) || (ldwq % 16)), QUAFF_ERR_ALIGNMENT);
     QUAFF_RETURN_IF(dX && (!aligned16(dX) || (lddx % 8)), QUAFF_ERR_ALIGNMENT);
     QUAFF_RETURN_IF(r > 0 && (!aligned16(A) || !aligned16(B)), QUAFF_ERR_ALIGNMENT);
-    QUAFF_RETURN_IF(r > 0 && dA && (!aligned16(X) || !aligned16(T) || (ldx % 8)), QUAFF_ERR_ALIGNMENT);
+    QUAFF_RETURN_IF(r > 0 && dA && (!aligned16(X) || !aligned16(T) || !aligned16(dA) || !aligned16(dB) || (ldx % 8)), QUAFF_ERR_ALIGNMENT);
     const BwdWorkspace w = bwd_workspace(M, K, N, nOp, r);
     QUAFF_RETURN_IF(!ws || !aligned16(ws) || ws_bytes < w.total, QUAFF_ERR_WORKSPACE_TOO_SMALL);
     if (M == 0) return QUAFF_OK;
@@ -630,7 +654,7 @@ extern "C" quaff_status_t quaff_qlinear_bwd(int M, int K, int N, const quaff_bf1
     if (want_dAB) {   // dB^T = dY^T T: the contraction runs over the tokens, the slow axis of dY and T: MN-major operands
         if (ss && !(forked1 = fork_to(ss, 1, st))) return QUAFF_ERR_CUDA;
         if ((rc = skinny_gemm(1, dY, lddy, T, r, N, M, r, part_b, status_opt, s_db, &S)) != QUAFF_OK) return rc;
-        launch_pdl(reduce_parts_kernel, dim3(ceil_div(N * r, 256)), dim3(256), 0, s_db, 1, part_b, S, N, r, lora_scale, 1, accumulate, dB);
+        launch_pdl(reduce_parts_kernel, dim3(ceil_div(N * r / 4, 256)), dim3(256), 0, s_db, 1, part_b, S, N, r, lora_scale, 1, accumulate, dB);
         if ((rc = launch_status()) != QUAFF_OK) return rc;
     }
     constexpr int CTAS = 2;
@@ -645,7 +669,7 @@ extern "C" quaff_status_t quaff_qlinear_bwd(int M, int K, int N, const quaff_bf1
     }
     if (r > 0) {   // G = bf16(lora_scale * dY B^T): B [r][N] is already K-major for this contraction over N
         if ((rc = skinny_gemm(0, dY, lddy, B, N, M, N, r, part, status_opt, st, &S)) != QUAFF_OK) return rc;
-        launch_pdl(reduce_parts_bf16_kernel, dim3(ceil_div(M * r, 256)), dim3(256), 0, st, 1, part, S, M, r, lora_scale, G);
+        launch_pdl(reduce_parts_bf16_kernel, dim3(ceil_div(M * r / 8, 256)), dim3(256), 0, st, 1, part, S, M, r, lora_scale, G);
         if ((rc = launch_status()) != QUAFF_OK) return rc;
     }
     if (dX) {
@@ -689,7 +713,7 @@ extern "C" quaff_status_t quaff_qlinear_bwd(int M, int K, int N, const quaff_bf1
             s_da = ss->s[0];
         }
         if ((rc = skinny_gemm(1, X, ldx, G, r, K, M, r, part_a, status_opt, s_da, &S)) != QUAFF_OK) return rc;
-        launch_pdl(reduce_parts_kernel, dim3(ceil_div(K * r, 256)), dim3(256), 0, s_da, 1, part_a, S, K, r, 1.0f, 0, accumulate, dA);
+        launch_pdl(reduce_parts_kernel, dim3(ceil_div(K * r / 4, 256)), dim3(256), 0, s_da, 1, part_a, S, K, r, 1.0f, 0, accumulate, dA);
         if ((rc = launch_status()) != QUAFF_OK) return rc;
         forked0 = forked_da;
     } else {
