@@ -18,7 +18,8 @@
 // pipe is a third of the way further into the main contraction of tile t+1.  Barriers beside the ring:
 //   tmem_full / tmem_empty : main accumulator of a tile complete / drained (as in umma_gemm.cuh)
 //   aux_ready / aux_free   : the two short accumulators of a round complete / drained
-// Roles, CTA-pair protocol, bounded waits and the exit path are those of umma_gemm.cuh.
+// Roles, CTA-pair protocol, bounded waits and the exit path are those of umma_gemm.cuh, with EIGHT epilogue
+// warps (two per TMEM lane quarter) so that a round is drained well within a third of a main contraction.
 #pragma once
 
 #include "umma_gemm.cuh"
@@ -27,6 +28,7 @@ namespace quaff {
 
 constexpr int kF192TN = 192;
 constexpr int kF192Round = 64;                               // output columns per round
+constexpr int kF192Threads = 64 + 8 * 32;                    // producer warp, MMA warp, eight epilogue warps
 constexpr int kF192StageBytes = kABytes + (kF192TN / 2) * 128;   // A: 128 rows, B: this CTA's 96 rows (a round uses 32 of them)
 constexpr int kF192ScaleBytes = 2 * 2 * kF192TN * 4;
 
@@ -83,7 +85,7 @@ __device__ __forceinline__ void for_each_item(int unit, int nunits, int ntiles, 
     }
 }
 
-__global__ void __launch_bounds__(kGemmThreads, 1) fwd192_kernel(const __grid_constant__ Fwd192Params p) {
+__global__ void __launch_bounds__(kF192Threads, 1) fwd192_kernel(const __grid_constant__ Fwd192Params p) {
     constexpr int TN = kF192TN;
     constexpr int kStages = kF192Stages;
     constexpr int kStageBytes = kF192StageBytes;
@@ -115,9 +117,9 @@ __global__ void __launch_bounds__(kGemmThreads, 1) fwd192_kernel(const __grid_co
             mbar_init(empty0 + 8u * s, 1);
         }
         mbar_init(tmem_full_bar, 1);
-        mbar_init(tmem_empty_bar, 4 * 2);
+        mbar_init(tmem_empty_bar, 8 * 2);       // eight epilogue warps in each CTA of the pair
         mbar_init(aux_ready_bar, 1);
-        mbar_init(aux_free_bar, 4 * 2);
+        mbar_init(aux_free_bar, 8 * 2);
         sm->abort_flag = 0;
         fence_barrier_init();
     }
@@ -218,10 +220,13 @@ __global__ void __launch_bounds__(kGemmThreads, 1) fwd192_kernel(const __grid_co
                 });
         }
     } else {
-        // ------------------------------------------------------------------ epilogue (128 threads per CTA)
+        // ------------------------------------------------------------------ epilogue (8 warps = 256 threads per CTA)
+        // Warps w and w + 4 share a TMEM lane quarter; of the 64 columns of a round, the first four warps take
+        // columns [0,32) and the other four [32,64): a round is drained by all eight warps at once.
         const int q = warp & 3;
+        const int g = (warp - 2) >> 2;           // which half of a round's columns
         const int row = q * 32 + lane;
-        const int et = threadIdx.x - 64;
+        const int et = threadIdx.x - 64;         // 0..255
         const bool has_o = p.nmma_o != 0, has_l = p.nmma_l != 0;
         bool ok = true;
         int t = 0, rounds = 0;
@@ -231,75 +236,76 @@ __global__ void __launch_bounds__(kGemmThreads, 1) fwd192_kernel(const __grid_co
             const int buf = t & 1;
             float* scale_w = scales + buf * 2 * TN;
             float* scale_o = scale_w + TN;
-            for (int c = et; c < TN; c += 128) {
-                const int n = n0 + c;
-                scale_w[c] = n < p.N ? p.dW[n] : 0.0f;
-                scale_o[c] = (n < p.N && has_o) ? p.dw_O[n] : 0.0f;
+            if (et < TN) {
+                const int n = n0 + et;
+                scale_w[et] = n < p.N ? p.dW[n] : 0.0f;
+                scale_o[et] = (n < p.N && has_o) ? p.dw_O[n] : 0.0f;
             }
-            named_bar_sync(1, 128);
-            if (!mbar_wait(tmem_full_bar, (uint32_t)(t & 1), abort_flag)) { ok = false; break; }
             const int m = m0 + row;
             const float dxm = m < p.M ? __ldg(p.dx + m) : 0.0f;
+            named_bar_sync(1, kF192Threads - 64);
+            if (!mbar_wait(tmem_full_bar, (uint32_t)(t & 1), abort_flag)) { ok = false; break; }
             const uint32_t lane_addr = tmem_base + ((uint32_t)(q * 32) << 16);
 #pragma unroll 1
-            for (int c = 0; c < TN / 32; ++c) {
-                if ((c & 1) == 0) {           // a new round: its two short accumulators
-                    if (!mbar_wait(aux_ready_bar, (uint32_t)(rounds & 1), abort_flag)) { ok = false; break; }
-                }
+            for (int j = 0; j < TN / kF192Round; ++j, ++rounds) {
+                if (!mbar_wait(aux_ready_bar, (uint32_t)(rounds & 1), abort_flag)) { ok = false; break; }
                 tc_fence_after();
-                const int nc = n0 + c * 32;
-                uint32_t r0[32], r1[32], r2[32];
-                tmem_ld_32x32(lane_addr + (uint32_t)(buf * TN + c * 32), r0);
-                if (has_o) tmem_ld_32x32(lane_addr + kColAuxO + (uint32_t)((c & 1) * 32), r1);
-                if (has_l) tmem_ld_32x32(lane_addr + kColAuxL + (uint32_t)((c & 1) * 32), r2);
-                tmem_ld_wait();
-                if (m < p.M && nc < p.N) {
-                    float y[32];
+                const int cl = j * kF192Round + g * 32;      // first of this warp's 32 columns inside the tile
 #pragma unroll
-                    for (int j = 0; j < 32; ++j) {
-                        float w = (float)(int)r0[j] * scale_w[c * 32 + j];
-                        if (has_o) w += (float)(int)r1[j] * scale_o[c * 32 + j];
-                        float v = dxm * w;
-                        if (has_l) v += p.lora_scale * __uint_as_float(r2[j]);
-                        y[j] = v;
-                    }
-                    const bool full = (nc + 32 <= p.N);
-                    if (p.y_f32) {
-                        float* out = reinterpret_cast<float*>(p.Y) + (int64_t)m * p.ldy + nc;
-                        if (full && (p.ldy % 4 == 0)) {
+                for (int h = 0; h < 2; ++h) {                // 16 columns at a time (register budget)
+                    const int c0 = cl + 16 * h;
+                    const int nc = n0 + c0;
+                    uint32_t r0[16], r1[16], r2[16];
+                    tmem_ld_32x16(lane_addr + (uint32_t)(buf * TN + c0), r0);
+                    if (has_o) tmem_ld_32x16(lane_addr + kColAuxO + (uint32_t)(g * 32 + 16 * h), r1);
+                    if (has_l) tmem_ld_32x16(lane_addr + kColAuxL + (uint32_t)(g * 32 + 16 * h), r2);
+                    tmem_ld_wait();
+                    if (m < p.M && nc < p.N) {
+                        float y[16];
 #pragma unroll
-                            for (int j = 0; j < 32; j += 4) *reinterpret_cast<float4*>(out + j) = make_float4(y[j], y[j + 1], y[j + 2], y[j + 3]);
-                        } else {
-                            for (int j = 0; j < 32; ++j) if (nc + j < p.N) out[j] = y[j];
+                        for (int i = 0; i < 16; ++i) {
+                            float w = (float)(int)r0[i] * scale_w[c0 + i];
+                            if (has_o) w += (float)(int)r1[i] * scale_o[c0 + i];
+                            float v = dxm * w;
+                            if (has_l) v += p.lora_scale * __uint_as_float(r2[i]);
+                            y[i] = v;
                         }
-                    } else {
-                        uint16_t* out = reinterpret_cast<uint16_t*>(p.Y) + (int64_t)m * p.ldy + nc;
-                        if (full && (p.ldy % 8 == 0)) {
+                        const bool full = (nc + 16 <= p.N);
+                        if (p.y_f32) {
+                            float* out = reinterpret_cast<float*>(p.Y) + (int64_t)m * p.ldy + nc;
+                            if (full && (p.ldy % 4 == 0)) {
 #pragma unroll
-                            for (int j = 0; j < 32; j += 8)
-                                *reinterpret_cast<uint4*>(out + j) = make_uint4(pack_bf16x2(y[j], y[j + 1]), pack_bf16x2(y[j + 2], y[j + 3]),
-                                                                                pack_bf16x2(y[j + 4], y[j + 5]), pack_bf16x2(y[j + 6], y[j + 7]));
+                                for (int i = 0; i < 16; i += 4) *reinterpret_cast<float4*>(out + i) = make_float4(y[i], y[i + 1], y[i + 2], y[i + 3]);
+                            } else {
+                                for (int i = 0; i < 16; ++i) if (nc + i < p.N) out[i] = y[i];
+                            }
                         } else {
-                            for (int j = 0; j < 32; ++j) if (nc + j < p.N) out[j] = (uint16_t)f32_to_bf16_bits(y[j]);
+                            uint16_t* out = reinterpret_cast<uint16_t*>(p.Y) + (int64_t)m * p.ldy + nc;
+                            if (full && (p.ldy % 8 == 0)) {
+#pragma unroll
+                                for (int i = 0; i < 16; i += 8)
+                                    *reinterpret_cast<uint4*>(out + i) = make_uint4(pack_bf16x2(y[i], y[i + 1]), pack_bf16x2(y[i + 2], y[i + 3]),
+                                                                                    pack_bf16x2(y[i + 4], y[i + 5]), pack_bf16x2(y[i + 6], y[i + 7]));
+                            } else {
+                                for (int i = 0; i < 16; ++i) if (nc + i < p.N) out[i] = (uint16_t)f32_to_bf16_bits(y[i]);
+                            }
                         }
-                    }
-                    if (p.dbg_main) {
-                        int32_t* d = p.dbg_main + (int64_t)m * p.N + nc;
-                        for (int j = 0; j < 32; ++j) if (nc + j < p.N) d[j] = (int32_t)r0[j];
-                    }
-                    if (p.dbg_out) {
-                        int32_t* d = p.dbg_out + (int64_t)m * p.N + nc;
-                        for (int j = 0; j < 32; ++j) if (nc + j < p.N) d[j] = has_o ? (int32_t)r1[j] : 0;
+                        if (p.dbg_main) {
+                            int32_t* d = p.dbg_main + (int64_t)m * p.N + nc;
+                            for (int i = 0; i < 16; ++i) if (nc + i < p.N) d[i] = (int32_t)r0[i];
+                        }
+                        if (p.dbg_out) {
+                            int32_t* d = p.dbg_out + (int64_t)m * p.N + nc;
+                            for (int i = 0; i < 16; ++i) if (nc + i < p.N) d[i] = has_o ? (int32_t)r1[i] : 0;
+                        }
                     }
                 }
-                if (c & 1) {                  // the round is drained (also when its columns lie past N)
-                    tc_fence_before();
-                    __syncwarp();
-                    if (lane == 0) {
-                        if (rank != 0) mbar_arrive_cluster(lead_aux_free);
-                        else mbar_arrive(aux_free_bar);
-                    }
-                    ++rounds;
+                // this warp's share of the round is drained (also when its columns lie past N)
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) {
+                    if (rank != 0) mbar_arrive_cluster(lead_aux_free);
+                    else mbar_arrive(aux_free_bar);
                 }
             }
             if (!ok) break;

@@ -151,7 +151,7 @@ static quaff_status_t launch_fwd192(const Fwd192Params& p, cudaStream_t st) {
         int units = sm_count() / 2;
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3(units * 2);
-        cfg.blockDim = dim3(kGemmThreads);
+        cfg.blockDim = dim3(kF192Threads);
         cfg.dynamicSmemBytes = kF192SmemBytes;
         cudaLaunchAttribute attr;
         attr.id = cudaLaunchAttributeClusterDimension;
@@ -174,7 +174,7 @@ static quaff_status_t launch_fwd192(const Fwd192Params& p, cudaStream_t st) {
         if (cudaStreamIsCapturing(st, &cap) == cudaSuccess && cap == cudaStreamCaptureStatusActive) ev_flags = cudaEventRecordExternal;
         cudaEventRecordWithFlags(g_time_start[0], st, ev_flags);
     }
-    launch_pdl(fwd192_kernel, dim3(units * 2), dim3(kGemmThreads), kF192SmemBytes, st, 2, p);
+    launch_pdl(fwd192_kernel, dim3(units * 2), dim3(kF192Threads), kF192SmemBytes, st, 2, p);
     const quaff_status_t rc = launch_status();
     if (timed) {
         cudaEventRecordWithFlags(g_time_stop[0], st, ev_flags);
@@ -325,7 +325,6 @@ __global__ void bwd_fixup_kernel(const float* __restrict__ P, int64_t ldp, int M
 
 static int pad16(int r) { return (r + 15) / 16 * 16; }
 
-constexpr int kFwd192MinK = 4096;   // shortest main contraction for which the 192-column forward wins
 constexpr int kPlanSMs = 148;   // split-K plans (and so workspace sizes) are fixed for the B200's 148 SMs
 
 // Split-K plan of a skinny GEMM with `rows_out` output rows and a contraction of `kc` elements (bf16,
@@ -536,11 +535,15 @@ extern "C" quaff_status_t quaff_qlinear_fwd(int M, int K, int N, const int8_t* X
     const int rp = pad16(r);
     constexpr int CTAS = 2;
     // Eq. 2 alone (no outlier set, no LoRA) takes 256-column tiles.  With the two short contractions: 192-column
-    // tiles with the short accumulators in rounds of 64 columns (fwd192.cuh) where the main contraction is long
-    // enough to pay for the rounds (measured: K >= 4096; a tcgen05.mma costs about 60 + N/2 clocks, so wider is
-    // cheaper per column, but each tile carries six extra ring stages and three more epilogue hand-shakes) and an
-    // outlier round is one k-block (nOp <= 128); otherwise 128-column tiles with all three accumulators in TMEM.
-    if ((nOp > 0 || r > 0) && nOp <= 128 && K >= kFwd192MinK) {
+    // tiles with the short accumulators in rounds of 64 columns (fwd192.cuh), or 128-column tiles with all three
+    // accumulators resident in TMEM.  A tcgen05.mma costs about 60 + N/2 clocks, so the wide tile is cheaper per
+    // column, but it carries six extra ring stages and three more epilogue hand-shakes: measured, a wave of
+    // 192-column tiles takes 1.47x (K < 4096) resp. 1.27x (K >= 4096) as long as a wave of 128-column tiles.  The
+    // rounds need an outlier round to be one k-block (nOp <= 128).
+    const int tiles_m2 = ceil_div(M, 2 * kTileM), pairs = kPlanSMs / 2;
+    const double waves128 = ceil_div(tiles_m2 * ceil_div(N, 128), pairs);
+    const double waves192 = ceil_div(tiles_m2 * ceil_div(N, kF192TN), pairs) * (K >= 4096 ? 1.27 : 1.47);
+    if ((nOp > 0 || r > 0) && nOp <= 128 && waves192 < waves128) {
         Fwd192Params q;
         memset(&q, 0, sizeof(q));
         quaff_status_t rc;

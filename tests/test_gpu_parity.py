@@ -143,9 +143,11 @@ FWD_SHAPES = [(1, 128, 16, 0, 0), (128, 128, 128, 32, 16), (200, 320, 136, 5, 8)
               (384, 1024, 640, 40, 16), (130, 2048, 296, 33, 64), (257, 384, 136, 0, 32), (100, 256, 256, 3, 0),
               (77, 256, 129, 7, 0), (520, 3072, 1032, 32, 16),
               (300, 1024, 392, 150, 16), (513, 640, 520, 128, 8),   # nOp > 128 or K < 4096: 128-column tiles, all accumulators in TMEM
-              # K >= 4096: 192-column tiles with the short accumulators in rounds (ragged N, LoRA only, outliers only, r = 8)
-              (130, 4096, 296, 33, 64), (257, 4224, 136, 0, 32), (100, 4096, 200, 3, 0), (300, 8192, 1032, 100, 16),
-              (520, 4096, 392, 40, 8), (1, 4096, 64, 5, 16),
+              (130, 4096, 296, 33, 64), (300, 8192, 1032, 100, 16), (1, 4096, 64, 5, 16),
+              # 192 to 222 tiles of 256 x 128 are three waves on the 74 CTA pairs, the same area in 256 x 192 tiles two:
+              # these take the 192-column forward with the short accumulators in rounds (ragged M and N, LoRA only,
+              # outliers only, r = 8, a single main k-block)
+              (2048, 256, 3072, 33, 64), (2040, 384, 3016, 0, 32), (2048, 256, 3061, 7, 0), (2048, 128, 3072, 40, 8),
               (200, 11008, 520, 1100, 16)]   # the paper's 10 % budget of down_proj: nO = 1100 outlier channels
 
 
