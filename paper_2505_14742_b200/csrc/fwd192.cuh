@@ -52,6 +52,7 @@ struct Fwd192Params {
     int nblk, nmma_last;             // main k-blocks per tile; MMAs of the last one (1..4)
     int nmma_o, nmma_l;              // MMAs of an outlier round (nOp / 32, 0 = no outliers) / of a LoRA round (rp / 16, 0 = no LoRA)
     int M, N, tiles_m, tiles_n;
+    int band_m;                      // row tiles per band of the tile order (see tile_coords)
     int32_t* status;
     const float* dx;
     const float* dW;
@@ -154,13 +155,15 @@ __global__ void __launch_bounds__(kF192Threads, 1) fwd192_kernel(const __grid_co
                 return true;
             };
             const uint32_t tx_main = kABytes + (TN / 2) * 128, tx_aux = kABytes + (kF192Round / 2) * 128;
+            int tm = 0, tn = 0;
             for_each_item(unit, nunits, ntiles, p.nblk,
                 [&](int, int tile, int b) -> bool {
-                    const int tm = tile % p.tiles_m, tn = tile / p.tiles_m;
+                    if (b == 0) tile_coords(tile, p.tiles_m, p.tiles_n, p.band_m, tm, tn);   // once per tile: this loop is the issue path
                     return load_stage(&p.map_xq, &p.map_wq, b * 128, tm * 256 + (int)rank * kTileM, tn * TN + (int)rank * (TN / 2), tx_main);
                 },
                 [&](int, int tile, int j) -> bool {
-                    const int tm = tile % p.tiles_m, tn = tile / p.tiles_m;
+                    int tm, tn;
+                    tile_coords(tile, p.tiles_m, p.tiles_n, p.band_m, tm, tn);
                     const int m0 = tm * 256 + (int)rank * kTileM;
                     const int nr = tn * TN + j * kF192Round + (int)rank * (kF192Round / 2);
                     if (p.nmma_o && !load_stage(&p.map_xo, &p.map_wo, 0, m0, nr, tx_aux)) return false;
@@ -231,7 +234,8 @@ __global__ void __launch_bounds__(kF192Threads, 1) fwd192_kernel(const __grid_co
         bool ok = true;
         int t = 0, rounds = 0;
         for (int tile = unit; tile < ntiles && ok; tile += nunits, ++t) {
-            const int tm = tile % p.tiles_m, tn = tile / p.tiles_m;
+            int tm, tn;
+            tile_coords(tile, p.tiles_m, p.tiles_n, p.band_m, tm, tn);
             const int m0 = tm * 256 + (int)rank * kTileM, n0 = tn * TN;
             const int buf = t & 1;
             float* scale_w = scales + buf * 2 * TN;
@@ -261,11 +265,18 @@ __global__ void __launch_bounds__(kF192Threads, 1) fwd192_kernel(const __grid_co
                     if (has_l) tmem_ld_32x16(lane_addr + kColAuxL + (uint32_t)(g * 32 + 16 * h), r2);
                     tmem_ld_wait();
                     if (m < p.M && nc < p.N) {
-                        float y[16];
+                        float y[16], sw[16], so[16];     // the 16 column scales by 128-bit shared loads
+#pragma unroll
+                        for (int i = 0; i < 16; i += 4) {
+                            const float4 a = *reinterpret_cast<const float4*>(scale_w + c0 + i);
+                            sw[i] = a.x; sw[i + 1] = a.y; sw[i + 2] = a.z; sw[i + 3] = a.w;
+                            const float4 b = has_o ? *reinterpret_cast<const float4*>(scale_o + c0 + i) : make_float4(0.f, 0.f, 0.f, 0.f);
+                            so[i] = b.x; so[i + 1] = b.y; so[i + 2] = b.z; so[i + 3] = b.w;
+                        }
 #pragma unroll
                         for (int i = 0; i < 16; ++i) {
-                            float w = (float)(int)r0[i] * scale_w[c0 + i];
-                            if (has_o) w += (float)(int)r1[i] * scale_o[c0 + i];
+                            float w = (float)(int)r0[i] * sw[i];
+                            if (has_o) w += (float)(int)r1[i] * so[i];
                             float v = dxm * w;
                             if (has_l) v += p.lora_scale * __uint_as_float(r2[i]);
                             y[i] = v;

@@ -325,6 +325,15 @@ __global__ void bwd_fixup_kernel(const float* __restrict__ P, int64_t ldp, int M
 
 static int pad16(int r) { return (r + 15) / 16 * 16; }
 
+// Row tiles per band of the tile order: a band of the A operand (band x rows_per_tile rows of a_row_bytes) should
+// stay in L2 while the column tiles sweep over it; at least enough row tiles to keep every CTA pair busy.
+static int band_rows(int tiles_m, int tiles_n, int rows_per_tile, size_t a_row_bytes) {
+    const size_t budget = 40u << 20;
+    int b = (int)max((size_t)1, budget / max((size_t)1, (size_t)rows_per_tile * a_row_bytes));
+    b = max(b, ceil_div(148 / 2, max(tiles_n, 1)));
+    return min(b, max(tiles_m, 1));
+}
+
 constexpr int kPlanSMs = 148;   // split-K plans (and so workspace sizes) are fixed for the B200's 148 SMs
 
 // Split-K plan of a skinny GEMM with `rows_out` output rows and a contraction of `kc` elements (bf16,
@@ -390,6 +399,7 @@ static quaff_status_t skinny_gemm(int mn_major, const void* A, int64_t lda, cons
     p.nphases = 1;
     p.M = rows_out; p.N = rp;
     p.tiles_m = ceil_div(rows_out, kTileM); p.tiles_n = sp.S;
+    p.band_m = p.tiles_m;
     p.status = status;
     p.part = part; p.part_ld = r; p.part_cols = r;
     *S_out = sp.S;
@@ -567,6 +577,7 @@ extern "C" quaff_status_t quaff_qlinear_fwd(int M, int K, int N, const int8_t* X
         }
         q.M = M; q.N = N;
         q.tiles_m = ceil_div(M, 2 * kTileM); q.tiles_n = ceil_div(N, kF192TN);
+        q.band_m = band_rows(q.tiles_m, q.tiles_n, 2 * kTileM, (size_t)K);
         q.status = status_opt;
         q.dx = dx; q.dW = dW; q.dw_O = dw_O; q.lora_scale = lora_scale;
         q.Y = Y; q.ldy = ldy; q.y_f32 = (y_dtype == QUAFF_F32);
@@ -603,6 +614,7 @@ extern "C" quaff_status_t quaff_qlinear_fwd(int M, int K, int N, const int8_t* X
     p.nphases = np;
     p.M = M; p.N = N;
     p.tiles_m = ceil_div(M, kTileM * CTAS); p.tiles_n = ceil_div(N, TN);
+    p.band_m = band_rows(p.tiles_m, p.tiles_n, kTileM * CTAS, (size_t)K);
     p.status = status_opt;
     p.dx = dx; p.dW = dW; p.dw_O = dw_O; p.lora_scale = lora_scale;
     p.has_outlier = nOp > 0; p.has_lora = r > 0;
@@ -703,6 +715,7 @@ extern "C" quaff_status_t quaff_qlinear_bwd(int M, int K, int N, const quaff_bf1
         p.N = Kext;
         p.tiles_m = ceil_div(M, kTileM * CTAS);
         p.tiles_n = ceil_div(p.N, TN);
+        p.band_m = band_rows(p.tiles_m, p.tiles_n, kTileM * CTAS, (size_t)N * 2);
         p.status = status_opt;
         p.dX = dX; p.lddx = lddx; p.P = P; p.ldp = 2 * nOp;
         rc = TN == 256 ? launch_gemm<EPI_BWD, CTAS, 256>(p, st) : launch_gemm<EPI_BWD, CTAS, 128>(p, st);

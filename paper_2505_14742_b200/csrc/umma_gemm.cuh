@@ -77,11 +77,23 @@ struct GemmPhase {
 
 enum { EPI_FWD = 0, EPI_BWD = 1, EPI_PART = 2 };
 
+// Tile order.  The tiles that run at the same time should share operands in L2: the row tiles are cut into
+// BANDS of band_m row tiles; inside a band the order is column tile by column tile, row tiles fastest, so that the
+// ~74 concurrent tiles cover one band of A (sized by the host to stay L2-resident) and a few column panels of B.
+__device__ __forceinline__ void tile_coords(int tile, int tiles_m, int tiles_n, int band_m, int& tm, int& tn) {
+    const int per_band = band_m * tiles_n;
+    const int band = tile / per_band, rem = tile - band * per_band;
+    const int rows = min(band_m, tiles_m - band * band_m);     // the last band may be shorter
+    tn = rem / rows;
+    tm = band * band_m + (rem - tn * rows);
+}
+
 struct GemmParams {
     GemmPhase ph[kMaxPhases];
     int nphases;
     int M, N;            // output extent (rows, columns)
     int tiles_m, tiles_n;
+    int band_m;          // row tiles per band of the tile order (tiles_m: one band)
     int32_t* status;
     // forward epilogue (Eq. 9 + LoRA)
     const float* dx;     // [M]
@@ -202,7 +214,8 @@ __global__ void __launch_bounds__(kGemmThreads, 1) umma_gemm_kernel(const __grid
             uint32_t stage = 0, phase = 0;
             bool ok = true;
             for (int tile = unit; tile < ntiles && ok; tile += nunits) {
-                const int tm = tile % p.tiles_m, tn = tile / p.tiles_m;
+                int tm, tn;
+                tile_coords(tile, p.tiles_m, p.tiles_n, p.band_m, tm, tn);
                 const int m0 = tm * (kTileM * CTAS) + (int)rank * kTileM;
                 for (int i = 0; i < p.nphases && ok; ++i) {
                     const GemmPhase& ph = p.ph[i];
@@ -245,7 +258,8 @@ __global__ void __launch_bounds__(kGemmThreads, 1) umma_gemm_kernel(const __grid
             bool ok = true;
             int t = 0;
             for (int tile = unit; tile < ntiles && ok; tile += nunits, ++t) {
-                const int tn = tile / p.tiles_m;
+                int tm, tn;
+                tile_coords(tile, p.tiles_m, p.tiles_n, p.band_m, tm, tn);
                 for (int i = 0; i < p.nphases && ok; ++i) {
                     const GemmPhase& ph = p.ph[i];
                     if (tn < ph.tn_limit) {
@@ -299,7 +313,8 @@ __global__ void __launch_bounds__(kGemmThreads, 1) umma_gemm_kernel(const __grid
         bool ok = true;
         int t = 0;
         for (int tile = unit; tile < ntiles && ok; tile += nunits, ++t) {
-            const int tm = tile % p.tiles_m, tn = tile / p.tiles_m;
+            int tm, tn;
+            tile_coords(tile, p.tiles_m, p.tiles_n, p.band_m, tm, tn);
             const int m0 = tm * (kTileM * CTAS) + (int)rank * kTileM, n0 = tn * TN;
             const int buf = t & 1;
             float* scale_w = scales + buf * 2 * TN;
