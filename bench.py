@@ -399,6 +399,49 @@ def run_micro(args):
     X[:, O.long()] *= 50.0
     s = 1.0 + 10.0 * torch.rand(nO, device="cuda", generator=g)
     flush = torch.empty(512 << 20, dtype=torch.uint8, device="cuda")
+    if args.micro in ("fwd", "bwd"):
+        # one layer's forward (or backward) call on random codes; the tensor-core GEMM inside it is timed by the
+        # library's event pair (quaff_debug_time_gemm), everything else of the call runs untimed around it
+        r = args.micro_rank
+        i8 = lambda *shape: torch.randint(-127, 128, shape, dtype=torch.int8, device="cuda", generator=g)
+        Xq, Wq, xqo, wqo = i8(M, K), i8(N, K), i8(M, nOp), i8(N, nOp)
+        dxv, dWv, dwOv = (torch.rand(n, device="cuda", generator=g) * 1e-2 for n in (M, N, N))
+        A = (0.02 * torch.randn((K, r), device="cuda", generator=g)).to(torch.bfloat16)
+        B = (0.02 * torch.randn((r, N), device="cuda", generator=g)).to(torch.bfloat16)
+        T = torch.empty((M, r), dtype=torch.bfloat16, device="cuda")
+        Y = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
+        dY = (0.01 * torch.randn((M, N), device="cuda", generator=g)).to(torch.bfloat16)
+        dX = torch.empty((M, K), dtype=torch.bfloat16, device="cuda")
+        dA = torch.zeros((K, r), device="cuda"); dB = torch.zeros((r, N), device="cuda")
+        st = torch.zeros(4, dtype=torch.int32, device="cuda")
+        ws = torch.empty(max(Q.workspace_bytes(Q.QUAFF_WS_FWD, M, K, N, nOp, r), Q.workspace_bytes(Q.QUAFF_WS_BWD, M, K, N, nOp, r)),
+                         dtype=torch.uint8, device="cuda")
+        Q.quaff_qlinear_fwd(Xq, xqo, dxv, Wq, dWv, wqo, dwOv, X, A, B, 1.0, T, Y, ws, None, None, st)
+        which = 0 if args.micro == "fwd" else 1
+        times = []
+        for i in range(args.warmup + args.steps):
+            flush.sum()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(); e1.record()
+            Q.quaff_debug_time_gemm(which, e0, e1)
+            if which == 0:
+                Q.quaff_qlinear_fwd(Xq, xqo, dxv, Wq, dWv, wqo, dwOv, X, A, B, 1.0, T, Y, ws, None, None, st)
+            else:
+                Q.quaff_qlinear_bwd(dY, Wq, dWv, wqo, dwOv, O, s, X, T, A, B, 1.0, dX, dA, dB, False, ws, st)
+            torch.cuda.synchronize()
+            if i >= args.warmup:
+                times.append(e0.elapsed_time(e1))
+        assert int(st[0].item()) == 0, "device-side wait timed out"
+        ms = float(np.median(times))
+        peaks = load_peaks()
+        work = 2.0 * M * N * (K + nOp + r) if which == 0 else 2.0 * M * N * (K + 2 * nOp) + 2.0 * M * K * r
+        peak = peaks["bf16_tflops"] * (2.0 if which == 0 else 1.0)
+        print(json.dumps({"micro": args.micro, "shape": {"M": M, "K": K, "N": N, "nO": nO, "r": r}, "ms_per_launch": ms, "launches": len(times),
+                          "roofline": {"bound": "tensor", "achieved": work / (ms * 1e-3) / 1e12, "peak": peak,
+                                       "unit": "TOP/s" if which == 0 else "TFLOP/s", "frac": work / (ms * 1e-3) / 1e12 / peak,
+                                       "peak_source": f"{peaks['source']} cuBLAS bf16 burst" + (" x2 (nominal int8:bf16 ratio)" if which == 0 else "")}}),
+              flush=True)
+        return
     if args.micro == "quant_act":
         Xq = torch.empty((M, K), dtype=torch.int8, device="cuda")
         xqo = torch.empty((M, nOp), dtype=torch.int8, device="cuda")
@@ -448,13 +491,14 @@ def run_micro(args):
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--micro", default=None, choices=["quant_act", "momentum", "requant", "outlier_count", "lora_down"],
+    ap.add_argument("--micro", default=None, choices=["quant_act", "momentum", "requant", "outlier_count", "lora_down", "fwd", "bwd"],
                     help="time one HBM-bound kernel alone instead of the step")
     ap.add_argument("--micro-shape", type=lambda v: tuple(int(x) for x in v.split(",")), default=(8192, 11008, 4096, 55),
                     help="M,K,N,nO of --micro (default: the LLaMA-2-7B down_proj rows)")
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=1000)
     ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--micro-rank", type=int, default=64, help="LoRA rank of --micro fwd / bwd")
     ap.add_argument("--workload", default="phi3_attn", choices=sorted(synth.WORKLOADS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--sample-tokens", type=int, default=128, help="tokens per step of the CPU oracle (reference arm); the cpu_baseline leg uses 8x this")
