@@ -418,15 +418,24 @@ static FwdWorkspace fwd_workspace(int M, int K, int N, int r) {
     return w;
 }
 
-// Output-column tile of the grad-input GEMM: a 256-wide MMA runs at nearly twice the rate of a 128-wide
-// one (measured), 128 fills the machine better when there are few tiles.  Cost model: waves x tile
-// width, 128-wide tiles 1.8x dearer per column.
+// Output-column tile of the grad-input GEMM.  A tcgen05.mma of a CTA pair costs about 60 + N/2 clocks
+// (measured: N = 128: 125, 192: 165, 256: 190), so wide tiles are cheaper per column, while narrow ones
+// leave a smaller ragged last wave.  Cost model: waves on the CTA pairs x cost of one MMA of that width.
 static int bwd_tile_n(int M, int K, int nOp) {
     const int units = kPlanSMs / 2;
     const int tm = ceil_div(M, 2 * kTileM);
-    const double c256 = (double)ceil_div(tm * (ceil_div(K, 256) + (nOp > 0)), units) * 256.0;
-    const double c128 = (double)ceil_div(tm * (ceil_div(K, 128) + (nOp > 0)), units) * 128.0 * 1.8;
-    return c256 <= c128 ? 256 : 128;
+    const int widths[3] = {256, 192, 128};
+    const double mma_cost[3] = {190.0, 165.0, 125.0};
+    int best = 256;
+    double best_cost = 0.0;
+    for (int i = 0; i < 3; ++i) {
+        const int tn = widths[i];
+        const int kpad = ceil_div(K, tn) * tn;
+        const int tiles = tm * ceil_div(kpad + 2 * nOp, tn);
+        const double cost = (double)ceil_div(tiles, units) * mma_cost[i];
+        if (i == 0 || cost < best_cost) { best = tn; best_cost = cost; }
+    }
+    return best;
 }
 
 struct BwdWorkspace {
@@ -718,7 +727,7 @@ extern "C" quaff_status_t quaff_qlinear_bwd(int M, int K, int N, const quaff_bf1
         p.band_m = band_rows(p.tiles_m, p.tiles_n, kTileM * CTAS, (size_t)N * 2);
         p.status = status_opt;
         p.dX = dX; p.lddx = lddx; p.P = P; p.ldp = 2 * nOp;
-        rc = TN == 256 ? launch_gemm<EPI_BWD, CTAS, 256>(p, st) : launch_gemm<EPI_BWD, CTAS, 128>(p, st);
+        rc = TN == 256 ? launch_gemm<EPI_BWD, CTAS, 256>(p, st) : TN == 192 ? launch_gemm<EPI_BWD, CTAS, 192>(p, st) : launch_gemm<EPI_BWD, CTAS, 128>(p, st);
         if (rc != QUAFF_OK) return rc;
     }
     if (want_dAB) {   // dA = X^T G (MN-major operands), beside the outlier fix-up

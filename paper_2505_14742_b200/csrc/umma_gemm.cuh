@@ -6,7 +6,8 @@
 //   warps 2..5  : epilogue - tcgen05.ld of the finished accumulators, dequantization / conversion, stores
 //
 // Template parameters: EPI (which epilogue), CTAS (1, or 2 = a CTA pair on two SMs that shares one
-// 256-row output tile through tcgen05 cta_group::2) and TN (output columns per tile, 128 or 256).
+// 256-row output tile through tcgen05 cta_group::2) and TN (output columns per tile: 128, 256, and 192 for
+// the grad-input GEMM).
 //
 // CTA pair (CTAS = 2, a cluster of two): each CTA loads its own 128 rows of A and its own half
 // (TN / 2 output columns) of B into its own shared memory, at the same offsets in both CTAs.  The
@@ -131,7 +132,9 @@ struct GemmSmem {
 
 template <int EPI, int CTAS, int TN>
 struct GemmCfg {
-    static constexpr int kBBytes = (TN / CTAS) * 128;                // B region of a stage, per CTA
+    // B region of a stage, per CTA: whole boxes of 64 output columns (an MN-major operand is loaded box by box;
+    // with TN = 192 a CTA of a pair owns 96 columns, one box and a half)
+    static constexpr int kBBytes = ((TN / CTAS + 63) / 64) * 64 * 128;
     static constexpr int kStageBytes = kABytes + kBBytes;
     static constexpr int kScaleBytes = (EPI == EPI_FWD) ? 2 * 2 * TN * 4 : 0;   // [2 buffers][dW | dw_O][TN]
     static constexpr int kFixed = 1024 + (int)sizeof(GemmSmem) + kScaleBytes;
@@ -158,7 +161,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) umma_gemm_kernel(const __grid
     constexpr int kStages = Cfg::kStages;
     constexpr int kStageBytes = Cfg::kStageBytes;
     static_assert(CTAS == 1 || CTAS == 2, "one CTA or a CTA pair");
-    static_assert(TN == 128 || TN == 256, "output-column tile");   // TN = 256: slot 0 only (no room for auxiliary accumulators)
+    static_assert(TN == 128 || TN == 256 || (TN == 192 && EPI == EPI_BWD && CTAS == 2), "output-column tile");   // TN > 128: slot 0 only (no room for auxiliary accumulators)
 
     extern __shared__ unsigned char smem_dyn[];
     const uint32_t raw = smem_u32(smem_dyn);
