@@ -217,6 +217,16 @@ def outlier_count(X: np.ndarray, thr: int, xi: np.ndarray) -> np.ndarray:
     return out
 
 
+def outlier_hits(X: np.ndarray, thr: int, O_idx: np.ndarray) -> np.ndarray:
+    """Hit-rate monitor (Sec. 3.2): [|R and O|, |R|] with R the Eq. 6 outlier channels of this batch X[M,K] (bf16 bits)."""
+    X = _c(X, np.uint16)
+    M, K = X.shape
+    O = _c(O_idx, np.int32)
+    hits = np.zeros(2, np.int32)
+    _load().qo_outlier_hits(_p(X), I64(K), I32(M), I32(K), I32(int(thr)), _p(O), I32(O.shape[0]), _p(hits))
+    return hits
+
+
 def select_outliers(xi: np.ndarray, nO: int) -> np.ndarray:
     """The nO channels with the largest xi (ties: lower index first), sorted ascending (int32)."""
     xi = _c(xi, np.int32)

@@ -386,6 +386,21 @@ void qo_outlier_count(const uint16_t* X, int64_t ldx, int M, int K, int thr, int
     }
 }
 
+/* Hit rate of the predefined outlier set during fine-tuning (Sec. 3.2, the hit-rate figures): of the channels that are
+ * outliers of the current batch X by the criterion of Eq. 6 (the "real-time" outliers R), how many lie in O.
+ *   hits[0] = |R and O|,  hits[1] = |R|;  the hit rate is hits[0] / hits[1] (undefined when the batch has no outlier).
+ * O_idx holds distinct channel indices. */
+void qo_outlier_hits(const uint16_t* X, int64_t ldx, int M, int K, int thr, const int32_t* O_idx, int nO, int32_t* hits) {
+    int32_t* ind = (int32_t*)calloc((size_t)(K > 0 ? K : 1), sizeof(int32_t));
+    qo_outlier_count(X, ldx, M, K, thr, ind); /* ind[k] = 1 for a real-time outlier channel */
+    int32_t in_set = 0, all = 0;
+    for (int k = 0; k < K; ++k) all += ind[k];
+    for (int i = 0; i < nO; ++i) in_set += ind[O_idx[i]];
+    hits[0] = in_set;
+    hits[1] = all;
+    free(ind);
+}
+
 /* The nO channels with the largest xi (ties: the lower channel index first), as a sorted index set. */
 void qo_select_outliers(const int32_t* xi, int K, int nO, int32_t* O_idx) {
     char* taken = (char*)calloc((size_t)(K > 0 ? K : 1), 1);

@@ -469,3 +469,31 @@ def test_select_outliers_ties_and_order():
     assert oracle.select_outliers(xi, 4).tolist() == [0, 1, 2, 4]   # sorted ascending
     assert oracle.select_outliers(xi, 0).tolist() == []
     assert oracle.select_outliers(xi, 6).tolist() == [0, 1, 2, 3, 4, 5]
+
+
+# ----------------------------------------------------------------------------- hit-rate monitor (Sec. 3.2)
+def test_outlier_hits_hand_case():
+    # one token; channels 1 and 4 are far above thr x mean: R = {1, 4}.  mean|X| = (4 + 2 * 640) / 6 = 214; thr = 2 -> 428
+    X = synth.f32_to_bf16_bits(np.array([[1.0, 640.0, 1.0, 1.0, 640.0, 1.0]], np.float32))
+    assert oracle.outlier_hits(X, 2, np.array([1, 4], np.int32)).tolist() == [2, 2]      # every real-time outlier predicted
+    assert oracle.outlier_hits(X, 2, np.array([0, 1], np.int32)).tolist() == [1, 2]      # one of two
+    assert oracle.outlier_hits(X, 2, np.array([0, 2, 3, 5], np.int32)).tolist() == [0, 2]
+    assert oracle.outlier_hits(X, 2, np.zeros(0, np.int32)).tolist() == [0, 2]           # empty O
+    assert oracle.outlier_hits(X, 1000, np.array([1, 4], np.int32)).tolist() == [0, 0]   # no channel crosses: rate undefined
+
+
+def test_outlier_hits_matches_brute_force_sets():
+    rng = np.random.default_rng(23)
+    for M, K, nO in ((3, 9, 2), (8, 40, 5), (16, 33, 33)):
+        x = rng.standard_normal((M, K)).astype(np.float32)
+        x[:, rng.choice(K, 3, replace=False)] *= 200.0
+        xb = synth.f32_to_bf16_bits(x)
+        O = np.sort(rng.choice(K, nO, replace=False)).astype(np.int32)
+        for thr in (1, 4, 30):
+            R = set(np.flatnonzero(_xi_brute(synth.bf16_bits_to_f32(xb), thr)).tolist())
+            got = oracle.outlier_hits(xb, thr, O).tolist()
+            assert got == [len(R & set(O.tolist())), len(R)], (M, K, thr, got)
+            # the full channel set predicts everything; the complement of O the rest
+            assert oracle.outlier_hits(xb, thr, np.arange(K, dtype=np.int32)).tolist() == [len(R), len(R)]
+            comp = np.setdiff1d(np.arange(K), O).astype(np.int32)
+            assert oracle.outlier_hits(xb, thr, comp)[0] == len(R) - got[0]
