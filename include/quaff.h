@@ -52,7 +52,8 @@ enum { /* `which` of quaff_workspace_bytes */
     QUAFF_WS_MOMENTUM = 1,
     QUAFF_WS_FWD = 2,
     QUAFF_WS_BWD = 3,
-    QUAFF_WS_CALIBRATE = 4   /* quaff_outlier_count and quaff_select_outliers (depends on K only) */
+    QUAFF_WS_CALIBRATE = 4,  /* quaff_outlier_count and quaff_select_outliers (depends on K only) */
+    QUAFF_WS_HITS = 5        /* quaff_outlier_hits (depends on K only) */
 };
 
 const char* quaff_status_string(quaff_status_t s);
@@ -78,6 +79,18 @@ quaff_status_t quaff_outlier_count(const quaff_bf16* X, int64_t ldx, int M, int 
  */
 quaff_status_t quaff_select_outliers(const int32_t* xi, int K, int nO, int32_t* O_idx, void* ws, size_t ws_bytes,
                                      quaff_stream_t stream);
+
+/*
+ * Hit-rate monitor during fine-tuning (Sec. 3.2, the hit-rate figures): of the channels that are outliers of the
+ * CURRENT batch X by the criterion of Eq. 6 (the "real-time" outliers R, same integer decision as quaff_outlier_count),
+ * how many lie in the predefined set O.
+ *   hits[0] = |R and O|,  hits[1] = |R|   (device int32[2], overwritten);  hit rate = hits[0] / hits[1], undefined
+ *   when the batch has no outlier channel.  The caller averages over iterations and layers.
+ *   X [M][K] bf16, ldx (ldx % 8 == 0);  O_idx [nO] distinct channel indices (an index outside [0,K) is ignored);
+ *   ws: QUAFF_WS_HITS bytes
+ */
+quaff_status_t quaff_outlier_hits(const quaff_bf16* X, int64_t ldx, int M, int K, int thr, const int32_t* O_idx, int nO,
+                                  int32_t* hits, void* ws, size_t ws_bytes, quaff_stream_t stream);
 
 /*
  * One-time weight preprocessing (Sec. 3.3, "weights preprocessing"; Eq. 1 per output channel).

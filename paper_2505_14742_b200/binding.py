@@ -22,9 +22,9 @@ QUAFF_ERR_WORKSPACE_TOO_SMALL = 4
 QUAFF_ERR_CUDA = 5
 QUAFF_ERR_TIMEOUT = 6
 QUAFF_BF16, QUAFF_F32 = 0, 1
-QUAFF_WS_PREPARE, QUAFF_WS_MOMENTUM, QUAFF_WS_FWD, QUAFF_WS_BWD, QUAFF_WS_CALIBRATE = 0, 1, 2, 3, 4
+QUAFF_WS_PREPARE, QUAFF_WS_MOMENTUM, QUAFF_WS_FWD, QUAFF_WS_BWD, QUAFF_WS_CALIBRATE, QUAFF_WS_HITS = 0, 1, 2, 3, 4, 5
 
-EXPORTS = ("quaff_status_string", "quaff_workspace_bytes", "quaff_debug_launch_count", "quaff_debug_time_gemm", "quaff_prepare_weight", "quaff_momentum_update", "quaff_lora_down", "quaff_outlier_count", "quaff_select_outliers",
+EXPORTS = ("quaff_status_string", "quaff_workspace_bytes", "quaff_debug_launch_count", "quaff_debug_time_gemm", "quaff_prepare_weight", "quaff_momentum_update", "quaff_lora_down", "quaff_outlier_count", "quaff_select_outliers", "quaff_outlier_hits",
            "quaff_momentum_update_static", "quaff_quant_act", "quaff_requant_weight_rows", "quaff_qlinear_fwd", "quaff_qlinear_bwd")
 
 _lib = None
@@ -64,6 +64,8 @@ def lib() -> ctypes.CDLL:
         L.quaff_quant_act.argtypes = [_vp, _i64, _i32, _i32, _vp, _i32, _vp, _vp, _i64, _vp, _i64, _i32, _vp, _vp]
         L.quaff_requant_weight_rows.restype = _i32
         L.quaff_requant_weight_rows.argtypes = [_vp, _i64, _i32, _i32, _vp, _vp, _i64, _i32, _vp, _vp]
+        L.quaff_outlier_hits.restype = _i32
+        L.quaff_outlier_hits.argtypes = [_vp, _i64, _i32, _i32, _i32, _vp, _i32, _vp, _vp, _sz, _vp]
         L.quaff_outlier_count.restype = _i32
         L.quaff_outlier_count.argtypes = [_vp, _i64, _i32, _i32, _i32, _vp, _vp, _sz, _vp]
         L.quaff_select_outliers.restype = _i32
@@ -127,6 +129,13 @@ def quaff_outlier_count(X, thr: int, xi, ws) -> None:
     M, K = X.shape
     _check(lib().quaff_outlier_count(_ptr(X), _ld(X), M, K, int(thr), _ptr(xi), _ptr(ws), ws.numel() * ws.element_size(),
                                      _stream()), "quaff_outlier_count")
+
+
+def quaff_outlier_hits(X, thr: int, O_idx, hits, ws) -> None:
+    M, K = X.shape
+    nO = 0 if O_idx is None else O_idx.numel()
+    _check(lib().quaff_outlier_hits(_ptr(X), _ld(X), M, K, int(thr), _ptr(O_idx), nO, _ptr(hits), _ptr(ws),
+                                    ws.numel() * ws.element_size(), _stream()), "quaff_outlier_hits")
 
 
 def quaff_select_outliers(xi, O_idx, ws) -> None:

@@ -171,6 +171,47 @@ __global__ void __launch_bounds__(1024) outlier_compact_kernel(const unsigned ch
     }
 }
 
+// Hit-rate monitor: ind[k] > 0 marks a real-time outlier channel of the batch; hits = {those inside O, all of them}.
+__global__ void __launch_bounds__(1024) outlier_hits_kernel(const int32_t* __restrict__ ind, int K, const int32_t* __restrict__ O_idx,
+                                                            int nO, int32_t* __restrict__ hits) {
+    pdl_launch_dependents();
+    pdl_wait();
+    __shared__ int acc[2];
+    if (threadIdx.x < 2) acc[threadIdx.x] = 0;
+    __syncthreads();
+    int in_set = 0, all = 0;
+    for (int k = threadIdx.x; k < K; k += blockDim.x) all += ind[k] > 0;
+    for (int i = threadIdx.x; i < nO; i += blockDim.x) {
+        const int o = O_idx[i];
+        if ((unsigned)o < (unsigned)K) in_set += ind[o] > 0;      // an index outside [0, K) is ignored
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        all += __shfl_xor_sync(0xffffffffu, all, o);
+        in_set += __shfl_xor_sync(0xffffffffu, in_set, o);
+    }
+    if ((threadIdx.x & 31) == 0) {
+        atomicAdd(&acc[0], in_set);
+        atomicAdd(&acc[1], all);
+    }
+    __syncthreads();
+    if (threadIdx.x < 2) hits[threadIdx.x] = acc[threadIdx.x];
+}
+
+// Eq. 6 indicator of one sample added to xi; ws = QUAFF_WS_CALIBRATE bytes (cleared here).
+static quaff_status_t launch_outlier_count(const quaff_bf16* X, int64_t ldx, int M, int K, int thr, int32_t* xi, void* ws, cudaStream_t st) {
+    const size_t need = quaff_workspace_bytes(QUAFF_WS_CALIBRATE, M, K, 0, 0, 0);
+    if (cudaMemsetAsync(ws, 0, need, st) != cudaSuccess) return QUAFF_ERR_CUDA;
+    unsigned int* colmax = reinterpret_cast<unsigned int*>(ws);
+    unsigned char* tail = reinterpret_cast<unsigned char*>(ws) + round_up((size_t)K * 4, 256);
+    const int bx = ceil_div(K, 256);
+    const int by = max(1, min(ceil_div(M, 32), ceil_div(4 * sm_count(), bx)));
+    const int rows_per_block = ceil_div(M, by);
+    launch_pdl(outlier_count_kernel, dim3(bx, ceil_div(M, rows_per_block)), dim3(256), 0, st, 1, X, ldx, M, K, thr, xi, colmax,
+               reinterpret_cast<unsigned long long*>(tail), reinterpret_cast<unsigned int*>(tail + 8), rows_per_block);
+    return launch_status();
+}
+
 }  // namespace quaff
 
 using namespace quaff;
@@ -181,15 +222,23 @@ extern "C" quaff_status_t quaff_outlier_count(const quaff_bf16* X, int64_t ldx, 
     QUAFF_RETURN_IF(!aligned16(X) || (ldx % 8), QUAFF_ERR_ALIGNMENT);
     const size_t need = quaff_workspace_bytes(QUAFF_WS_CALIBRATE, M, K, 0, 0, 0);
     QUAFF_RETURN_IF(!ws || !aligned16(ws) || ws_bytes < need, QUAFF_ERR_WORKSPACE_TOO_SMALL);
+    return launch_outlier_count(X, ldx, M, K, thr, xi, ws, (cudaStream_t)stream);
+}
+
+extern "C" quaff_status_t quaff_outlier_hits(const quaff_bf16* X, int64_t ldx, int M, int K, int thr, const int32_t* O_idx, int nO,
+                                             int32_t* hits, void* ws, size_t ws_bytes, quaff_stream_t stream) {
+    QUAFF_RETURN_IF(!X || !hits || M <= 0 || K <= 0 || ldx < K || thr < 0 || nO < 0 || nO > K || (nO > 0 && !O_idx), QUAFF_ERR_INVALID_ARG);
+    QUAFF_RETURN_IF(!aligned16(X) || (ldx % 8), QUAFF_ERR_ALIGNMENT);
+    const size_t need = quaff_workspace_bytes(QUAFF_WS_HITS, M, K, 0, 0, 0);
+    QUAFF_RETURN_IF(!ws || !aligned16(ws) || ws_bytes < need, QUAFF_ERR_WORKSPACE_TOO_SMALL);
     cudaStream_t st = (cudaStream_t)stream;
-    if (cudaMemsetAsync(ws, 0, need, st) != cudaSuccess) return QUAFF_ERR_CUDA;
-    unsigned int* colmax = reinterpret_cast<unsigned int*>(ws);
-    unsigned char* tail = reinterpret_cast<unsigned char*>(ws) + round_up((size_t)K * 4, 256);
-    const int bx = ceil_div(K, 256);
-    const int by = max(1, min(ceil_div(M, 32), ceil_div(4 * sm_count(), bx)));
-    const int rows_per_block = ceil_div(M, by);
-    launch_pdl(outlier_count_kernel, dim3(bx, ceil_div(M, rows_per_block)), dim3(256), 0, st, 1, X, ldx, M, K, thr, xi, colmax,
-               reinterpret_cast<unsigned long long*>(tail), reinterpret_cast<unsigned int*>(tail + 8), rows_per_block);
+    // workspace: the counting pass's own scratch, then the indicator of this batch (one int32 per channel)
+    const size_t off_ind = quaff_workspace_bytes(QUAFF_WS_CALIBRATE, M, K, 0, 0, 0);
+    int32_t* ind = reinterpret_cast<int32_t*>(reinterpret_cast<unsigned char*>(ws) + off_ind);
+    if (cudaMemsetAsync(ind, 0, (size_t)K * 4, st) != cudaSuccess) return QUAFF_ERR_CUDA;
+    quaff_status_t rc = launch_outlier_count(X, ldx, M, K, thr, ind, ws, st);
+    if (rc != QUAFF_OK) return rc;
+    launch_pdl(outlier_hits_kernel, dim3(1), dim3(1024), 0, st, 1, (const int32_t*)ind, K, O_idx, nO, hits);
     return launch_status();
 }
 

@@ -522,6 +522,7 @@ extern "C" size_t quaff_workspace_bytes(int which, int M, int K, int N, int nOp,
         case QUAFF_WS_FWD: return fwd_workspace(M, K, N, r).total;
         case QUAFF_WS_BWD: return bwd_workspace(M, K, N, nOp, r).total;
         case QUAFF_WS_CALIBRATE: return round_up((size_t)max(K, 0) * 4, 256) + 256;   // column maxima / flags, sum, ticket
+        case QUAFF_WS_HITS: return 2 * round_up((size_t)max(K, 0) * 4, 256) + 256;    // the same, then this batch's indicator
     }
     return 0;
 }
