@@ -504,8 +504,14 @@ def main():
     ap.add_argument("--sample-tokens", type=int, default=128, help="tokens per step of the CPU oracle (reference arm); the cpu_baseline leg uses 8x this")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--eager", action="store_true", help="enqueue every launch from Python instead of replaying a CUDA graph of the step")
+    ap.add_argument("--fwd-tile", type=int, default=0, choices=[0, 128, 192, 256],
+                    help="force the forward kernel's output-column tile (0: the library's cost model decides)")
     args = ap.parse_args()
     wl = synth.WORKLOADS[args.workload]
+    if args.fwd_tile and args.impl != "reference":
+        from paper_2505_14742_b200 import binding, build
+        build.build_library()
+        binding.quaff_debug_force_fwd_tile(args.fwd_tile)
     if args.micro:
         if args.steps == 1000:
             args.steps = 30

@@ -252,6 +252,10 @@ quaff_status_t quaff_momentum_update_static(const quaff_bf16* X, int64_t ldx, in
  *
  * quaff_debug_launch_count: number of kernels this library has launched since it was loaded.
  *
+ * quaff_debug_force_fwd_tile: quaff_qlinear_fwd picks the output-column tile of its kernel (128, 192 or 256) by a
+ * cost model; tile_n = 128 / 192 / 256 forces that kernel where the shape allows it (outlier set or LoRA present,
+ * nOp <= 128), 0 gives the choice back to the cost model.  For tests and timing of each kernel on the same shape.
+ *
  * quaff_debug_time_gemm: arm a one-shot pair of CUDA events (cudaEvent_t, created by the caller
  * with timing enabled) around the next launch of the forward (which = 0) or grad-input
  * (which = 1) tensor-core GEMM kernel: `start` is recorded on the launch stream right before the
@@ -260,6 +264,7 @@ quaff_status_t quaff_momentum_update_static(const quaff_bf16* X, int64_t ldx, in
  * them again, and the elapsed time between them is that of the latest replay.
  */
 uint64_t quaff_debug_launch_count(void);
+void quaff_debug_force_fwd_tile(int tile_n);
 void quaff_debug_time_gemm(int which, void* start_event, void* stop_event);
 
 #ifdef __cplusplus

@@ -24,7 +24,7 @@ QUAFF_ERR_TIMEOUT = 6
 QUAFF_BF16, QUAFF_F32 = 0, 1
 QUAFF_WS_PREPARE, QUAFF_WS_MOMENTUM, QUAFF_WS_FWD, QUAFF_WS_BWD, QUAFF_WS_CALIBRATE, QUAFF_WS_HITS = 0, 1, 2, 3, 4, 5
 
-EXPORTS = ("quaff_status_string", "quaff_workspace_bytes", "quaff_debug_launch_count", "quaff_debug_time_gemm", "quaff_prepare_weight", "quaff_momentum_update", "quaff_lora_down", "quaff_outlier_count", "quaff_select_outliers", "quaff_outlier_hits",
+EXPORTS = ("quaff_status_string", "quaff_workspace_bytes", "quaff_debug_launch_count", "quaff_debug_force_fwd_tile", "quaff_debug_time_gemm", "quaff_prepare_weight", "quaff_momentum_update", "quaff_lora_down", "quaff_outlier_count", "quaff_select_outliers", "quaff_outlier_hits",
            "quaff_momentum_update_static", "quaff_quant_act", "quaff_requant_weight_rows", "quaff_qlinear_fwd", "quaff_qlinear_bwd")
 
 _lib = None
@@ -80,6 +80,8 @@ def lib() -> ctypes.CDLL:
                                         _vp, _i64, _vp, _vp, _vp, _i32, _f32, _vp, _i64, _vp, _vp, _i32, _vp, _vp, _sz, _vp]
         L.quaff_debug_launch_count.restype = ctypes.c_uint64
         L.quaff_debug_launch_count.argtypes = []
+        L.quaff_debug_force_fwd_tile.restype = None
+        L.quaff_debug_force_fwd_tile.argtypes = [_i32]
         L.quaff_debug_time_gemm.restype = None
         L.quaff_debug_time_gemm.argtypes = [_i32, _vp, _vp]
         _lib = L
@@ -96,6 +98,11 @@ def workspace_bytes(which: int, M: int, K: int, N: int, nOp: int, r: int) -> int
 
 def quaff_debug_launch_count() -> int:
     return int(lib().quaff_debug_launch_count())
+
+
+def quaff_debug_force_fwd_tile(tile_n: int) -> None:
+    """Force the forward kernel's tile width (128 / 192 / 256); 0 = the library's cost model decides."""
+    lib().quaff_debug_force_fwd_tile(int(tile_n))
 
 
 def quaff_debug_time_gemm(which: int, start: Optional["torch.cuda.Event"], stop: Optional["torch.cuda.Event"]) -> None:

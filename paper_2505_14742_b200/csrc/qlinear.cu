@@ -4,7 +4,7 @@
 #include <stdlib.h>
 #include <string.h>
 
-#include "fwd192.cuh"
+#include "fwd256.cuh"
 
 namespace quaff {
 
@@ -139,34 +139,37 @@ static quaff_status_t launch_gemm(const GemmParams& p, cudaStream_t st) {
     return rc;
 }
 
-static quaff_status_t launch_fwd192(const Fwd192Params& p, cudaStream_t st) {
-    static bool configured[64] = {false};
-    static int units_of[64] = {0};
+// The wide forward kernels (fwd192.cuh, fwd256.cuh): which = 0 / 1
+static quaff_status_t launch_fwd_wide(int which, const Fwd192Params& p, cudaStream_t st) {
+    static bool configured[2][64] = {{false}};
+    static int units_of[2][64] = {{0}};
+    void (*const kernel)(const Fwd192Params) = which ? fwd256_kernel : fwd192_kernel;
+    const int threads = which ? kF256Threads : kF192Threads;
+    const size_t smem = which ? kF256SmemBytes : kF192SmemBytes;
     int dev = 0;
     cudaGetDevice(&dev);
     if (dev < 0 || dev >= 64) return QUAFF_ERR_CUDA;
-    if (!configured[dev]) {
-        if (cudaFuncSetAttribute(fwd192_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kF192SmemBytes) != cudaSuccess)
-            return QUAFF_ERR_CUDA;
+    if (!configured[which][dev]) {
+        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return QUAFF_ERR_CUDA;
         int units = sm_count() / 2;
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3(units * 2);
-        cfg.blockDim = dim3(kF192Threads);
-        cfg.dynamicSmemBytes = kF192SmemBytes;
+        cfg.blockDim = dim3(threads);
+        cfg.dynamicSmemBytes = smem;
         cudaLaunchAttribute attr;
         attr.id = cudaLaunchAttributeClusterDimension;
         attr.val.clusterDim.x = 2; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
         cfg.attrs = &attr;
         cfg.numAttrs = 1;
         int nclusters = 0;
-        if (cudaOccupancyMaxActiveClusters(&nclusters, fwd192_kernel, &cfg) == cudaSuccess && nclusters > 0) units = min(units, nclusters);
+        if (cudaOccupancyMaxActiveClusters(&nclusters, kernel, &cfg) == cudaSuccess && nclusters > 0) units = min(units, nclusters);
         else cudaGetLastError();
-        units_of[dev] = max(units, 1);
-        configured[dev] = true;
+        units_of[which][dev] = max(units, 1);
+        configured[which][dev] = true;
     }
     const int ntiles = p.tiles_m * p.tiles_n;
     if (ntiles == 0) return QUAFF_OK;
-    const int units = min(ntiles, units_of[dev]);
+    const int units = min(ntiles, units_of[which][dev]);
     const bool timed = g_time_start[0] && g_time_stop[0];
     unsigned int ev_flags = cudaEventRecordDefault;
     if (timed) {
@@ -174,7 +177,7 @@ static quaff_status_t launch_fwd192(const Fwd192Params& p, cudaStream_t st) {
         if (cudaStreamIsCapturing(st, &cap) == cudaSuccess && cap == cudaStreamCaptureStatusActive) ev_flags = cudaEventRecordExternal;
         cudaEventRecordWithFlags(g_time_start[0], st, ev_flags);
     }
-    launch_pdl(fwd192_kernel, dim3(units * 2), dim3(kF192Threads), kF192SmemBytes, st, 2, p);
+    launch_pdl(kernel, dim3(units * 2), dim3(threads), smem, st, 2, p);
     const quaff_status_t rc = launch_status();
     if (timed) {
         cudaEventRecordWithFlags(g_time_stop[0], st, ev_flags);
@@ -406,6 +409,16 @@ static quaff_status_t skinny_gemm(int mn_major, const void* A, int64_t lda, cons
     return launch_gemm<EPI_PART, 1, 128>(p, st);
 }
 
+static int g_force_fwd_tile = 0;   // quaff_debug_force_fwd_tile: 0 = the cost model decides
+
+// Cost model of the three forward kernels, fitted to sweeps of the number of waves at fixed shapes (B200, clocks of
+// 1965 MHz): a tile of width W takes about  max(MMAs x kFwdMmaClk + kFwdTileOvh, kFwdTileMin)  clocks; the floor is
+// the epilogue of a tile (stores of 16 bytes per row and instruction), which short contractions cannot hide.
+constexpr int kFwdWidths[3] = {128, 192, 256};
+constexpr double kFwdMmaClk[3] = {125.0, 157.0, 190.0};
+constexpr double kFwdTileOvh[3] = {4100.0, 1500.0, 5000.0};
+constexpr double kFwdTileMin[3] = {10900.0, 22500.0, 18700.0};
+
 struct FwdWorkspace { size_t off_bt, off_at, off_part, total; };
 static FwdWorkspace fwd_workspace(int M, int K, int N, int r) {
     FwdWorkspace w;
@@ -496,6 +509,8 @@ extern "C" quaff_status_t quaff_lora_down(const quaff_bf16* X, int64_t ldx, int 
 
 extern "C" uint64_t quaff_debug_launch_count(void) { return g_launch_count; }
 
+extern "C" void quaff_debug_force_fwd_tile(int tile_n) { g_force_fwd_tile = tile_n; }
+
 extern "C" void quaff_debug_time_gemm(int which, void* start_event, void* stop_event) {
     if (which < 0 || which > 1) return;
     g_time_start[which] = (cudaEvent_t)start_event;
@@ -554,45 +569,62 @@ extern "C" quaff_status_t quaff_qlinear_fwd(int M, int K, int N, const int8_t* X
     cudaStream_t st = (cudaStream_t)stream;
     const int rp = pad16(r);
     constexpr int CTAS = 2;
-    // Eq. 2 alone (no outlier set, no LoRA) takes 256-column tiles.  With the two short contractions: 192-column
-    // tiles with the short accumulators in rounds of 64 columns (fwd192.cuh), or 128-column tiles with all three
-    // accumulators resident in TMEM.  A tcgen05.mma costs about 60 + N/2 clocks, so the wide tile is cheaper per
-    // column, but it carries six extra ring stages and three more epilogue hand-shakes: measured, a wave of
-    // 192-column tiles takes 1.47x (K < 4096) resp. 1.27x (K >= 4096) as long as a wave of 128-column tiles.  The
-    // rounds need an outlier round to be one k-block (nOp <= 128).
+    // Eq. 2 alone (no outlier set, no LoRA) takes 256-column tiles.  With the two short contractions there are
+    // three kernels: 128-column tiles with all three accumulators resident in TMEM (umma_gemm.cuh), 192-column
+    // tiles with the short accumulators in rounds of 64 columns (fwd192.cuh), 256-column tiles with a single main
+    // accumulator that the epilogue copies out at once and rounds of 128 columns (fwd256.cuh).  A tcgen05.mma
+    // costs about 60 + N/2 clocks, so the wide tiles are cheaper per column; each kernel has its own overhead per
+    // tile (ring stages of the rounds, hand-shakes, the wait for the accumulator).  The host takes the variant with
+    // the smallest  waves x time per tile  (cost model above).  The rounds need an outlier round to be one k-block
+    // (nOp <= 128).
     const int tiles_m2 = ceil_div(M, 2 * kTileM), pairs = kPlanSMs / 2;
-    const double waves128 = ceil_div(tiles_m2 * ceil_div(N, 128), pairs);
-    const double waves192 = ceil_div(tiles_m2 * ceil_div(N, kF192TN), pairs) * (K >= 4096 ? 1.27 : 1.47);
-    if ((nOp > 0 || r > 0) && nOp <= 128 && waves192 < waves128) {
+    int wide = 0;     // 0: 128-column tiles, else the tile width of the wide kernel
+    if ((nOp > 0 || r > 0) && nOp <= 128) {
+        const double nmma = ceil_div(K, 32);
+        double best = 0.0;
+        for (int i = 0; i < 3; ++i) {
+            const double tile = fmax(nmma * kFwdMmaClk[i] + kFwdTileOvh[i], kFwdTileMin[i]);
+            const double cost = (double)ceil_div(tiles_m2 * ceil_div(N, kFwdWidths[i]), pairs) * tile;
+            if (i == 0 || cost < best) { best = cost; wide = i == 0 ? 0 : kFwdWidths[i]; }
+        }
+        if (g_force_fwd_tile == 128) wide = 0;
+        if (g_force_fwd_tile == 192 || g_force_fwd_tile == 256) wide = g_force_fwd_tile;
+    }
+    if (wide) {
+        const int WTN = wide, WR = wide == 256 ? kF256Round : kF192Round;
         Fwd192Params q;
         memset(&q, 0, sizeof(q));
         quaff_status_t rc;
         if ((rc = make_tmap_2d(&q.map_xq, Xq, 1, M, K, ldxq, kTileM, 128)) != QUAFF_OK) return rc;
-        if ((rc = make_tmap_2d(&q.map_wq, Wq, 1, N, K, ldwq_main, kF192TN / 2, 128)) != QUAFF_OK) return rc;
+        if ((rc = make_tmap_2d(&q.map_wq, Wq, 1, N, K, ldwq_main, WTN / 2, 128)) != QUAFF_OK) return rc;
         q.nblk = ceil_div(K, 128);
         q.nmma_last = ceil_div(K - (q.nblk - 1) * 128, 32);
         if (nOp > 0) {
             if ((rc = make_tmap_2d(&q.map_xo, xq_O, 1, M, nOp, ldxo, kTileM, 128)) != QUAFF_OK) return rc;
-            if ((rc = make_tmap_2d(&q.map_wo, wq_O, 1, N, nOp, ldwq, kF192Round / 2, 128)) != QUAFF_OK) return rc;
+            if ((rc = make_tmap_2d(&q.map_wo, wq_O, 1, N, nOp, ldwq, WR / 2, 128)) != QUAFF_OK) return rc;
             q.nmma_o = nOp / 32;
         }
         if (r > 0) {
             if (!have_T && (rc = lora_down(X, ldx, M, K, A, r, T_out, w, ws, status_opt, st)) != QUAFF_OK) return rc;
-            uint16_t* Bt = reinterpret_cast<uint16_t*>(reinterpret_cast<unsigned char*>(ws) + w.off_bt);
-            launch_pdl(transpose_pad_kernel, dim3(ceil_div(N * rp, 256)), dim3(256), 0, st, 1, B, r, N, Bt, rp);   // Bt[n][j] = B[j][n]
-            if ((rc = launch_status()) != QUAFF_OK) return rc;
             if ((rc = make_tmap_2d(&q.map_t, T_out, 2, M, r, r, kTileM, 64)) != QUAFF_OK) return rc;
-            if ((rc = make_tmap_2d(&q.map_bt, Bt, 2, N, rp, rp, kF192Round / 2, 64)) != QUAFF_OK) return rc;
+            if (wide == 256) {   // B [r][N] is read in place as an MN-major operand (rows = contraction)
+                if ((rc = make_tmap_2d(&q.map_bt, B, 2, r, N, N, rp, 64)) != QUAFF_OK) return rc;
+            } else {             // rounds of 64 columns, 32 per CTA: K-major copy Bt[n][j] = B[j][n]
+                uint16_t* Bt = reinterpret_cast<uint16_t*>(reinterpret_cast<unsigned char*>(ws) + w.off_bt);
+                launch_pdl(transpose_pad_kernel, dim3(ceil_div(N * rp, 256)), dim3(256), 0, st, 1, B, r, N, Bt, rp);
+                if ((rc = launch_status()) != QUAFF_OK) return rc;
+                if ((rc = make_tmap_2d(&q.map_bt, Bt, 2, N, rp, rp, WR / 2, 64)) != QUAFF_OK) return rc;
+            }
             q.nmma_l = rp / 16;
         }
         q.M = M; q.N = N;
-        q.tiles_m = ceil_div(M, 2 * kTileM); q.tiles_n = ceil_div(N, kF192TN);
+        q.tiles_m = ceil_div(M, 2 * kTileM); q.tiles_n = ceil_div(N, WTN);
         q.band_m = band_rows(q.tiles_m, q.tiles_n, 2 * kTileM, (size_t)K);
         q.status = status_opt;
         q.dx = dx; q.dW = dW; q.dw_O = dw_O; q.lora_scale = lora_scale;
         q.Y = Y; q.ldy = ldy; q.y_f32 = (y_dtype == QUAFF_F32);
         q.dbg_main = dbg_acc_main; q.dbg_out = dbg_acc_out;
-        return launch_fwd192(q, st);
+        return launch_fwd_wide(wide == 256 ? 1 : 0, q, st);
     }
     const int TN = (nOp == 0 && r == 0) ? 256 : 128;
 

@@ -154,6 +154,26 @@ FWD_SHAPES = [(1, 128, 16, 0, 0), (128, 128, 128, 32, 16), (200, 320, 136, 5, 8)
 @pytest.mark.parametrize("M,K,N,nO,r", FWD_SHAPES)
 @pytest.mark.parametrize("y_f32", [True, False])
 def test_qlinear_fwd(Q, M, K, N, nO, r, y_f32):
+    _check_fwd(Q, M, K, N, nO, r, y_f32)
+
+
+# Each of the three forward kernels (128-, 192-, 256-column tiles) on the same shapes: several tiles per CTA pair
+# (96 to 200 tiles on 74 pairs), ragged M and N, LoRA only, outliers only, a single main k-block, one tiny tile.
+FORCED_SHAPES = [(2048, 256, 3072, 33, 64), (2040, 384, 3016, 0, 32), (2048, 256, 3061, 7, 0), (2048, 128, 6400, 40, 8),
+                 (300, 1024, 392, 100, 16), (1, 128, 16, 5, 8), (520, 3072, 1032, 32, 16)]
+
+
+@pytest.mark.parametrize("M,K,N,nO,r", FORCED_SHAPES)
+@pytest.mark.parametrize("tile_n", [128, 192, 256])
+def test_qlinear_fwd_each_tile_width(Q, M, K, N, nO, r, tile_n):
+    Q.quaff_debug_force_fwd_tile(tile_n)
+    try:
+        _check_fwd(Q, M, K, N, nO, r, (M + tile_n) % 2 == 0)
+    finally:
+        Q.quaff_debug_force_fwd_tile(0)
+
+
+def _check_fwd(Q, M, K, N, nO, r, y_f32):
     import torch
     O, X, Wt, A, B, _ = _mk_inputs(500 + M + N, M, K, N, nO, r)
     Wq, dW, W_O, wmax, s, Xq, xqo, dx, wq, dw = _oracle_state(O, X, Wt)
