@@ -418,6 +418,7 @@ constexpr int kFwdWidths[3] = {128, 192, 256};
 constexpr double kFwdMmaClk[3] = {125.0, 157.0, 190.0};
 constexpr double kFwdTileOvh[3] = {4100.0, 1500.0, 5000.0};
 constexpr double kFwdTileMin[3] = {10900.0, 22500.0, 18700.0};
+constexpr double kFwdTransposeClk = 7000.0;
 
 struct FwdWorkspace { size_t off_bt, off_at, off_part, total; };
 static FwdWorkspace fwd_workspace(int M, int K, int N, int r) {
@@ -584,7 +585,8 @@ extern "C" quaff_status_t quaff_qlinear_fwd(int M, int K, int N, const int8_t* X
         double best = 0.0;
         for (int i = 0; i < 3; ++i) {
             const double tile = fmax(nmma * kFwdMmaClk[i] + kFwdTileOvh[i], kFwdTileMin[i]);
-            const double cost = (double)ceil_div(tiles_m2 * ceil_div(N, kFwdWidths[i]), pairs) * tile;
+            // (the 192-column kernel wants LoRA B transposed: one more small kernel in front of it)
+            const double cost = (double)ceil_div(tiles_m2 * ceil_div(N, kFwdWidths[i]), pairs) * tile + ((i == 1 && r > 0) ? kFwdTransposeClk : 0.0);
             if (i == 0 || cost < best) { best = cost; wide = i == 0 ? 0 : kFwdWidths[i]; }
         }
         if (g_force_fwd_tile == 128) wide = 0;
