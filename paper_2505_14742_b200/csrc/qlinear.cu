@@ -710,8 +710,17 @@ extern "C" quaff_status_t quaff_qlinear_bwd(int M, int K, int N, const quaff_bf1
     cudaStream_t s_db = ss ? ss->s[1] : st;        // dB
     bool forked0 = false, forked1 = false;
 
+    // Launch order = the order in which the block scheduler hands out SM slots while everything below runs at once:
+    // the chain the grad-input GEMM waits for longest (G) first, the bulk dequantization last.  The side streams fork
+    // off before any of it, so that they depend on nothing launched here.
+    if (ss && want_dAB && !(forked1 = fork_to(ss, 1, st))) return QUAFF_ERR_CUDA;
+    if (ss && dX && !(forked0 = fork_to(ss, 0, st))) return QUAFF_ERR_CUDA;
+    if (r > 0) {   // G = bf16(lora_scale * dY B^T): B [r][N] is already K-major for this contraction over N
+        if ((rc = skinny_gemm(0, dY, lddy, B, N, M, N, r, part, status_opt, st, &S)) != QUAFF_OK) return rc;
+        launch_pdl(reduce_parts_bf16_kernel, dim3(ceil_div(M * r / 8, 256)), dim3(256), 0, st, 1, part, S, M, r, lora_scale, G);
+        if ((rc = launch_status()) != QUAFF_OK) return rc;
+    }
     if (want_dAB) {   // dB^T = dY^T T: the contraction runs over the tokens, the slow axis of dY and T: MN-major operands
-        if (ss && !(forked1 = fork_to(ss, 1, st))) return QUAFF_ERR_CUDA;
         if ((rc = skinny_gemm(1, dY, lddy, T, r, N, M, r, part_b, status_opt, s_db, &S)) != QUAFF_OK) return rc;
         launch_pdl(reduce_parts_kernel, dim3(ceil_div(N * r / 4, 256)), dim3(256), 0, s_db, 1, part_b, S, N, r, lora_scale, 1, accumulate, dB);
         if ((rc = launch_status()) != QUAFF_OK) return rc;
@@ -720,15 +729,9 @@ extern "C" quaff_status_t quaff_qlinear_bwd(int M, int K, int N, const quaff_bf1
     const int TN = w.tile_n, Kpad = w.Kpad;
     const int Kext = nOp > 0 ? Kpad + 2 * nOp : K;
     if (dX) {
-        if (ss && !(forked0 = fork_to(ss, 0, st))) return QUAFF_ERR_CUDA;
         const int chunks = (Kpad + 2 * nOp) / 16;
         launch_pdl(dequant_weight_kernel, dim3(N, ceil_div(chunks, 256)), dim3(256), 0, s_deq, 1, Wq, ldwq_main, dW, wq_O, ldwq, dw_O, O_idx,
                    nO, nOp, K, Kpad, Wd, w.ldwd);
-        if ((rc = launch_status()) != QUAFF_OK) return rc;
-    }
-    if (r > 0) {   // G = bf16(lora_scale * dY B^T): B [r][N] is already K-major for this contraction over N
-        if ((rc = skinny_gemm(0, dY, lddy, B, N, M, N, r, part, status_opt, st, &S)) != QUAFF_OK) return rc;
-        launch_pdl(reduce_parts_bf16_kernel, dim3(ceil_div(M * r / 8, 256)), dim3(256), 0, st, 1, part, S, M, r, lora_scale, G);
         if ((rc = launch_status()) != QUAFF_OK) return rc;
     }
     if (dX) {
