@@ -223,6 +223,11 @@ __global__ void __launch_bounds__(kF256Threads, 1) fwd256_kernel(const __grid_co
         float* scale_w = scales + (warp - 2) * 128;      // [round][32]
         float* scale_o = scale_w + 64;
 
+        // A lane stores its own row: 32 rows per store instruction, so the LSU spends one transaction per row whatever
+        // the width.  Where Y's base and row pitch allow it, a store is 32 bytes (a whole sector) instead of 16:
+        // 8 f32 columns, or 16 bf16 columns (the even group of 8 waits in `carry` for the odd one).
+        const bool wide = ((reinterpret_cast<uintptr_t>(p.Y) | (uintptr_t)(p.ldy * (p.y_f32 ? 4 : 2))) & 31u) == 0;
+        uint4 carry = make_uint4(0u, 0u, 0u, 0u);
         // y = dx (acc dW + acc_o dw_O) + lora_scale acc_l for 8 consecutive columns of row m (h = which 8 of the warp's 32)
         auto finish8 = [&](int m, float dxm, int nc, int h, int jj, const uint32_t (&a0)[8], const uint32_t (&a1)[8], const uint32_t (&a2)[8]) {
             float y[8];
@@ -244,7 +249,10 @@ __global__ void __launch_bounds__(kF256Threads, 1) fwd256_kernel(const __grid_co
             {
                 if (p.y_f32) {
                     float* out = reinterpret_cast<float*>(p.Y) + (int64_t)m * p.ldy + nc;
-                    if (full && (p.ldy % 4 == 0)) {
+                    if (full && wide) {
+                        st_global_v8(out, __float_as_uint(y[0]), __float_as_uint(y[1]), __float_as_uint(y[2]), __float_as_uint(y[3]),
+                                     __float_as_uint(y[4]), __float_as_uint(y[5]), __float_as_uint(y[6]), __float_as_uint(y[7]));
+                    } else if (full && (p.ldy % 4 == 0)) {
                         *reinterpret_cast<float4*>(out) = make_float4(y[0], y[1], y[2], y[3]);
                         *reinterpret_cast<float4*>(out + 4) = make_float4(y[4], y[5], y[6], y[7]);
                     } else {
@@ -252,7 +260,12 @@ __global__ void __launch_bounds__(kF256Threads, 1) fwd256_kernel(const __grid_co
                     }
                 } else {
                     uint16_t* out = reinterpret_cast<uint16_t*>(p.Y) + (int64_t)m * p.ldy + nc;
-                    if (full && (p.ldy % 8 == 0)) {
+                    if (wide && !(h & 1) && nc + 16 <= p.N) {          // stored together with the next group
+                        carry = make_uint4(pack_bf16x2(y[0], y[1]), pack_bf16x2(y[2], y[3]), pack_bf16x2(y[4], y[5]), pack_bf16x2(y[6], y[7]));
+                    } else if (wide && (h & 1) && full) {              // (the even group is in `carry`: nc - 8 + 16 <= N)
+                        st_global_v8(out - 8, carry.x, carry.y, carry.z, carry.w, pack_bf16x2(y[0], y[1]), pack_bf16x2(y[2], y[3]),
+                                     pack_bf16x2(y[4], y[5]), pack_bf16x2(y[6], y[7]));
+                    } else if (full && (p.ldy % 8 == 0)) {
                         *reinterpret_cast<uint4*>(out) = make_uint4(pack_bf16x2(y[0], y[1]), pack_bf16x2(y[2], y[3]),
                                                                     pack_bf16x2(y[4], y[5]), pack_bf16x2(y[6], y[7]));
                     } else {
