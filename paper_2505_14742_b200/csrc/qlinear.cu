@@ -251,7 +251,7 @@ __global__ void reduce_parts_kernel(const float* __restrict__ part, int S, int C
 // Dequantized weight for the grad-input GEMM, in the stored orientation [N][.] (the contraction index n
 // is the row, so the GEMM reads it as an MN-major operand; nothing is transposed):
 //   columns 0..K-1              : Wd[n][k]          = bf16(Wq[n][k]   * dW[n])
-//   columns K..Kpad-1           : 0   (Kpad = K rounded up to the tile width, so the columns below start a tile)
+//   columns K..Kpad-1           : 0   (Kpad = K rounded up to 32: the epilogue tells dX from P columns per chunk)
 //   columns Kpad..Kpad+nOp-1    : Wd[n][Kpad+i]     = bf16(Wq[n][O_i] * dW[n])   (i < nO, else 0)
 //   columns Kpad+nOp..Kpad+2nOp : Wd[n][Kpad+nOp+i] = bf16(wq_O[n][i] * dw_O[n])
 // One thread converts 16 consecutive columns of one row (one 128-bit load of codes, two 128-bit stores).
@@ -432,22 +432,23 @@ static FwdWorkspace fwd_workspace(int M, int K, int N, int r) {
     return w;
 }
 
-// Output-column tile of the grad-input GEMM.  A tcgen05.mma of a CTA pair costs about 60 + N/2 clocks
-// (measured: N = 128: 125, 192: 165, 256: 190), so wide tiles are cheaper per column, while narrow ones
-// leave a smaller ragged last wave.  Cost model: waves on the CTA pairs x cost of one MMA of that width.
+// Output-column tile of the grad-input GEMM: 128, 192 or 256.  A tcgen05.mma of a CTA pair costs about 60 + N/2
+// clocks (measured: N = 128: 125, 192: 165, 256: 190), so wide tiles are cheaper per column, while the width also
+// decides how full the last wave is.  Cost model: waves on the CTA pairs x cost of one MMA of that width; among equals
+// the wider tile (fewer tiles, fewer epilogues).  (The kernel takes any multiple of 16, but widths that are not a
+// multiple of 64 run far below this model - measured: 176 columns 208 clocks per MMA, 240 columns 215 - so they are
+// not candidates.)
+static int round_up32(int k) { return (k + 31) / 32 * 32; }
 static int bwd_tile_n(int M, int K, int nOp) {
     const int units = kPlanSMs / 2;
     const int tm = ceil_div(M, 2 * kTileM);
-    const int widths[3] = {256, 192, 128};
-    const double mma_cost[3] = {190.0, 165.0, 125.0};
+    const int kext = nOp > 0 ? round_up32(K) + 2 * nOp : K;
     int best = 256;
     double best_cost = 0.0;
-    for (int i = 0; i < 3; ++i) {
-        const int tn = widths[i];
-        const int kpad = ceil_div(K, tn) * tn;
-        const int tiles = tm * ceil_div(kpad + 2 * nOp, tn);
-        const double cost = (double)ceil_div(tiles, units) * mma_cost[i];
-        if (i == 0 || cost < best_cost) { best = tn; best_cost = cost; }
+    for (int tn = 256; tn >= 128; tn -= 64) {
+        const int tiles = tm * ceil_div(kext, tn);
+        const double cost = (double)ceil_div(tiles, units) * (60.0 + 0.5 * tn);
+        if (tn == 256 || cost < best_cost) { best = tn; best_cost = cost; }
     }
     return best;
 }
@@ -455,14 +456,14 @@ static int bwd_tile_n(int M, int K, int nOp) {
 struct BwdWorkspace {
     size_t off_wd, off_g, off_p, off_part, off_part_a, off_part_b, total;
     int tile_n;       // output-column tile of the grad-input GEMM
-    int Kpad;         // K rounded up to tile_n
+    int Kpad;         // K rounded up to 32: where the outlier columns start
     int64_t ldwd;     // row pitch of Wd in elements
 };
 
 static BwdWorkspace bwd_workspace(int M, int K, int N, int nOp, int r) {
     BwdWorkspace w;
     w.tile_n = bwd_tile_n(M, K, nOp);
-    w.Kpad = ceil_div(K, w.tile_n) * w.tile_n;
+    w.Kpad = round_up32(K);
     w.ldwd = (int64_t)w.Kpad + 2 * nOp;
     size_t off = 0;
     w.off_wd = off;   off += round_up((size_t)N * (size_t)w.ldwd * 2, 256);
@@ -756,7 +757,8 @@ extern "C" quaff_status_t quaff_qlinear_bwd(int M, int K, int N, const quaff_bf1
         }
         p.nphases = np;
         p.M = M;
-        // columns [0,K) -> dX; the outlier partial products start at the next tile boundary Kpad
+        // columns [0,K) -> dX; the outlier partial products start at Kpad (K rounded up to 32), inside whatever tile that is:
+        // the LoRA phase of that tile adds nothing to them (rows of A beyond K read as zeros)
         p.n_split = K;
         p.p_col0 = Kpad;
         p.N = Kext;
@@ -765,7 +767,8 @@ extern "C" quaff_status_t quaff_qlinear_bwd(int M, int K, int N, const quaff_bf1
         p.band_m = band_rows(p.tiles_m, p.tiles_n, kTileM * CTAS, (size_t)N * 2);
         p.status = status_opt;
         p.dX = dX; p.lddx = lddx; p.P = P; p.ldp = 2 * nOp;
-        rc = TN == 256 ? launch_gemm<EPI_BWD, CTAS, 256>(p, st) : TN == 192 ? launch_gemm<EPI_BWD, CTAS, 192>(p, st) : launch_gemm<EPI_BWD, CTAS, 128>(p, st);
+        p.tile_n = TN;      // the 256-column instance serves every width above 128
+        rc = TN > 128 ? launch_gemm<EPI_BWD, CTAS, 256>(p, st) : launch_gemm<EPI_BWD, CTAS, 128>(p, st);
         if (rc != QUAFF_OK) return rc;
     }
     if (want_dAB) {   // dA = X^T G (MN-major operands), beside the outlier fix-up

@@ -95,6 +95,7 @@ struct GemmParams {
     int M, N;            // output extent (rows, columns)
     int tiles_m, tiles_n;
     int band_m;          // row tiles per band of the tile order (tiles_m: one band)
+    int tile_n;          // EPI_BWD: output columns per tile, any multiple of 16 up to TN (0: TN); other epilogues: TN
     int32_t* status;
     // forward epilogue (Eq. 9 + LoRA)
     const float* dx;     // [M]
@@ -133,7 +134,7 @@ struct GemmSmem {
 template <int EPI, int CTAS, int TN>
 struct GemmCfg {
     // B region of a stage, per CTA: whole boxes of 64 output columns (an MN-major operand is loaded box by box;
-    // with TN = 192 a CTA of a pair owns 96 columns, one box and a half)
+    // the grad-input GEMM may use part of the last box)
     static constexpr int kBBytes = ((TN / CTAS + 63) / 64) * 64 * 128;
     static constexpr int kStageBytes = kABytes + kBBytes;
     static constexpr int kScaleBytes = (EPI == EPI_FWD) ? 2 * 2 * TN * 4 : 0;   // [2 buffers][dW | dw_O][TN]
@@ -155,13 +156,39 @@ __device__ __forceinline__ uint64_t make_desc(uint32_t lo, uint32_t hi) {
     return (static_cast<uint64_t>(hi) << 32) | lo;
 }
 
+// Grad-input epilogue: W accumulator columns of row m, starting at column nc.  Columns below n_split go to dX (bf16);
+// columns from p_col0 on (a multiple of 32) are outlier partial products and go to P (f32); in between: padding.
+template <int W>
+__device__ __forceinline__ void bwd_store_chunk(const GemmParams& p, int m, int nc, const uint32_t (&r0)[W]) {
+    if (nc < p.p_col0) {
+        uint16_t* out = p.dX + (int64_t)m * p.lddx + nc;
+        if (nc + W <= p.n_split && (p.lddx % 8 == 0)) {
+#pragma unroll
+            for (int j = 0; j < W; j += 8)
+                *reinterpret_cast<uint4*>(out + j) =
+                    make_uint4(pack_bf16x2(__uint_as_float(r0[j]), __uint_as_float(r0[j + 1])),
+                               pack_bf16x2(__uint_as_float(r0[j + 2]), __uint_as_float(r0[j + 3])),
+                               pack_bf16x2(__uint_as_float(r0[j + 4]), __uint_as_float(r0[j + 5])),
+                               pack_bf16x2(__uint_as_float(r0[j + 6]), __uint_as_float(r0[j + 7])));
+        } else {
+            for (int j = 0; j < W; ++j) if (nc + j < p.n_split) out[j] = (uint16_t)f32_to_bf16_bits(__uint_as_float(r0[j]));
+        }
+    } else {
+        float* out = p.P + (int64_t)m * p.ldp + (nc - p.p_col0);
+        for (int j = 0; j < W; ++j) if (nc + j < p.N) out[j] = __uint_as_float(r0[j]);
+    }
+}
+
 template <int EPI, int CTAS, int TN>
 __global__ void __launch_bounds__(kGemmThreads, 1) umma_gemm_kernel(const __grid_constant__ GemmParams p) {
     using Cfg = GemmCfg<EPI, CTAS, TN>;
     constexpr int kStages = Cfg::kStages;
     constexpr int kStageBytes = Cfg::kStageBytes;
     static_assert(CTAS == 1 || CTAS == 2, "one CTA or a CTA pair");
-    static_assert(TN == 128 || TN == 256 || (TN == 192 && EPI == EPI_BWD && CTAS == 2), "output-column tile");   // TN > 128: slot 0 only (no room for auxiliary accumulators)
+    static_assert(TN == 128 || TN == 256, "output-column tile");   // TN = 256: slot 0 only (no room for auxiliary accumulators)
+    // The grad-input epilogue takes its tile width at run time (p.tile_n <= TN): the two buffers of its accumulator
+    // then sit at columns 0 and TN.
+    constexpr int kAccStride = TN;
 
     extern __shared__ unsigned char smem_dyn[];
     const uint32_t raw = smem_u32(smem_dyn);
@@ -266,7 +293,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) umma_gemm_kernel(const __grid
                 for (int i = 0; i < p.nphases && ok; ++i) {
                     const GemmPhase& ph = p.ph[i];
                     if (tn < ph.tn_limit) {
-                        const uint32_t acc = tmem_base + (ph.acc_slot == 0 ? (uint32_t)((t & 1) * TN) : (uint32_t)((ph.acc_slot + 1) * TN));
+                        const uint32_t acc = tmem_base + (ph.acc_slot == 0 ? (uint32_t)((t & 1) * kAccStride) : (uint32_t)((ph.acc_slot + 1) * TN));
                         const int nblk = ph.nblk;
                         const int nmma_last = ph.nmma_last;
                         const bool i8 = ph.is_i8 != 0;
@@ -318,7 +345,8 @@ __global__ void __launch_bounds__(kGemmThreads, 1) umma_gemm_kernel(const __grid
         for (int tile = unit; tile < ntiles && ok; tile += nunits, ++t) {
             int tm, tn;
             tile_coords(tile, p.tiles_m, p.tiles_n, p.band_m, tm, tn);
-            const int m0 = tm * (kTileM * CTAS) + (int)rank * kTileM, n0 = tn * TN;
+            const int tn_cols = (EPI == EPI_BWD && p.tile_n) ? p.tile_n : TN;
+            const int m0 = tm * (kTileM * CTAS) + (int)rank * kTileM, n0 = tn * tn_cols;
             const int buf = t & 1;
             float* scale_w = scales + buf * 2 * TN;
             float* scale_o = scale_w + TN;
@@ -348,6 +376,28 @@ __global__ void __launch_bounds__(kGemmThreads, 1) umma_gemm_kernel(const __grid
                             if (c * 32 + j < p.part_cols)
                                 *reinterpret_cast<float4*>(out + j) = make_float4(__uint_as_float(r0[j]), __uint_as_float(r0[j + 1]),
                                                                                  __uint_as_float(r0[j + 2]), __uint_as_float(r0[j + 3]));
+                    }
+                }
+            } else if (EPI == EPI_BWD) {
+                if ((tn_cols & 31) == 0) {
+#pragma unroll 1
+                    for (int c = 0; c < tn_cols; c += 32) {
+                        const int nc = n0 + c;
+                        if (nc >= p.N) break;            // uniform across the warp
+                        uint32_t r0[32];
+                        tmem_ld_32x32(lane_addr + (uint32_t)(buf * kAccStride + c), r0);
+                        tmem_ld_wait();
+                        if (m < p.M) bwd_store_chunk<32>(p, m, nc, r0);
+                    }
+                } else {                                 // a tile width that is a multiple of 16 only
+#pragma unroll 1
+                    for (int c = 0; c < tn_cols; c += 16) {
+                        const int nc = n0 + c;
+                        if (nc >= p.N) break;
+                        uint32_t r0[16];
+                        tmem_ld_32x16(lane_addr + (uint32_t)(buf * kAccStride + c), r0);
+                        tmem_ld_wait();
+                        if (m < p.M) bwd_store_chunk<16>(p, m, nc, r0);
                     }
                 }
             } else {
@@ -400,27 +450,6 @@ __global__ void __launch_bounds__(kGemmThreads, 1) umma_gemm_kernel(const __grid
                             if (p.dbg_out) {
                                 int32_t* d = p.dbg_out + (int64_t)m * p.N + nc;
                                 for (int j = 0; j < 32; ++j) if (nc + j < p.N) d[j] = p.has_outlier ? (int32_t)r1[j] : 0;
-                            }
-                        }
-                    } else {
-                        tmem_ld_wait();
-                        if (m < p.M) {
-                            if (nc < p.p_col0) {
-                                uint16_t* out = p.dX + (int64_t)m * p.lddx + nc;
-                                if (nc + 32 <= p.n_split && (p.lddx % 8 == 0)) {
-#pragma unroll
-                                    for (int j = 0; j < 32; j += 8)
-                                        *reinterpret_cast<uint4*>(out + j) =
-                                            make_uint4(pack_bf16x2(__uint_as_float(r0[j]), __uint_as_float(r0[j + 1])),
-                                                       pack_bf16x2(__uint_as_float(r0[j + 2]), __uint_as_float(r0[j + 3])),
-                                                       pack_bf16x2(__uint_as_float(r0[j + 4]), __uint_as_float(r0[j + 5])),
-                                                       pack_bf16x2(__uint_as_float(r0[j + 6]), __uint_as_float(r0[j + 7])));
-                                } else {
-                                    for (int j = 0; j < 32; ++j) if (nc + j < p.n_split) out[j] = (uint16_t)f32_to_bf16_bits(__uint_as_float(r0[j]));
-                                }
-                            } else {
-                                float* out = p.P + (int64_t)m * p.ldp + (nc - p.p_col0);
-                                for (int j = 0; j < 32; ++j) if (nc + j < p.N) out[j] = __uint_as_float(r0[j]);
                             }
                         }
                     }
