@@ -45,7 +45,8 @@ constexpr int kF192Stages = (kSmemLimit - kF192Fixed) / kF192StageBytes < kMaxSt
 constexpr size_t kF192SmemBytes = (size_t)kF192Fixed + (size_t)kF192Stages * kF192StageBytes;
 static_assert(sizeof(Fwd192Smem) <= 256, "barrier block");
 
-struct Fwd192Params {
+// Parameters of the wide forward kernels (this one and fwd256.cuh, which states its own box sizes).
+struct FwdWideParams {
     CUtensorMap map_xq, map_wq;      // main: Xq [M][K] (box 128 rows), Wq [N][K] (box 96 rows), 128-byte boxes
     CUtensorMap map_xo, map_wo;      // outlier: xq_O [M][nOp] (box 128 rows), wq_O [N][nOp] (box 32 rows)
     CUtensorMap map_t, map_bt;       // LoRA: T [M][r] bf16 (box 128 rows), B^T [N][rp] bf16 (box 32 rows), 64-element boxes
@@ -86,7 +87,7 @@ __device__ __forceinline__ void for_each_item(int unit, int nunits, int ntiles, 
     }
 }
 
-__global__ void __launch_bounds__(kF192Threads, 1) fwd192_kernel(const __grid_constant__ Fwd192Params p) {
+__global__ void __launch_bounds__(kF192Threads, 1) fwd192_kernel(const __grid_constant__ FwdWideParams p) {
     constexpr int TN = kF192TN;
     constexpr int kStages = kF192Stages;
     constexpr int kStageBytes = kF192StageBytes;

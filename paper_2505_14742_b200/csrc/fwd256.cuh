@@ -64,9 +64,9 @@ __device__ __forceinline__ void for_each_item256(int unit, int nunits, int ntile
     if (prev >= 0) aux_fn(t - 1, prev, 1);
 }
 
-// Parameters: those of the 192-column kernel (Fwd192Params) with the boxes of map_wq 128 rows and of map_wo 64 rows high;
+// Parameters: FwdWideParams with the boxes of map_wq 128 rows and of map_wo 64 rows high;
 // map_bt is LoRA B [r][N] itself, boxes of rp contraction rows x 64 columns.
-__global__ void __launch_bounds__(kF256Threads, 1) fwd256_kernel(const __grid_constant__ Fwd192Params p) {
+__global__ void __launch_bounds__(kF256Threads, 1) fwd256_kernel(const __grid_constant__ FwdWideParams p) {
     constexpr int TN = kF256TN;
     constexpr int kStages = kF256Stages;
     constexpr int kStageBytes = kF256StageBytes;

@@ -140,10 +140,10 @@ static quaff_status_t launch_gemm(const GemmParams& p, cudaStream_t st) {
 }
 
 // The wide forward kernels (fwd192.cuh, fwd256.cuh): which = 0 / 1
-static quaff_status_t launch_fwd_wide(int which, const Fwd192Params& p, cudaStream_t st) {
+static quaff_status_t launch_fwd_wide(int which, const FwdWideParams& p, cudaStream_t st) {
     static bool configured[2][64] = {{false}};
     static int units_of[2][64] = {{0}};
-    void (*const kernel)(const Fwd192Params) = which ? fwd256_kernel : fwd192_kernel;
+    void (*const kernel)(const FwdWideParams) = which ? fwd256_kernel : fwd192_kernel;
     const int threads = which ? kF256Threads : kF192Threads;
     const size_t smem = which ? kF256SmemBytes : kF192SmemBytes;
     int dev = 0;
@@ -595,7 +595,7 @@ extern "C" quaff_status_t quaff_qlinear_fwd(int M, int K, int N, const int8_t* X
     }
     if (wide) {
         const int WTN = wide, WR = wide == 256 ? kF256Round : kF192Round;
-        Fwd192Params q;
+        FwdWideParams q;
         memset(&q, 0, sizeof(q));
         quaff_status_t rc;
         if ((rc = make_tmap_2d(&q.map_xq, Xq, 1, M, K, ldxq, kTileM, 128)) != QUAFF_OK) return rc;
