@@ -224,13 +224,10 @@ __global__ void __launch_bounds__(kF256Threads, 1) fwd256_kernel(const __grid_co
         float* scale_o = scale_w + 64;
 
         // A lane stores its own row: 32 rows per store instruction, so the LSU spends one transaction per row whatever
-        // the width.  Where Y's base and row pitch allow it, a store is 32 bytes (a whole sector) instead of 16:
-        // 8 f32 columns, or 16 bf16 columns (the even group of 8 waits in `carry` for the odd one).
+        // the width.  Where Y's base and row pitch allow it, a store is 32 bytes (a whole sector) instead of 16.
         const bool wide = ((reinterpret_cast<uintptr_t>(p.Y) | (uintptr_t)(p.ldy * (p.y_f32 ? 4 : 2))) & 31u) == 0;
-        uint4 carry = make_uint4(0u, 0u, 0u, 0u);
-        // y = dx (acc dW + acc_o dw_O) + lora_scale acc_l for 8 consecutive columns of row m (h = which 8 of the warp's 32)
-        auto finish8 = [&](int m, float dxm, int nc, int h, int jj, const uint32_t (&a0)[8], const uint32_t (&a1)[8], const uint32_t (&a2)[8]) {
-            float y[8];
+        // y = dx (acc dW + acc_o dw_O) + lora_scale acc_l for 8 consecutive columns (h = which 8 of the warp's 32 in round jj)
+        auto compute8 = [&](float dxm, int h, int jj, const uint32_t (&a0)[8], const uint32_t (&a1)[8], const uint32_t (&a2)[8], float (&y)[8]) {
 #pragma unroll
             for (int i = 0; i < 8; i += 4) {
                 const float4 a = *reinterpret_cast<const float4*>(scale_w + jj * 32 + 8 * h + i);
@@ -245,40 +242,44 @@ __global__ void __launch_bounds__(kF256Threads, 1) fwd256_kernel(const __grid_co
                     y[i + u] = v;
                 }
             }
-            const bool full = (nc + 8 <= p.N);
-            {
-                if (p.y_f32) {
-                    float* out = reinterpret_cast<float*>(p.Y) + (int64_t)m * p.ldy + nc;
-                    if (full && wide) {
-                        st_global_v8(out, __float_as_uint(y[0]), __float_as_uint(y[1]), __float_as_uint(y[2]), __float_as_uint(y[3]),
-                                     __float_as_uint(y[4]), __float_as_uint(y[5]), __float_as_uint(y[6]), __float_as_uint(y[7]));
-                    } else if (full && (p.ldy % 4 == 0)) {
-                        *reinterpret_cast<float4*>(out) = make_float4(y[0], y[1], y[2], y[3]);
-                        *reinterpret_cast<float4*>(out + 4) = make_float4(y[4], y[5], y[6], y[7]);
-                    } else {
-                        for (int i = 0; i < 8; ++i) if (nc + i < p.N) out[i] = y[i];
-                    }
-                } else {
-                    uint16_t* out = reinterpret_cast<uint16_t*>(p.Y) + (int64_t)m * p.ldy + nc;
-                    if (wide && !(h & 1) && nc + 16 <= p.N) {          // stored together with the next group
-                        carry = make_uint4(pack_bf16x2(y[0], y[1]), pack_bf16x2(y[2], y[3]), pack_bf16x2(y[4], y[5]), pack_bf16x2(y[6], y[7]));
-                    } else if (wide && (h & 1) && full) {              // (the even group is in `carry`: nc - 8 + 16 <= N)
-                        st_global_v8(out - 8, carry.x, carry.y, carry.z, carry.w, pack_bf16x2(y[0], y[1]), pack_bf16x2(y[2], y[3]),
-                                     pack_bf16x2(y[4], y[5]), pack_bf16x2(y[6], y[7]));
-                    } else if (full && (p.ldy % 8 == 0)) {
-                        *reinterpret_cast<uint4*>(out) = make_uint4(pack_bf16x2(y[0], y[1]), pack_bf16x2(y[2], y[3]),
-                                                                    pack_bf16x2(y[4], y[5]), pack_bf16x2(y[6], y[7]));
-                    } else {
-                        for (int i = 0; i < 8; ++i) if (nc + i < p.N) out[i] = (uint16_t)f32_to_bf16_bits(y[i]);
-                    }
-                }
+        };
+        auto store8_f32 = [&](int m, int nc, const float (&y)[8]) {
+            float* out = reinterpret_cast<float*>(p.Y) + (int64_t)m * p.ldy + nc;
+            if (nc + 8 <= p.N && wide) {
+                st_global_v8(out, __float_as_uint(y[0]), __float_as_uint(y[1]), __float_as_uint(y[2]), __float_as_uint(y[3]),
+                             __float_as_uint(y[4]), __float_as_uint(y[5]), __float_as_uint(y[6]), __float_as_uint(y[7]));
+            } else if (nc + 8 <= p.N && (p.ldy % 4 == 0)) {
+                *reinterpret_cast<float4*>(out) = make_float4(y[0], y[1], y[2], y[3]);
+                *reinterpret_cast<float4*>(out + 4) = make_float4(y[4], y[5], y[6], y[7]);
+            } else {
+#pragma unroll
+                for (int i = 0; i < 8; ++i) if (nc + i < p.N) out[i] = y[i];
             }
-            if (p.dbg_main) {                    // test aids: the raw integer accumulators
+        };
+        // 16 consecutive bf16 columns of row m from column nc, packed two to a word
+        auto store16_bf16 = [&](int m, int nc, uint32_t w0, uint32_t w1, uint32_t w2, uint32_t w3, uint32_t w4, uint32_t w5, uint32_t w6,
+                                uint32_t w7) {
+            uint16_t* out = reinterpret_cast<uint16_t*>(p.Y) + (int64_t)m * p.ldy + nc;
+            if (nc + 16 <= p.N && wide) {
+                st_global_v8(out, w0, w1, w2, w3, w4, w5, w6, w7);
+            } else if (nc + 16 <= p.N && (p.ldy % 8 == 0)) {
+                *reinterpret_cast<uint4*>(out) = make_uint4(w0, w1, w2, w3);
+                *reinterpret_cast<uint4*>(out + 8) = make_uint4(w4, w5, w6, w7);
+            } else {
+                const uint32_t w[8] = {w0, w1, w2, w3, w4, w5, w6, w7};
+#pragma unroll
+                for (int i = 0; i < 16; ++i) if (nc + i < p.N) out[i] = (uint16_t)((w[i >> 1] >> ((i & 1) * 16)) & 0xFFFFu);
+            }
+        };
+        auto dbg8 = [&](int m, int nc, const uint32_t (&a0)[8], const uint32_t (&a1)[8]) {     // test aids: the raw integer accumulators
+            if (p.dbg_main) {
                 int32_t* d = p.dbg_main + (int64_t)m * p.N + nc;
+#pragma unroll
                 for (int i = 0; i < 8; ++i) if (nc + i < p.N) d[i] = (int32_t)a0[i];
             }
             if (p.dbg_out) {
                 int32_t* d = p.dbg_out + (int64_t)m * p.N + nc;
+#pragma unroll
                 for (int i = 0; i < 8; ++i) if (nc + i < p.N) d[i] = has_o ? (int32_t)a1[i] : 0;
             }
         };
@@ -300,7 +301,10 @@ __global__ void __launch_bounds__(kF256Threads, 1) fwd256_kernel(const __grid_co
             const float dxm = m < p.M ? __ldg(p.dx + m) : 0.0f;
             if (!mbar_wait(tmem_full_bar, (uint32_t)(t & 1), abort_flag)) { ok = false; break; }
             tc_fence_after();
-            // columns [0,128) of the tile: main accumulator and round 0, straight from TMEM
+            // columns [0,128) of the tile: main accumulator and round 0, straight from TMEM.  A bf16 result stays in
+            // registers (16 words for this thread's 32 columns) and is stored after the hand-over below: the stores
+            // then overlap the next tile's main contraction instead of keeping the tensor pipe waiting.
+            uint32_t ypk[16];
 #pragma unroll
             for (int h = 0; h < 4; ++h) {
                 const int nc = n0 + cq * 32 + 8 * h;
@@ -309,7 +313,14 @@ __global__ void __launch_bounds__(kF256Threads, 1) fwd256_kernel(const __grid_co
                 if (has_o) tmem_ld_32x8(aux_o + (uint32_t)(8 * h), a1);
                 if (has_l) tmem_ld_32x8(aux_l + (uint32_t)(8 * h), a2);
                 tmem_ld_wait();
-                if (m < p.M && nc < p.N) finish8(m, dxm, nc, h, 0, a0, a1, a2);
+                float y[8];
+                compute8(dxm, h, 0, a0, a1, a2, y);
+#pragma unroll
+                for (int i = 0; i < 4; ++i) ypk[4 * h + i] = pack_bf16x2(y[2 * i], y[2 * i + 1]);
+                if (m < p.M && nc < p.N) {
+                    if (p.y_f32) store8_f32(m, nc, y);
+                    dbg8(m, nc, a0, a1);
+                }
             }
             // columns [128,256): the main accumulator goes into registers until round 1 is there
             uint32_t acc[32];
@@ -320,6 +331,10 @@ __global__ void __launch_bounds__(kF256Threads, 1) fwd256_kernel(const __grid_co
             if (lane == 0) {
                 if (rank != 0) mbar_arrive_cluster(lead_tmem_empty);
                 else mbar_arrive(tmem_empty_bar);
+            }
+            if (!p.y_f32 && m < p.M) {
+                store16_bf16(m, n0 + cq * 32, ypk[0], ypk[1], ypk[2], ypk[3], ypk[4], ypk[5], ypk[6], ypk[7]);
+                store16_bf16(m, n0 + cq * 32 + 16, ypk[8], ypk[9], ypk[10], ypk[11], ypk[12], ypk[13], ypk[14], ypk[15]);
             }
             if (!mbar_wait(aux_ready_bar, (uint32_t)(t & 1), abort_flag)) { ok = false; break; }
             tc_fence_after();
@@ -332,7 +347,17 @@ __global__ void __launch_bounds__(kF256Threads, 1) fwd256_kernel(const __grid_co
                 tmem_ld_wait();
 #pragma unroll
                 for (int i = 0; i < 8; ++i) a0[i] = acc[8 * h + i];
-                if (m < p.M && nc < p.N) finish8(m, dxm, nc, h, 1, a0, a1, a2);
+                float y[8];
+                compute8(dxm, h, 1, a0, a1, a2, y);
+#pragma unroll
+                for (int i = 0; i < 4; ++i) ypk[4 * h + i] = pack_bf16x2(y[2 * i], y[2 * i + 1]);
+                if (m < p.M && nc < p.N) {
+                    if (p.y_f32) store8_f32(m, nc, y);
+                    dbg8(m, nc, a0, a1);
+                }
+                if ((h & 1) && !p.y_f32 && m < p.M)
+                    store16_bf16(m, nc - 8, ypk[4 * h - 4], ypk[4 * h - 3], ypk[4 * h - 2], ypk[4 * h - 1], ypk[4 * h], ypk[4 * h + 1], ypk[4 * h + 2],
+                                 ypk[4 * h + 3]);
             }
             tc_fence_before();
             __syncwarp();
