@@ -301,9 +301,9 @@ __global__ void __launch_bounds__(kF256Threads, 1) fwd256_kernel(const __grid_co
             const float dxm = m < p.M ? __ldg(p.dx + m) : 0.0f;
             if (!mbar_wait(tmem_full_bar, (uint32_t)(t & 1), abort_flag)) { ok = false; break; }
             tc_fence_after();
-            // columns [0,128) of the tile: main accumulator and round 0, straight from TMEM.  A bf16 result stays in
-            // registers (16 words for this thread's 32 columns) and is stored after the hand-over below: the stores
-            // then overlap the next tile's main contraction instead of keeping the tensor pipe waiting.
+            // columns [0,128) of the tile: main accumulator and round 0, straight from TMEM.  Half of a bf16 result
+            // (8 packed words of this thread's 32 columns; more would spill) stays in registers and is stored after the
+            // hand-over below: those stores overlap the next tile's main contraction instead of keeping the tensor pipe waiting.
             uint32_t ypk[16];
 #pragma unroll
             for (int h = 0; h < 4; ++h) {
@@ -321,6 +321,8 @@ __global__ void __launch_bounds__(kF256Threads, 1) fwd256_kernel(const __grid_co
                     if (p.y_f32) store8_f32(m, nc, y);
                     dbg8(m, nc, a0, a1);
                 }
+                if (h == 1 && !p.y_f32 && m < p.M)
+                    store16_bf16(m, n0 + cq * 32, ypk[0], ypk[1], ypk[2], ypk[3], ypk[4], ypk[5], ypk[6], ypk[7]);
             }
             // columns [128,256): the main accumulator goes into registers until round 1 is there
             uint32_t acc[32];
@@ -333,7 +335,6 @@ __global__ void __launch_bounds__(kF256Threads, 1) fwd256_kernel(const __grid_co
                 else mbar_arrive(tmem_empty_bar);
             }
             if (!p.y_f32 && m < p.M) {
-                store16_bf16(m, n0 + cq * 32, ypk[0], ypk[1], ypk[2], ypk[3], ypk[4], ypk[5], ypk[6], ypk[7]);
                 store16_bf16(m, n0 + cq * 32 + 16, ypk[8], ypk[9], ypk[10], ypk[11], ypk[12], ypk[13], ypk[14], ypk[15]);
             }
             if (!mbar_wait(aux_ready_bar, (uint32_t)(t & 1), abort_flag)) { ok = false; break; }
