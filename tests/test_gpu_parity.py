@@ -173,12 +173,15 @@ def test_qlinear_fwd_each_tile_width(Q, M, K, N, nO, r, tile_n):
         Q.quaff_debug_force_fwd_tile(0)
 
 
-def _check_fwd(Q, M, K, N, nO, r, y_f32):
+def _check_fwd(Q, M, K, N, nO, r, y_f32, y_pad=0):
     import torch
     O, X, Wt, A, B, _ = _mk_inputs(500 + M + N, M, K, N, nO, r)
     Wq, dW, W_O, wmax, s, Xq, xqo, dx, wq, dw = _oracle_state(O, X, Wt)
     nOp = _pad32(nO)
-    Y = torch.full((M, N), float("nan"), dtype=torch.float32 if y_f32 else torch.bfloat16, device="cuda")
+    # Y is a view of a wider buffer with two more rows: whatever lands outside [M][N] shows in the sentinel
+    SENT = -777.0
+    Ybuf = torch.full((M + 2, N + y_pad), SENT, dtype=torch.float32 if y_f32 else torch.bfloat16, device="cuda")
+    Y = Ybuf[:M, :N]
     a1 = torch.full((M, N), -7, dtype=torch.int32, device="cuda")
     a2 = torch.full((M, N), -7, dtype=torch.int32, device="cuda")
     T = torch.empty((M, r), dtype=torch.bfloat16, device="cuda") if r else None
@@ -199,6 +202,19 @@ def _check_fwd(Q, M, K, N, nO, r, y_f32):
     slack = flip_slack(f32(oT).T, f32(B), 0.5) if r else None
     err = max_rel_err(host(Y), oY, slack)
     assert err <= tol, f"max rel err {err:.3e}"
+    assert bool((Ybuf[M:, :] == SENT).all()) and bool((Ybuf[:, N:] == SENT).all()), "write outside Y"
+
+
+# Row pitches of Y that take the three store paths of the wide forward kernels: 32-byte stores (pitch a multiple of 32
+# bytes), 16-byte stores (a multiple of 16 only), element stores (neither); ragged M and N.
+@pytest.mark.parametrize("tile_n", [128, 192, 256])
+@pytest.mark.parametrize("y_f32,y_pad", [(False, 16), (False, 8), (False, 3), (True, 8), (True, 4), (True, 1)])
+def test_qlinear_fwd_padded_output(Q, tile_n, y_f32, y_pad):
+    Q.quaff_debug_force_fwd_tile(tile_n)
+    try:
+        _check_fwd(Q, 300, 512, 1000, 20, 16, y_f32, y_pad)
+    finally:
+        Q.quaff_debug_force_fwd_tile(0)
 
 
 # ----------------------------------------------------------------------------- S6-S8 backward
@@ -217,7 +233,8 @@ def test_qlinear_bwd(Q, M, K, N, nO, r):
     nOp = _pad32(nO)
     oY, oT, _, _ = oracle.qlinear_fwd(Xq, xqo, dx, Wq, dW, wq, dw, X, A, B, 0.5)
     odX, odA, odB, oG = oracle.qlinear_bwd(dY, Wq, dW, wq, dw, O, s, X, oT, A, B, 0.5)
-    dX = torch.full((M, K), float("nan"), dtype=torch.bfloat16, device="cuda")
+    dXbuf = torch.full((M + 2, K + 8), -777.0, dtype=torch.bfloat16, device="cuda")     # dX: a view with a sentinel frame
+    dX = dXbuf[:M, :K]
     dA = torch.full((K, r), 1.0, dtype=torch.float32, device="cuda") if r else None
     dB = torch.full((r, N), 1.0, dtype=torch.float32, device="cuda") if r else None
     st = torch.zeros(4, dtype=torch.int32, device="cuda")
@@ -237,6 +254,7 @@ def test_qlinear_bwd(Q, M, K, N, nO, r):
     sl_dB = flip_slack(f32(oT), f32(dY), 0.5) if r else None         # [r][N]
     err = max_rel_err(host(dX), odX, sl_dX)
     assert err <= TOL_BF16, f"dX max rel err {err:.3e}"
+    assert bool((dXbuf[M:, :] == -777.0).all()) and bool((dXbuf[:, K:] == -777.0).all()), "write outside dX"
     if nO:
         err_o = max_rel_err(host(dX)[:, O], odX[:, O], sl_dX[:, O] if r else None)
         assert err_o <= TOL_BF16, f"dX outlier columns max rel err {err_o:.3e}"
