@@ -348,6 +348,40 @@ def run_gpu(args, wl):
 
     # ---- per-kernel figures and the roofline of the dominant kernel
     peaks = load_peaks()
+    # The HBM-bound kernels of every layer, each alone on the layer's own buffers: one launch between two events, L2
+    # flushed before it (the launch latency is inside the figure, which is what bounds the small shapes).
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    hbm_kernels = []
+    layers0, xs0, _ = sets[0]
+
+    def alone_ms(fn):
+        ts = []
+        for i in range(13):
+            flush.sum()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(); fn(); b.record()
+            torch.cuda.synchronize()
+            if i >= 3:
+                ts.append(a.elapsed_time(b))
+        return float(np.median(ts))
+
+    one = torch.zeros(1, device="cuda")
+    launch_floor_ms = alone_ms(lambda: one.zero_())      # the same bracket around a one-element fill: what no kernel can go below
+    for li, sp in enumerate(wl.layers):
+        l = layers0[li]
+        nOp = synth.pad_to(sp.nO, 32)
+        cases = [("quant_act", lambda l=l, li=li: Q.quaff_quant_act(xs0[li], l.O_idx, l.s_O, l.Xq, l.xq_O, l.dx),
+                  M * sp.K * 3 + M * nOp + 4 * M)]
+        if sp.nO:
+            cases.append(("momentum", lambda l=l, li=li: Q.quaff_momentum_update(xs0[li], l.O_idx, l.wmax_O, l.gamma, l.s_O, l.ws, l.colmax_O, l.beta_O),
+                          32 * M * sp.nO))
+            cases.append(("requant_rows", lambda l=l: Q.quaff_requant_weight_rows(l.W_O, l.s_O, l.wq_O, l.dw_O),
+                          2 * sp.nO * sp.N + nOp * sp.N + 4 * sp.N))
+        for kname, fn, nbytes in cases:
+            kms = alone_ms(fn)
+            gbs = nbytes / (kms * 1e-3) / 1e9
+            hbm_kernels.append({"layer": sp.name, "kernel": kname, "ms": kms, "algorithmic_bytes": nbytes, "gbs": gbs,
+                                "frac_of_hbm_peak": gbs / peaks["hbm_gbs"]})
     # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the ncu captures summarised under
     # profiles/; only for the shapes captured there, and only while those kernels are unchanged
     ncu_traffic = {("fwd_int8_gemm", 2048, 3072, 9216, 32, 16): 40.3e6, ("bwd_bf16_gemm", 2048, 3072, 9216, 32, 16): 131.6e6}
@@ -393,7 +427,10 @@ def run_gpu(args, wl):
             "e2e": {"value": qdist.whole_job_rate(M, world, e2e_ms), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                     "ms_per_step": e2e_ms, "steps": e2e_steps},
             "gpu_launches": int(launches),
-            "roofline": roofline, "layers": per_layer, "cpu_baseline": cpu}
+            "roofline": roofline, "layers": per_layer, "hbm_kernels": {"timing": "each kernel alone on the layer's buffers, one launch between two events, L2 flushed before it; "
+                                      "launch_floor_ms is the same bracket around a one-element fill",
+                            "launch_floor_ms": launch_floor_ms, "hbm_peak_gbs": peaks["hbm_gbs"], "kernels": hbm_kernels},
+            "cpu_baseline": cpu}
     print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
