@@ -14,7 +14,8 @@
 //   round (t-1, 1) | main(t) block 0 .. last | round (t, 0) | round (t, 1) | main(t+1) ...
 //
 // When the main accumulator of tile t and its round 0 are complete (tmem_full), the sixteen epilogue warps
-//   1. finish columns [0,128) straight from TMEM (main + round 0) and store them,
+//   1. finish columns [0,128) straight from TMEM (main + round 0); half of a bf16 result is stored at once, the other
+//      half waits packed in registers and is stored after the hand-over,
 //   2. copy columns [128,256) of the main accumulator into registers (32 per thread),
 // and hand main accumulator and round accumulators back (tmem_empty): the tensor pipe waits only for that.  It then
 // runs round 1 of tile t and starts the main contraction of tile t+1, during which the warps combine their registers
