@@ -48,7 +48,7 @@ quaff_status_t make_tmap_2d(CUtensorMap* map, const void* base, int elem_bytes, 
 // branches of the graph.
 struct SideStreams {
     cudaStream_t s[2];
-    cudaEvent_t fork[2], join[2];
+    cudaEvent_t fork[2], join[2], g_ready;
     bool ok;
 };
 static SideStreams* side_streams() {
@@ -60,8 +60,13 @@ static SideStreams* side_streams() {
     if (!tried[dev]) {
         tried[dev] = true;
         ss.ok = true;
+        // lowest priority: where a side-stream kernel and the caller's kernel are ready at the same time, the block
+        // scheduler serves the caller's (the big GEMM) first and fills the side work in as SMs come free
+        int least = 0, greatest = 0;
+        cudaDeviceGetStreamPriorityRange(&least, &greatest);
+        ss.ok = ss.ok && cudaEventCreateWithFlags(&ss.g_ready, cudaEventDisableTiming) == cudaSuccess;
         for (int i = 0; i < 2; ++i) {
-            ss.ok = ss.ok && cudaStreamCreateWithFlags(&ss.s[i], cudaStreamNonBlocking) == cudaSuccess;
+            ss.ok = ss.ok && cudaStreamCreateWithPriority(&ss.s[i], cudaStreamNonBlocking, least) == cudaSuccess;
             ss.ok = ss.ok && cudaEventCreateWithFlags(&ss.fork[i], cudaEventDisableTiming) == cudaSuccess;
             ss.ok = ss.ok && cudaEventCreateWithFlags(&ss.join[i], cudaEventDisableTiming) == cudaSuccess;
         }
@@ -720,6 +725,7 @@ extern "C" quaff_status_t quaff_qlinear_bwd(int M, int K, int N, const quaff_bf1
         if ((rc = skinny_gemm(0, dY, lddy, B, N, M, N, r, part, status_opt, st, &S)) != QUAFF_OK) return rc;
         launch_pdl(reduce_parts_bf16_kernel, dim3(ceil_div(M * r / 8, 256)), dim3(256), 0, st, 1, part, S, M, r, lora_scale, G);
         if ((rc = launch_status()) != QUAFF_OK) return rc;
+        if (ss && cudaEventRecord(ss->g_ready, st) != cudaSuccess) return QUAFF_ERR_CUDA;
     }
     if (want_dAB) {   // dB^T = dY^T T: the contraction runs over the tokens, the slow axis of dY and T: MN-major operands
         if ((rc = skinny_gemm(1, dY, lddy, T, r, N, M, r, part_b, status_opt, s_db, &S)) != QUAFF_OK) return rc;
@@ -771,11 +777,15 @@ extern "C" quaff_status_t quaff_qlinear_bwd(int M, int K, int N, const quaff_bf1
         rc = TN > 128 ? launch_gemm<EPI_BWD, CTAS, 256>(p, st) : launch_gemm<EPI_BWD, CTAS, 128>(p, st);
         if (rc != QUAFF_OK) return rc;
     }
-    if (want_dAB) {   // dA = X^T G (MN-major operands), beside the outlier fix-up
+    if (want_dAB) {
+        // dA = X^T G (MN-major operands) needs G, not the grad-input GEMM: on side stream 0 it follows the weight
+        // dequantization and waits for G only.  It is enqueued BEHIND the GEMM, so the persistent GEMM gets every SM
+        // first and the split-K CTAs of dA move in as the pairs that have no tile left in the last wave retire.
         cudaStream_t s_da = st;
         bool forked_da = false;
-        if (ss && dX && nO > 0) {
-            if (!(forked_da = fork_to(ss, 0, st))) return QUAFF_ERR_CUDA;
+        if (ss && dX) {
+            if (cudaStreamWaitEvent(ss->s[0], ss->g_ready, 0) != cudaSuccess) return QUAFF_ERR_CUDA;
+            forked_da = true;
             s_da = ss->s[0];
         }
         if ((rc = skinny_gemm(1, X, ldx, G, r, K, M, r, part_a, status_opt, s_da, &S)) != QUAFF_OK) return rc;
