@@ -413,6 +413,32 @@ def run_gpu(args, wl):
                 "avg_launch_ms": ms,
                 "timing": f"CUDA event pair around the kernel in an instrumented pass over the same steps ({inst_steps} steps, "
                           f"{inst_ms_per_step:.4f} ms per step with the event nodes in the graph)"}
+    if kind == "bwd_bf16_gemm":
+        # Inside the step the grad-input GEMM shares the SMs: the split-K GEMMs of dA and dB are scheduled into the SMs
+        # its last wave leaves idle, which shortens the step and lengthens the GEMM.  The same kernel alone (a backward
+        # call for dX only on the same layer's buffers, L2 flushed before it) is reported beside it.
+        li = [sp.name for sp in wl.layers].index(name)
+        l = layers0[li]
+        dY0 = sets[0][2][li]
+        def gemm_alone():
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(); b.record()
+            Q.quaff_debug_time_gemm(1, a, b)
+            Q.quaff_qlinear_bwd(dY0, l.Wq, l.dW, l.wq_O, l.dw_O, l.O_idx, l.s_O, l._X, l.T, l.A, l.B, l.lora_scale, l.dX, None, None,
+                                False, l.ws, l.status)
+            torch.cuda.synchronize()
+            return a.elapsed_time(b)
+        ts = []
+        for i in range(13):
+            flush.sum()
+            t_ms = gemm_alone()
+            if i >= 3:
+                ts.append(t_ms)
+        alone_ms_ = float(np.median(ts))
+        roofline["alone"] = {"avg_launch_ms": alone_ms_, "achieved": work / (alone_ms_ * 1e-3) / 1e12,
+                             "frac": work / (alone_ms_ * 1e-3) / 1e12 / peaks["bf16_tflops"],
+                             "note": "the same kernel without the LoRA-gradient GEMMs beside it (backward for dX only, L2 flushed), "
+                                     "against the burst peak"}
 
     cpu = cpu_baseline(wl, min(wl.M, 8 * args.sample_tokens), reps=5) if not args.no_cpu_baseline else None
     line = {"metric": METRIC, "value": qdist.whole_job_rate(M, world, ms_per_step), "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -481,7 +507,8 @@ def run_micro(args):
             if which == 0:
                 Q.quaff_qlinear_fwd(Xq, xqo, dxv, Wq, dWv, wqo, dwOv, X, A, B, 1.0, T, Y, ws, None, None, st)
             else:
-                Q.quaff_qlinear_bwd(dY, Wq, dWv, wqo, dwOv, O, s, X, T, A, B, 1.0, dX, dA, dB, False, ws, st)
+                # (dX only: with dA / dB the library schedules their split-K GEMMs into the SMs the grad-input GEMM leaves idle)
+                Q.quaff_qlinear_bwd(dY, Wq, dWv, wqo, dwOv, O, s, X, T, A, B, 1.0, dX, None, None, False, ws, st)
             torch.cuda.synchronize()
             if i >= args.warmup:
                 times.append(e0.elapsed_time(e1))

@@ -717,8 +717,8 @@ extern "C" quaff_status_t quaff_qlinear_bwd(int M, int K, int N, const quaff_bf1
     bool forked0 = false, forked1 = false;
 
     // Launch order = the order in which the block scheduler hands out SM slots while everything below runs at once:
-    // the chain the grad-input GEMM waits for longest (G) first, the bulk dequantization last.  The side streams fork
-    // off before any of it, so that they depend on nothing launched here.
+    // the chain the grad-input GEMM waits for longest (G) first, then the bulk dequantization; dB and dA come behind
+    // the GEMM.  The side streams fork off before any of it, so that they depend on nothing launched here.
     if (ss && want_dAB && !(forked1 = fork_to(ss, 1, st))) return QUAFF_ERR_CUDA;
     if (ss && dX && !(forked0 = fork_to(ss, 0, st))) return QUAFF_ERR_CUDA;
     if (r > 0) {   // G = bf16(lora_scale * dY B^T): B [r][N] is already K-major for this contraction over N
@@ -726,11 +726,6 @@ extern "C" quaff_status_t quaff_qlinear_bwd(int M, int K, int N, const quaff_bf1
         launch_pdl(reduce_parts_bf16_kernel, dim3(ceil_div(M * r / 8, 256)), dim3(256), 0, st, 1, part, S, M, r, lora_scale, G);
         if ((rc = launch_status()) != QUAFF_OK) return rc;
         if (ss && cudaEventRecord(ss->g_ready, st) != cudaSuccess) return QUAFF_ERR_CUDA;
-    }
-    if (want_dAB) {   // dB^T = dY^T T: the contraction runs over the tokens, the slow axis of dY and T: MN-major operands
-        if ((rc = skinny_gemm(1, dY, lddy, T, r, N, M, r, part_b, status_opt, s_db, &S)) != QUAFF_OK) return rc;
-        launch_pdl(reduce_parts_kernel, dim3(ceil_div(N * r / 4, 256)), dim3(256), 0, s_db, 1, part_b, S, N, r, lora_scale, 1, accumulate, dB);
-        if ((rc = launch_status()) != QUAFF_OK) return rc;
     }
     constexpr int CTAS = 2;
     const int TN = w.tile_n, Kpad = w.Kpad;
@@ -743,9 +738,6 @@ extern "C" quaff_status_t quaff_qlinear_bwd(int M, int K, int N, const quaff_bf1
     }
     if (dX) {
         if (forked0 && !join_from(ss, 0, st)) return QUAFF_ERR_CUDA;     // the dequantized weight is ready
-        // dB is joined here too: the persistent GEMM wants every SM, a straggler beside it only delays its CTAs
-        if (forked1 && !join_from(ss, 1, st)) return QUAFF_ERR_CUDA;
-        forked1 = false;
         GemmParams p;
         memset(&p, 0, sizeof(p));
         int np = 0;
@@ -776,6 +768,16 @@ extern "C" quaff_status_t quaff_qlinear_bwd(int M, int K, int N, const quaff_bf1
         p.tile_n = TN;      // the 256-column instance serves every width above 128
         rc = TN > 128 ? launch_gemm<EPI_BWD, CTAS, 256>(p, st) : launch_gemm<EPI_BWD, CTAS, 128>(p, st);
         if (rc != QUAFF_OK) return rc;
+    }
+    if (want_dAB) {
+        // dB^T = dY^T T: the contraction runs over the tokens, the slow axis of dY and T: MN-major operands.  It needs
+        // nothing computed here, but it is held back (side stream 1 waits for the end of the dequantization) until the
+        // grad-input GEMM is ready too and enqueued behind it: with the lowest priority it then runs in the SMs the GEMM
+        // leaves free instead of competing with G and the dequantization for HBM in front of the GEMM.
+        if (ss && dX && cudaStreamWaitEvent(ss->s[1], ss->join[0], 0) != cudaSuccess) return QUAFF_ERR_CUDA;
+        if ((rc = skinny_gemm(1, dY, lddy, T, r, N, M, r, part_b, status_opt, s_db, &S)) != QUAFF_OK) return rc;
+        launch_pdl(reduce_parts_kernel, dim3(ceil_div(N * r / 4, 256)), dim3(256), 0, s_db, 1, part_b, S, N, r, lora_scale, 1, accumulate, dB);
+        if ((rc = launch_status()) != QUAFF_OK) return rc;
     }
     if (want_dAB) {
         // dA = X^T G (MN-major operands) needs G, not the grad-input GEMM: on side stream 0 it follows the weight
