@@ -205,11 +205,12 @@ quaff_status_t quaff_qlinear_fwd(int M, int K, int N,
  *   dY [M][N] bf16, lddy (lddy % 8 == 0);  T [M][r] bf16 from the forward
  *   Wq, wq_O: 16-byte aligned, ldwq_main and ldwq multiples of 16 (as in the forward)
  *   ws: QUAFF_WS_BWD bytes;  status_opt as in the forward.
- * Independent parts of the backward (weight dequantization, G, dB; later dA and the outlier fix-up) are forked
- * onto two library-owned side streams per device and joined back into `stream` before the call returns its
- * last launch: for the caller everything is still ordered on `stream`.  The side streams are created by the
- * first backward call on a device (make that call outside any stream capture); under capture the forks become
- * parallel branches of the captured graph.
+ * Independent parts of the backward are forked onto two library-owned side streams per device (lowest priority) and
+ * joined back into `stream` before the call returns its last launch: for the caller everything is still ordered on
+ * `stream`.  The weight dequantization runs beside G in front of the grad-input GEMM; dA and dB are enqueued behind the
+ * GEMM without depending on it, so that their split-K CTAs run in the SMs the GEMM's last wave leaves idle.  The side
+ * streams are created by the first backward call on a device (make that call outside any stream capture); under
+ * capture the forks become parallel branches of the captured graph.
  */
 quaff_status_t quaff_qlinear_bwd(int M, int K, int N,
                                  const quaff_bf16* dY, int64_t lddy,
