@@ -60,8 +60,8 @@ static SideStreams* side_streams() {
     if (!tried[dev]) {
         tried[dev] = true;
         ss.ok = true;
-        // lowest priority: where a side-stream kernel and the caller's kernel are ready at the same time, the block
-        // scheduler serves the caller's (the big GEMM) first and fills the side work in as SMs come free
+        // lowest priority, so that the side work never outranks the caller's stream (a default stream has the same
+        // priority: there the launch order decides, which is why the backward enqueues dA and dB behind its GEMM)
         int least = 0, greatest = 0;
         cudaDeviceGetStreamPriorityRange(&least, &greatest);
         ss.ok = ss.ok && cudaEventCreateWithFlags(&ss.g_ready, cudaEventDisableTiming) == cudaSuccess;
