@@ -261,6 +261,16 @@ def test_qlinear_bwd(Q, M, K, N, nO, r):
     if r:
         assert max_rel_err(host(dA), odA, sl_dA) <= TOL_BF16
         assert max_rel_err(host(dB), odB, sl_dB) <= TOL_BF16
+    # the two halves of the call on their own (other stream layout inside the library): the same kernels, the same bits
+    dX2 = torch.full((M, K), float("nan"), dtype=torch.bfloat16, device="cuda")
+    Q.quaff_qlinear_bwd(*args[:12], dX2, None, None, False, ws, st)            # dX only
+    torch.cuda.synchronize()
+    assert host(st)[0] == 0 and np.array_equal(host_bits(dX2), host_bits(dX.contiguous()))
+    if r:
+        dA2, dB2 = torch.full_like(dA, 2.0), torch.full_like(dB, 2.0)
+        Q.quaff_qlinear_bwd(*args[:12], None, dA2, dB2, False, ws, st)         # LoRA gradients only
+        torch.cuda.synchronize()
+        assert host(st)[0] == 0 and np.array_equal(host(dA2), host(dA)) and np.array_equal(host(dB2), host(dB))
         # gradient accumulation: a second call with accumulate adds the same gradients again
         Q.quaff_qlinear_bwd(*args, True, ws, st)
         torch.cuda.synchronize()
