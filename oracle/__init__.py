@@ -89,6 +89,26 @@ def momentum_update(X: np.ndarray, O_idx: np.ndarray, wmax_O: np.ndarray, gamma:
     return s, cm, be
 
 
+def outlier_colmax(X: np.ndarray, O_idx: np.ndarray) -> np.ndarray:
+    """Column maxima max_m |X[m, O_i]| of a batch (or of one shard of it), f32 [nO]."""
+    X = _c(X, np.uint16)
+    O_idx = _c(O_idx, np.int32)
+    M, K = X.shape
+    cm = np.empty(O_idx.shape[0], np.float32)
+    _load().qo_outlier_colmax(_p(X), I64(K), I32(M), _p(O_idx), I32(O_idx.shape[0]), _p(cm))
+    return cm
+
+
+def momentum_apply(colmax_O: np.ndarray, wmax_O: np.ndarray, gamma: float, s_O: np.ndarray):
+    """Eq. 8 then Eq. 7 from given column maxima.  Returns (s_new, beta); s_O is not modified."""
+    cm = _c(colmax_O, np.float32)
+    wmax_O = _c(wmax_O, np.float32)
+    s = _c(s_O, np.float32).copy()
+    be = np.empty(cm.shape[0], np.float32)
+    _load().qo_momentum_apply(_p(cm), _p(wmax_O), I32(cm.shape[0]), F32(gamma), _p(s), _p(be))
+    return s, be
+
+
 def quant_act(X: np.ndarray, O_idx: np.ndarray, s_O: np.ndarray, nOp: int, count_literal: bool = False):
     """Returns (Xq[M,K] int8, xq_O[M,nOp] int8, dx[M] f32[, n_literal_diff])."""
     X = _c(X, np.uint16)
@@ -134,8 +154,10 @@ def int_gemm(A: np.ndarray, B: np.ndarray) -> np.ndarray:
     return C
 
 
-def qlinear_fwd(Xq, xq_O, dx, Wq, dW, wq_O, dw_O, X, A, B, lora_scale: float):
-    """Returns (Y[M,N] f64, T[M,r] bf16 bits, acc1[M,N] i32, acc2[M,N] i32)."""
+def qlinear_fwd(Xq, xq_O, dx, Wq, dW, wq_O, dw_O, X, A, B, lora_scale: float, T_in=None):
+    """Returns (Y[M,N] f64, T[M,r] bf16 bits, acc1[M,N] i32, acc2[M,N] i32).
+
+    T_in (bf16 bits [M,r]): evaluate the LoRA up-projection on these bits of T instead of rounding X A here."""
     Xq = _c(Xq, np.int8)
     M, K = Xq.shape
     Wq = _c(Wq, np.int8)
@@ -151,13 +173,15 @@ def qlinear_fwd(Xq, xq_O, dx, Wq, dW, wq_O, dw_O, X, A, B, lora_scale: float):
     A_ = _c(A, np.uint16) if r else None
     B_ = _c(B, np.uint16) if r else None
     T = np.zeros((M, max(r, 1)), np.uint16)
+    if T_in is not None and r:
+        T[:, :r] = _c(T_in, np.uint16)
     Y = np.empty((M, N), np.float64)
     a1 = np.empty((M, N), np.int32)
     a2 = np.empty((M, N), np.int32)
     ov = _load().qo_qlinear_fwd(I32(M), I32(K), I32(N), _p(Xq), I64(K), _p(xq_O), I64(xq_O.shape[1]), I32(nOp), _p(dx),
                                 _p(Wq), I64(K), _p(dW), _p(wq_O), I64(wq_O.shape[1]), _p(dw_O),
                                 _p(X), I64(K), _p(A_), _p(B_), I32(r), F32(lora_scale),
-                                _p(T), _p(Y), _p(a1), _p(a2))
+                                _p(T), I32(1 if (T_in is not None and r) else 0), _p(Y), _p(a1), _p(a2))
     assert ov == 0, "integer accumulator overflow"
     return Y, T[:, :r], a1, a2
 
@@ -174,13 +198,15 @@ def lora_down(X, A):
     _load().qo_qlinear_fwd(I32(M), I32(K), I32(0), _p(_c(np.zeros((M, 1), np.int8), np.int8)), I64(1), _p(z8), I64(1), I32(0),
                            _p(_c(np.zeros(M, np.float32), np.float32)), _p(z8), I64(1), _p(zf), _p(z8), I64(1), _p(zf),
                            _p(X), I64(K), _p(_c(A, np.uint16)), _p(np.zeros((r, 1), np.uint16)), I32(r), F32(1.0),
-                           _p(T), _p(np.zeros(1, np.float64)), _p(None), _p(None))
+                           _p(T), I32(0), _p(np.zeros(1, np.float64)), _p(None), _p(None))
     return T
 
 
 def qlinear_bwd(dY, Wq, dW, wq_O, dw_O, O_idx, s_O, X, T, A, B, lora_scale: float,
-                want_dX: bool = True, want_dAB: bool = True):
-    """Returns (dX[M,K] f64 | None, dA[K,r] f64 | None, dB[r,N] f64 | None, G[M,r] bf16 bits)."""
+                want_dX: bool = True, want_dAB: bool = True, G_in=None):
+    """Returns (dX[M,K] f64 | None, dA[K,r] f64 | None, dB[r,N] f64 | None, G[M,r] bf16 bits).
+
+    G_in (bf16 bits [M,r]): use these bits of G = bf16(lora_scale dY B^T) instead of rounding the sum here."""
     dY = _c(dY, np.uint16)
     M, N = dY.shape
     Wq = _c(Wq, np.int8)
@@ -201,10 +227,11 @@ def qlinear_bwd(dY, Wq, dW, wq_O, dw_O, O_idx, s_O, X, T, A, B, lora_scale: floa
     dA = np.empty((K, r), np.float64) if (want_dAB and r) else None
     dB = np.empty((r, N), np.float64) if (want_dAB and r) else None
     G = np.zeros((M, max(r, 1)), np.uint16)
+    G_in_ = _c(G_in, np.uint16) if (G_in is not None and r) else None
     _load().qo_qlinear_bwd(I32(M), I32(K), I32(N), _p(dY), I64(N), _p(Wq), I64(K), _p(dW),
                            _p(wq_O), I64(wq_O.shape[1]), _p(dw_O), I32(nOp), _p(O_idx), I32(nO), _p(s_O),
                            _p(X), I64(K), _p(T_), _p(A_), _p(B_), I32(r), F32(lora_scale),
-                           _p(dX), _p(dA), _p(dB), _p(G))
+                           _p(dX), _p(dA), _p(dB), _p(G), _p(G_in_))
     return dX, dA, dB, G[:, :r]
 
 

@@ -143,6 +143,35 @@ void qo_momentum_update(const uint16_t* X, int64_t ldx, int M, int K, const int3
     }
 }
 
+/* The same update in two halves, for a batch whose tokens are spread over several workers: the column maxima of
+ * Eq. 8 are taken per shard (qo_outlier_colmax), combined by an elementwise maximum (max over a union of rows is the
+ * maximum of the per-shard maxima), and Eq. 8 / Eq. 7 are then applied to the combined maxima. */
+void qo_outlier_colmax(const uint16_t* X, int64_t ldx, int M, const int32_t* O_idx, int nO, float* colmax_O) {
+    for (int i = 0; i < nO; ++i) {
+        float cmax = 0.0f;
+        for (int m = 0; m < M; ++m) {
+            float a = fabsf(bf2f(X[(int64_t)m * ldx + O_idx[i]]));
+            if (a > cmax) cmax = a;
+        }
+        colmax_O[i] = cmax;
+    }
+}
+
+void qo_momentum_apply(const float* colmax_O, const float* wmax_O, int nO, float gamma, float* s_O, float* beta_O) {
+    float one_minus_gamma = 1.0f - gamma;
+    for (int i = 0; i < nO; ++i) {
+        float beta = 1.0f;
+        if (wmax_O[i] > 0.0f) {
+            float q = colmax_O[i] / wmax_O[i];
+            beta = fmaxf(1.0f, sqrtf(q));
+        }
+        float hist = gamma * s_O[i];
+        float cur = one_minus_gamma * beta;
+        s_O[i] = hist + cur;
+        if (beta_O) beta_O[i] = beta;
+    }
+}
+
 /* ---------------------------------------------------------------- Eq. 5 scaling + Eq. 1 per token
  *   Xhat[m][k] = X[m][k] / s_i   if k = O_i,  X[m][k] otherwise      (Xhat = X s^-1, s_i = 1 off O)
  *   Delta[m]   = max_k |Xhat[m][k]| / 127 ;  Xq[m][k] = [Xhat[m][k] / Delta[m]]
@@ -233,6 +262,8 @@ int64_t qo_int_gemm(const int8_t* A, int64_t lda, const int8_t* B, int64_t ldb, 
  *   Y[m][n] = dx[m] * (acc1 * dW[n] + acc2 * dw_O[n])                             Eq. 9, double
  *           + lora_scale * sum_j T[m][j] B[j][n],  T = bf16(X A)                  LoRA on the unquantized X
  * T_out [M][r] bf16, Y [M][N] double, acc1/acc2 [M][N] int32 (nullable).  r = 0 disables LoRA.
+ * t_given != 0: T_out is an INPUT (the bf16 down-projection as somebody else rounded it; a sum taken in another
+ * order may round one unit in the last place differently) and the LoRA up-projection is evaluated on those bits.
  * Returns the number of accumulators outside int32 (must be 0).
  */
 int64_t qo_qlinear_fwd(int M, int K, int N,
@@ -240,9 +271,9 @@ int64_t qo_qlinear_fwd(int M, int K, int N,
                        const int8_t* Wq, int64_t ldwq_main, const float* dW,
                        const int8_t* wq_O, int64_t ldwq, const float* dw_O,
                        const uint16_t* X, int64_t ldx, const uint16_t* A, const uint16_t* B, int r, float lora_scale,
-                       uint16_t* T_out, double* Y, int32_t* acc1_out, int32_t* acc2_out) {
+                       uint16_t* T_out, int t_given, double* Y, int32_t* acc1_out, int32_t* acc2_out) {
     int64_t overflow = 0;
-    if (r > 0) {
+    if (r > 0 && !t_given) {
 #pragma omp parallel for schedule(static)
         for (int m = 0; m < M; ++m)
             for (int j = 0; j < r; ++j) {
@@ -284,6 +315,7 @@ int64_t qo_qlinear_fwd(int M, int K, int N,
  *   G = bf16(lora_scale * dY B^T)  [M][r]
  *   dX = dXhat + G A^T ;  dA = X^T G  [K][r] ;  dB = lora_scale * T^T dY  [r][N]
  * dX [M][K], dA, dB in double (nullable each); G_out [M][r] bf16 (nullable).
+ * G_in (nullable): use these bf16 bits for G instead of rounding the sum here (see t_given of the forward).
  */
 void qo_qlinear_bwd(int M, int K, int N,
                     const uint16_t* dY, int64_t lddy,
@@ -292,18 +324,22 @@ void qo_qlinear_bwd(int M, int K, int N,
                     const int32_t* O_idx, int nO, const float* s_O,
                     const uint16_t* X, int64_t ldx, const uint16_t* T, const uint16_t* A, const uint16_t* B,
                     int r, float lora_scale,
-                    double* dX, double* dA, double* dB, uint16_t* G_out) {
+                    double* dX, double* dA, double* dB, uint16_t* G_out, const uint16_t* G_in) {
     (void)nOp;
     uint16_t* G = NULL;
     if (r > 0) {
         G = (uint16_t*)malloc(sizeof(uint16_t) * (size_t)M * (size_t)r);
+        if (G_in) {
+            memcpy(G, G_in, sizeof(uint16_t) * (size_t)M * (size_t)r);
+        } else {
 #pragma omp parallel for schedule(static)
-        for (int m = 0; m < M; ++m)
-            for (int j = 0; j < r; ++j) {
-                double g = 0.0;
-                for (int n = 0; n < N; ++n) g += (double)bf2f(dY[(int64_t)m * lddy + n]) * (double)bf2f(B[(int64_t)j * N + n]);
-                G[(int64_t)m * r + j] = d2bf((double)lora_scale * g);
-            }
+            for (int m = 0; m < M; ++m)
+                for (int j = 0; j < r; ++j) {
+                    double g = 0.0;
+                    for (int n = 0; n < N; ++n) g += (double)bf2f(dY[(int64_t)m * lddy + n]) * (double)bf2f(B[(int64_t)j * N + n]);
+                    G[(int64_t)m * r + j] = d2bf((double)lora_scale * g);
+                }
+        }
         if (G_out) memcpy(G_out, G, sizeof(uint16_t) * (size_t)M * (size_t)r);
     }
     if (dX) {

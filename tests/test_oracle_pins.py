@@ -156,6 +156,46 @@ def test_momentum_touches_only_outlier_columns():
     assert np.array_equal(cm, cm2)
 
 
+def test_split_momentum_update_equals_the_whole_batch_update():
+    """Tokens spread over shards: per-shard column maxima, elementwise maximum, then Eq. 8 / Eq. 7 - the same
+    s, bit for bit, as the update on the whole batch (a maximum does not depend on how the rows are grouped)."""
+    rng = np.random.default_rng(41)
+    X = rand_bf(rng, (37, 24), 30.0)
+    O = np.array([0, 5, 11, 23], np.int32)
+    wmax = np.array([0.04, 0.0, 0.07, 0.5], np.float32)
+    s0 = np.array([1.0, 2.5, 9.0, 1.25], np.float32)
+    s_ref, cm_ref, be_ref = oracle.momentum_update(X, O, wmax, 0.2, s0)
+    parts = [oracle.outlier_colmax(X[a:b], O) for a, b in ((0, 10), (10, 11), (11, 37))]
+    assert np.array_equal(parts[1], np.abs(f32(X[10]))[O])            # a one-row shard: the row itself
+    cm = np.maximum(np.maximum(parts[0], parts[1]), parts[2])
+    assert np.array_equal(cm, np.abs(f32(X))[:, O].max(axis=0)) and np.array_equal(cm, cm_ref)
+    s, be = oracle.momentum_apply(cm, wmax, 0.2, s0)
+    assert np.array_equal(s, s_ref) and np.array_equal(be, be_ref)
+    # Eq. 8 / Eq. 7 from given maxima: colmax = 9 wmax -> beta = 3; s = 0.5 * 5 + 0.5 * 3 = 4; zero weight row -> beta = 1
+    s, be = oracle.momentum_apply(np.array([2.25, 7.0], np.float32), np.array([0.25, 0.0], np.float32), 0.5,
+                                  np.array([5.0, 3.0], np.float32))
+    assert be.tolist() == [3.0, 1.0] and s.tolist() == [4.0, 2.0]
+
+
+# ----------------------------------------------------------------------------- weight preprocessing: W_O and max|W_i|
+def test_prepare_weight_outlier_rows_and_row_maxima_on_a_non_square_weight():
+    """Eq. 8's max|W_i| is taken over row i of W in R^{c_in x c_out}: over ALL outputs of input channel i, i.e. down
+    column O_i of the stored [N][K] layout.  A maximum over the wrong axis, or over the codes, fails here."""
+    rng = np.random.default_rng(42)
+    N, K = 7, 19                                   # non-square, so the two axes cannot be confused
+    Wt = rand_bf(rng, (N, K), 0.02)
+    Wt[3, 4] = 0x3F40                                # 0.75: the largest entry of input channel 4 sits in output channel 3
+    Wt[6, 17] = 0xBF00                              # -0.5: the maximum is over magnitudes
+    O = np.array([2, 4, 17], np.int32)
+    Wq, dW, W_O, wmax = oracle.prepare_weight(Wt, O)
+    assert W_O.shape == (3, N) and wmax.shape == (3,)
+    assert np.array_equal(W_O, Wt[:, O].T)                                         # W_O[i][n] = W[O_i][n] = Wt[n][O_i], bit for bit
+    assert np.array_equal(wmax, np.abs(f32(Wt))[:, O].max(axis=0))                 # over n, per input channel
+    assert wmax[1] == np.float32(0.75) and wmax[2] == np.float32(0.5)
+    # and the step sizes are per OUTPUT channel: over k, per row of the stored layout
+    assert np.array_equal(dW, np.abs(f32(Wt)).max(axis=1) / np.float32(127.0))
+
+
 # ----------------------------------------------------------------------------- integer GEMM
 def test_int_gemm_brute_force_python_ints():
     rng = np.random.default_rng(5)
@@ -305,6 +345,45 @@ def test_lora_branch_against_numpy_float64():
     # B = 0 (the usual initialisation): the branch vanishes
     Yz = _forward(O, X, Wq, dW, W_O, s, A, np.zeros_like(B), 2.0, 4)[0]
     assert np.array_equal(Yz, Y0)
+
+
+def test_supplied_intermediates_T_and_G_are_used_as_given():
+    """qlinear_fwd(T_in=...) and qlinear_bwd(G_in=...) evaluate everything downstream of the bf16 intermediate on the
+    given bits: with the oracle's own bits nothing changes; with one entry moved by one bf16 ulp the outputs move by
+    exactly that entry's term (numpy float64)."""
+    rng = np.random.default_rng(43)
+    M, K, N, nO, r = 9, 64, 20, 2, 8
+    O, X, Wt, A, B, Wq, dW, W_O, wmax, s = _setup(rng, M, K, N, nO, r)
+    nOp = 4
+    Xq, xqo, dx = oracle.quant_act(X, O, s, nOp)
+    wq, dw = oracle.requant_weight_rows(W_O, s, nOp)
+    Y, T, a1, a2 = oracle.qlinear_fwd(Xq, xqo, dx, Wq, dW, wq, dw, X, A, B, 0.5)
+    Y2, T2, b1, b2 = oracle.qlinear_fwd(Xq, xqo, dx, Wq, dW, wq, dw, X, A, B, 0.5, T_in=T)
+    assert np.array_equal(Y, Y2) and np.array_equal(T, T2) and np.array_equal(a1, b1) and np.array_equal(a2, b2)
+    Tm = T.copy()
+    Tm[4, 3] += 1                                              # next bf16 value away from zero
+    Y3, T3, _, _ = oracle.qlinear_fwd(Xq, xqo, dx, Wq, dW, wq, dw, X, A, B, 0.5, T_in=Tm)
+    assert np.array_equal(T3, Tm)
+    d = (f32(Tm).astype(np.float64) - f32(T).astype(np.float64))[4, 3]
+    expect = np.zeros_like(Y)
+    expect[4] = 0.5 * d * f32(B).astype(np.float64)[3]
+    assert d != 0 and np.allclose(Y3 - Y, expect, rtol=1e-9, atol=1e-15)
+
+    dY = rand_bf(rng, (M, N), 1e-2)
+    dX, dA, dB, G = oracle.qlinear_bwd(dY, Wq, dW, wq, dw, O, s, X, T, A, B, 0.5)
+    dX2, dA2, dB2, G2 = oracle.qlinear_bwd(dY, Wq, dW, wq, dw, O, s, X, T, A, B, 0.5, G_in=G)
+    assert np.array_equal(dX, dX2) and np.array_equal(dA, dA2) and np.array_equal(dB, dB2) and np.array_equal(G, G2)
+    Gm = G.copy()
+    Gm[2, 5] += 1
+    dX3, dA3, dB3, G3 = oracle.qlinear_bwd(dY, Wq, dW, wq, dw, O, s, X, T, A, B, 0.5, G_in=Gm)
+    assert np.array_equal(G3, Gm) and np.array_equal(dB3, dB)                  # dB does not depend on G
+    dg = (f32(Gm).astype(np.float64) - f32(G).astype(np.float64))[2, 5]
+    ex = np.zeros_like(dX)
+    ex[2] = dg * f32(A).astype(np.float64)[:, 5]                               # dX += G A^T
+    assert dg != 0 and np.allclose(dX3 - dX, ex, rtol=1e-9, atol=1e-15)
+    ea = np.zeros_like(dA)
+    ea[:, 5] = f32(X).astype(np.float64)[2] * dg                               # dA = X^T G
+    assert np.allclose(dA3 - dA, ea, rtol=1e-9, atol=1e-15)
 
 
 # ----------------------------------------------------------------------------- backward
