@@ -4,14 +4,19 @@
 A step is one pass of the whole path - momentum scale update, outlier weight-row re-quantization,
 activation scaling + quantization, INT8 forward GEMM with fused dequantization and LoRA, and the
 backward (grad-input through the dequantized INT8 weight, LoRA gradients) - over one batch of
-synthetic tokens through every linear layer of the workload.  Default workload: Phi-3-mini attention
-projections (2048 tokens; fused qkv 3072->9216 and o_proj 3072->3072; 32 outlier channels; LoRA r=16).
+synthetic tokens through every linear layer of the workload.  Default workload: the LLaMA-2-7B-shaped decoder
+block (8192 tokens; q/k/v/o 4096->4096, gate/up 4096->11008, down 11008->4096; 0.5 % outlier channels; LoRA r=64),
+the largest configuration that is timed on one GPU.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference]
+    python bench.py --workload sweep          # the shape sweep: one JSON line with a table of 324 points
 
-Prints ONE JSON line (rank 0).  `--impl reference` times the CPU oracle on a bounded token sample.
+Prints ONE JSON line (rank 0).  The timed region (`--steps` steps between two CUDA events) is repeated `--repeats`
+times; `ms_per_step` is the median over the repeats.  `--impl reference` times the CPU oracle on a bounded token sample.
 """
 import argparse
+import dataclasses
+import hashlib
 import json
 import os
 import subprocess
@@ -90,11 +95,39 @@ class ClockSampler:
 
 
 def layer_ops(M, sp, nOp):
-    """Algorithmic work of one layer-step: INT8 ops of the forward GEMMs, bf16 flops of the grad-input GEMM."""
+    """Algorithmic work of one layer-step: INT8 ops of the forward GEMMs (Eq. 9: main and outlier contraction), bf16
+    flops of the LoRA up-projection, bf16 flops of the grad-input GEMM (through the weight, the outlier rows, G A^T)."""
     fwd_int8 = 2.0 * M * sp.N * (sp.K + nOp)
     fwd_lora = 2.0 * M * sp.N * sp.r
-    bwd_bf16 = 2.0 * M * sp.N * sp.K + 2.0 * M * sp.N * 2 * nOp + 2.0 * M * sp.K * sp.r
+    bwd_bf16 = 2.0 * M * sp.N * sp.K + 2.0 * M * sp.N * nOp + 2.0 * M * sp.K * sp.r
     return fwd_int8, fwd_lora, bwd_bf16
+
+
+def kernel_source_hash():
+    """Hash of the CUDA sources: DRAM traffic figures taken with ncu are only valid for the sources they were taken on."""
+    h = hashlib.sha256()
+    csrc = os.path.join(ROOT, "paper_2505_14742_b200", "csrc")
+    for name in sorted(os.listdir(csrc)):
+        if name.endswith((".cu", ".cuh")):
+            h.update(open(os.path.join(csrc, name), "rb").read())
+    return h.hexdigest()[:16]
+
+
+def ncu_traffic_table():
+    """profiles/dram_traffic.txt: lines `kind M K N nO r bytes_per_launch source_hash` copied from ncu captures
+    (dram__bytes_read.sum + dram__bytes_write.sum).  Entries taken on other sources than the present ones are dropped."""
+    path = os.path.join(ROOT, "profiles", "dram_traffic.txt")
+    table = {}
+    if not os.path.exists(path):
+        return table
+    now = kernel_source_hash()
+    for line in open(path):
+        f = line.split()
+        if len(f) != 8 or line.startswith("#"):
+            continue
+        if f[7] == now:
+            table[(f[0],) + tuple(int(v) for v in f[1:6])] = float(f[6])
+    return table
 
 
 # --------------------------------------------------------------------------------------- CPU oracle legs
@@ -121,11 +154,11 @@ def oracle_setup(wl, sample_tokens):
     oracle.build()
     lins = [synth.layer_inputs(wl, li, b_std=0.02) for li in range(len(wl.layers))]
     state = []
+    small = dataclasses.replace(wl, M=sample_tokens)      # the same workload with a batch of `sample_tokens` tokens
     for li, lin in enumerate(lins):
         Wq, dW, W_O, wmax = oracle.prepare_weight(lin.W, lin.O_idx)
-        X, dY = synth.step_inputs(wl, li, 0, lin)
-        state.append({"Wq": Wq, "dW": dW, "W_O": W_O, "wmax": wmax, "s": np.ones(lin.spec.nO, np.float32),
-                      "X": np.ascontiguousarray(X[:sample_tokens]), "dY": np.ascontiguousarray(dY[:sample_tokens])})
+        X, dY = synth.step_inputs(small, li, 0, lin)
+        state.append({"Wq": Wq, "dW": dW, "W_O": W_O, "wmax": wmax, "s": np.ones(lin.spec.nO, np.float32), "X": X, "dY": dY})
     return lins, state
 
 
@@ -254,17 +287,20 @@ def run_gpu(args, wl):
         for l in layers:
             assert int(l.status[0].item()) == 0, "device-side wait timed out"
 
-    # ---- device-resident timed region
+    # ---- device-resident timed region: `steps` steps between two events, repeated; the median repeat counts
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    with ClockSampler(local) as clocks:
-        sync_all()
-        e0.record()
-        for i in range(args.steps):
-            run_step(i)
-        e1.record()
-        sync_all()
+    region_ms = []
+    with ClockSampler(local, period_ms=10) as clocks:
+        for rep in range(args.repeats):
+            sync_all()
+            e0.record()
+            for i in range(args.steps):
+                run_step(i)
+            e1.record()
+            sync_all()
+            region_ms.append(qdist.max_over_ranks(e0.elapsed_time(e1), "cuda"))
     launches = launches_per_step * args.steps
-    ms_per_step = qdist.max_over_ranks(e0.elapsed_time(e1), "cuda") / args.steps
+    ms_per_step = float(np.median(region_ms)) / args.steps
     # ---- the same steps once more with the event pairs: GEMM durations of the latest step on each buffer set
     inst_steps = max(REPLICAS, min(args.steps, 200))
     sync_all()
@@ -382,34 +418,40 @@ def run_gpu(args, wl):
             gbs = nbytes / (kms * 1e-3) / 1e9
             hbm_kernels.append({"layer": sp.name, "kernel": kname, "ms": kms, "algorithmic_bytes": nbytes, "gbs": gbs,
                                 "frac_of_hbm_peak": gbs / peaks["hbm_gbs"]})
-    # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the ncu captures summarised under
-    # profiles/; only for the shapes captured there, and only while those kernels are unchanged
-    ncu_traffic = {("fwd_int8_gemm", 2048, 3072, 9216, 32, 16): 40.3e6, ("bwd_bf16_gemm", 2048, 3072, 9216, 32, 16): 131.6e6}
+    ncu_traffic = ncu_traffic_table()
+    timed_total_ms = float(np.sum(region_ms))
+    sustained = timed_total_ms > 1000.0       # a region longer than a second runs under the power cap
+    bf16_peak = peaks["bf16_tflops_sustained"] if sustained else peaks["bf16_tflops"]
+    peak_note = f"{peaks['source']} cuBLAS bf16 {'sustained' if sustained else 'burst'}"
     per_layer = []
     dominant = None
     for li, sp in enumerate(wl.layers):
         nOp = synth.pad_to(sp.nO, 32)
         f_ms, b_ms = gemm_ms[li]
         fwd_int8, fwd_lora, bwd_bf16 = layer_ops(M, sp, nOp)
+        f_tops, b_tflops = (fwd_int8 + fwd_lora) / (f_ms * 1e-3) / 1e12, bwd_bf16 / (b_ms * 1e-3) / 1e12
         entry = {"layer": sp.name, "K": sp.K, "N": sp.N, "nO": sp.nO, "r": sp.r,
                  "fwd_gemm_ms": f_ms, "fwd_int8_tops": fwd_int8 / (f_ms * 1e-3) / 1e12,
                  "fwd_pct_of_int8_nominal_4500": 100.0 * fwd_int8 / (f_ms * 1e-3) / 4.5e15,
-                 "bwd_gemm_ms": b_ms, "bwd_bf16_tflops": bwd_bf16 / (b_ms * 1e-3) / 1e12,
-                 "bwd_pct_of_bf16_nominal_2250": 100.0 * bwd_bf16 / (b_ms * 1e-3) / 2.25e15}
+                 "fwd_roofline": {"bound": "tensor", "achieved": f_tops, "peak": 2.0 * bf16_peak, "unit": "TOP/s", "frac": f_tops / (2.0 * bf16_peak),
+                                  "traffic": ncu_traffic.get(("fwd_int8_gemm", M, sp.K, sp.N, sp.nO, sp.r))},
+                 "bwd_gemm_ms": b_ms, "bwd_bf16_tflops": b_tflops,
+                 "bwd_pct_of_bf16_nominal_2250": 100.0 * b_tflops / 2.25e3,
+                 "bwd_pct_of_int8_nominal_4500": 100.0 * b_tflops / 4.5e3,
+                 "bwd_roofline": {"bound": "tensor", "achieved": b_tflops, "peak": bf16_peak, "unit": "TFLOP/s", "frac": b_tflops / bf16_peak,
+                                  "traffic": ncu_traffic.get(("bwd_bf16_gemm", M, sp.K, sp.N, sp.nO, sp.r))}}
         per_layer.append(entry)
         for kind, ms, work in (("fwd_int8_gemm", f_ms, fwd_int8 + fwd_lora), ("bwd_bf16_gemm", b_ms, bwd_bf16)):
             if dominant is None or ms > dominant[2]:
                 dominant = (sp.name, kind, ms, work, ncu_traffic.get((kind, M, sp.K, sp.N, sp.nO, sp.r)))
-    sustained = ms_per_step * args.steps > 1000.0
-    bf16_peak = peaks["bf16_tflops_sustained"] if sustained else peaks["bf16_tflops"]
     name, kind, ms, work, traffic = dominant
     achieved = work / (ms * 1e-3) / 1e12
     peak = bf16_peak * (2.0 if kind == "fwd_int8_gemm" else 1.0)
-    roofline = {"bound": "tensor", "kernel": f"umma_gemm_kernel<{'EPI_FWD' if kind == 'fwd_int8_gemm' else 'EPI_BWD'}> ({name})",
+    roofline = {"bound": "tensor", "kernel": f"{'forward INT8 GEMM (Eq. 9 + LoRA)' if kind == 'fwd_int8_gemm' else 'umma_gemm_kernel<EPI_BWD> grad-input GEMM'} ({name})",
                 "achieved": achieved, "peak": peak, "unit": "TFLOP/s" if kind == "bwd_bf16_gemm" else "TOP/s",
                 "frac": achieved / peak, "traffic": traffic,
-                "peak_source": f"{peaks['source']} cuBLAS bf16 {'sustained' if sustained else 'burst'}"
-                               + (" x2 (nominal int8:bf16 ratio)" if kind == "fwd_int8_gemm" else ""),
+                "peak_source": peak_note + (" x2 (nominal int8:bf16 ratio)" if kind == "fwd_int8_gemm" else "")
+                               + f"; the timed region ran {timed_total_ms:.0f} ms",
                 "avg_launch_ms": ms,
                 "timing": f"CUDA event pair around the kernel in an instrumented pass over the same steps ({inst_steps} steps, "
                           f"{inst_ms_per_step:.4f} ms per step with the event nodes in the graph)"}
@@ -440,9 +482,11 @@ def run_gpu(args, wl):
                              "note": "the same kernel without the LoRA-gradient GEMMs beside it (backward for dX only, L2 flushed), "
                                      "against the burst peak"}
 
-    cpu = cpu_baseline(wl, min(wl.M, 8 * args.sample_tokens), reps=5) if not args.no_cpu_baseline else None
+    cpu = cpu_baseline(wl, min(wl.M, 8 * args.sample_tokens), reps=2) if not args.no_cpu_baseline else None
     line = {"metric": METRIC, "value": qdist.whole_job_rate(M, world, ms_per_step), "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+            "repeats": {"n": args.repeats, "ms_per_step_min": float(np.min(region_ms)) / args.steps,
+                        "ms_per_step_max": float(np.max(region_ms)) / args.steps, "ms_per_step_median": ms_per_step},
             "vs_baseline": None, "dtype": "int8 forward (int32 accumulate), bf16 backward (f32 accumulate)",
             "data": "synthetic",
             "config": {"workload": wl.name, "tokens_per_gpu": M,
@@ -570,6 +614,84 @@ def run_micro(args):
                                    "peak_source": f"{peaks['source']} copy bandwidth"}}), flush=True)
 
 
+def run_sweep(args):
+    """--workload sweep: one quantized linear layer, forward + backward, over the shape sweep - tokens M in {512, 2048,
+    8192, 32768}, K and N in {2048, 4096, 8192}, LoRA rank in {8, 32, 64}, outlier fraction in {0.5 %, 1 %, 5 %} of K -
+    324 points, 1 warm-up + 20 timed steps each (one CUDA graph replay per step, CUDA events around the 20).  Inputs
+    are drawn on the device (N(0,1) activations with nO seeded channels at 20-100x, N(0, 0.02) weight and LoRA factors):
+    this mode only times; parity at sweep points is the tests' business.  One JSON line with the table."""
+    import torch
+    from paper_2505_14742_b200 import binding as Q, build
+    from paper_2505_14742_b200.layer import QuaffLinear, StepGraph
+    build.build_library()
+    Q.lib()
+    torch.cuda.set_device(0)
+    peaks = load_peaks()
+    g = torch.Generator(device="cuda").manual_seed(synth.BASE_SEED + 4)
+    Ms = (512, 2048, 8192, 32768) if not args.sweep_quick else (512, 8192)
+    KN = (2048, 4096, 8192) if not args.sweep_quick else (2048, 8192)
+    ranks, fracs, steps = (8, 32, 64), (0.005, 0.01, 0.05), 20
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    points = []
+    launches = 0
+    with ClockSampler(0, period_ms=50) as clocks:
+        for K in KN:
+            for N in KN:
+                W = (0.02 * torch.randn((N, K), device="cuda", generator=g)).to(torch.bfloat16)
+                for frac in fracs:
+                    nO = max(1, int(round(frac * K)))
+                    nOp = synth.pad_to(nO, 32)
+                    O = torch.sort(torch.randperm(K, device="cuda", generator=g)[:nO])[0].to(torch.int32)
+                    mag = 20.0 + 80.0 * torch.rand(nO, device="cuda", generator=g)
+                    for r in ranks:
+                        A = (0.02 * torch.randn((K, r), device="cuda", generator=g)).to(torch.bfloat16)
+                        B = (0.02 * torch.randn((r, N), device="cuda", generator=g)).to(torch.bfloat16)
+                        for M in Ms:
+                            layer = QuaffLinear(W, O, A, B, 1.0, 0.2, M)
+                            X = torch.randn((M, K), device="cuda", generator=g)
+                            X[:, O.long()] *= mag
+                            X = X.to(torch.bfloat16)
+                            dY = (0.01 * torch.randn((M, N), device="cuda", generator=g)).to(torch.bfloat16)
+
+                            def body():
+                                layer.forward(X)
+                                layer.backward(dY)
+
+                            n0 = Q.quaff_debug_launch_count()
+                            body()                                        # warm-up step (also sets function attributes)
+                            per_step = Q.quaff_debug_launch_count() - n0
+                            torch.cuda.synchronize()
+                            graph = StepGraph(body)
+                            flush.zero_()                                 # the first timed step starts from cold HBM data
+                            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                            e0.record()
+                            for _ in range(steps):
+                                graph.replay()
+                            e1.record()
+                            torch.cuda.synchronize()
+                            assert int(layer.status[0].item()) == 0, "device-side wait timed out"
+                            ms = e0.elapsed_time(e1) / steps
+                            launches += per_step * steps
+                            fwd = 2.0 * M * N * (K + nOp + r)
+                            bwd = 2.0 * M * N * (K + nOp) + 2.0 * M * K * r
+                            # against a step whose forward ran at the INT8 rate and whose grad-input ran at the bf16 rate
+                            t_roof = (fwd / (2.0 * peaks["bf16_tflops"]) + bwd / peaks["bf16_tflops"]) / 1e12 * 1e3
+                            points.append({"M": M, "K": K, "N": N, "r": r, "frac": frac, "nO": nO, "ms_per_step": round(ms, 5),
+                                           "tokens_per_s": round(M / (ms * 1e-3), 1), "tera_ops_per_s": round((fwd + bwd) / (ms * 1e-3) / 1e12, 1),
+                                           "frac_of_gemm_roofline": round(t_roof / ms, 4)})
+                            del graph, layer, X, dY
+    fr = [p["frac_of_gemm_roofline"] for p in points]
+    line = {"workload": "sweep", "metric": METRIC, "unit": UNIT, "n_gpus": 1, "points": len(points), "steps_per_point": steps,
+            "warmup_per_point": 1, "data": "synthetic (drawn on the device)", "gpu_launches": int(launches), "clocks": clocks.summary(),
+            "roofline_of_a_point": "time of the forward's INT8 ops at 2x the measured bf16 burst peak plus the grad-input's bf16 flops at that "
+                                   "peak, over the measured step (everything else of the step - quantization, LoRA GEMMs - counts as overhead)",
+            "frac_of_gemm_roofline": {"min": min(fr), "median": float(np.median(fr)), "max": max(fr)},
+            "columns": ["M", "K", "N", "r", "frac", "nO", "ms_per_step", "tokens_per_s", "tera_ops_per_s", "frac_of_gemm_roofline"],
+            "table": [[p[c] for c in ("M", "K", "N", "r", "frac", "nO", "ms_per_step", "tokens_per_s", "tera_ops_per_s", "frac_of_gemm_roofline")]
+                      for p in points]}
+    print(json.dumps(line), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--micro", default=None, choices=["quant_act", "momentum", "requant", "outlier_count", "lora_down", "fwd", "bwd"],
@@ -577,10 +699,12 @@ def main():
     ap.add_argument("--micro-shape", type=lambda v: tuple(int(x) for x in v.split(",")), default=(8192, 11008, 4096, 55),
                     help="M,K,N,nO of --micro (default: the LLaMA-2-7B down_proj rows)")
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=1000)
+    ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--micro-rank", type=int, default=64, help="LoRA rank of --micro fwd / bwd")
-    ap.add_argument("--workload", default="phi3_attn", choices=sorted(synth.WORKLOADS))
+    ap.add_argument("--workload", default="llama7b_block", choices=sorted(synth.WORKLOADS) + ["sweep"])
+    ap.add_argument("--sweep-quick", action="store_true", help="--workload sweep on a 2 x 2 x 2 corner of the (M, K, N) grid only")
+    ap.add_argument("--repeats", type=int, default=30, help="how often the timed region of --steps steps is repeated (median reported)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--sample-tokens", type=int, default=128, help="tokens per step of the CPU oracle (reference arm); the cpu_baseline leg uses 8x this")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -588,13 +712,15 @@ def main():
     ap.add_argument("--fwd-tile", type=int, default=0, choices=[0, 128, 192, 256],
                     help="force the forward kernel's output-column tile (0: the library's cost model decides)")
     args = ap.parse_args()
+    if args.workload == "sweep":
+        return run_sweep(args)
     wl = synth.WORKLOADS[args.workload]
     if args.fwd_tile and args.impl != "reference":
         from paper_2505_14742_b200 import binding, build
         build.build_library()
         binding.quaff_debug_force_fwd_tile(args.fwd_tile)
     if args.micro:
-        if args.steps == 1000:
+        if args.steps == 20:
             args.steps = 30
         return run_micro(args)
     if args.impl == "reference":

@@ -17,10 +17,19 @@
  *  - bf16 data are raw 16-bit patterns (quaff_bf16); INT8 codes are symmetric in [-127, 127].
  *  - Scratch memory comes from the caller (`ws`, `ws_bytes`); quaff_workspace_bytes() gives
  *    the size each entry point needs.  A workspace may be shared by calls on one stream.
- *  - Return value: QUAFF_OK or an error code; on error nothing has been launched.
- *    A device-side wait that gave up is reported through the optional `status` word
+ *  - Return value: QUAFF_OK or an error code.  Arguments are checked, and every tensor map is built, before the
+ *    first launch: an argument error (codes 1-4) means nothing has been launched.  QUAFF_ERR_CUDA may come from a
+ *    launch in the middle of a call; what was enqueued before it stays enqueued, every stream the call forked is
+ *    joined back into `stream`, and the outputs are undefined.
+ *    A device-side wait that gave up (after about two seconds) is reported through the optional `status` word
  *    (QUAFF_ERR_TIMEOUT) after the stream has been synchronised; outputs are then undefined.
  *  - Inputs must be finite.  Results are deterministic (no floating-point atomics).
+ *  - The outlier set: 0 <= nO <= K and nO <= 4096 in every entry point that takes one (more: QUAFF_ERR_UNSUPPORTED_SHAPE).
+ *  - Threads: every entry point may be called from several host threads at once, on the same or on different
+ *    devices and streams (lazily created per-device resources are guarded; quaff_qlinear_bwd calls on one device are
+ *    enqueued one after the other).  The usual CUDA rule remains: calls that share an output, a workspace or the
+ *    built-in scratch of quaff_momentum_update_static must be ordered by the caller.  The library keeps no state
+ *    that changes results between calls; the only switches are the per-thread measurement aids at the end of this file.
  */
 #ifndef QUAFF_H_
 #define QUAFF_H_
@@ -73,7 +82,7 @@ quaff_status_t quaff_outlier_count(const quaff_bf16* X, int64_t ldx, int M, int 
                                    void* ws, size_t ws_bytes, quaff_stream_t stream);
 
 /*
- * The outlier set O from the counts of Eq. 6 ("selecting outlier channels o based on xi_o"): the nO channels
+ * The outlier set O from the counts of Eq. 6 (Sec. 3.3, weight preprocessing): the nO channels
  * with the largest xi, ties going to the lower channel index, written as a sorted index set.
  *   xi [K] int32 (in);  O_idx [nO] int32 (out, ascending);  nO <= K is the layer's budget;  ws: QUAFF_WS_CALIBRATE bytes
  */
@@ -122,6 +131,21 @@ quaff_status_t quaff_momentum_update(const quaff_bf16* X, int64_t ldx, int M, in
                                      void* ws, size_t ws_bytes, quaff_stream_t stream);
 
 /*
+ * The same update in two halves, for a batch whose tokens are spread over several GPUs (the paper runs on one):
+ * each GPU takes the column maxima of its own rows, the trainer combines them with an elementwise MAX all-reduce
+ * (the maximum over all rows is the maximum of the per-shard maxima, so s_O comes out bit-identical to the
+ * single-GPU update), and every GPU applies Eq. 8 and Eq. 7 to the combined maxima.
+ *   quaff_outlier_colmax:  colmax_O[i] = max_m |X[m][O_i]|   ([nO] f32, out);  ws: QUAFF_WS_MOMENTUM bytes
+ *   quaff_momentum_apply:  beta_i = max(1, sqrt(colmax_O[i] / wmax_O[i]))  (1 if wmax_O[i] = 0);
+ *                          s_O[i] <- gamma * s_O[i] + (1 - gamma) * beta_i;  beta_O_opt [nO] optional
+ * nO = 0 is a no-op in both.
+ */
+quaff_status_t quaff_outlier_colmax(const quaff_bf16* X, int64_t ldx, int M, int K, const int32_t* O_idx, int nO,
+                                    float* colmax_O, void* ws, size_t ws_bytes, quaff_stream_t stream);
+quaff_status_t quaff_momentum_apply(const float* colmax_O, const float* wmax_O, int nO, float gamma, float* s_O,
+                                    float* beta_O_opt, quaff_stream_t stream);
+
+/*
  * Scale and quantize the activations (Eq. 5: Xhat = X s^-1, s_i = 1 off O; Eq. 1 per token).
  *   Xhat[m][O_i] = X[m][O_i] / s_O[i];  dx[m] = max_k|Xhat[m][k]| / 127;
  *   Xq[m][k] = round_to_nearest_even(Xhat[m][k] * (127 / max_k|Xhat[m][k]|)), clamped to +-127
@@ -137,8 +161,8 @@ quaff_status_t quaff_quant_act(const quaff_bf16* X, int64_t ldx, int M, int K,
                                float* dx, quaff_stream_t stream);
 
 /*
- * Re-quantize the scaled outlier rows of the weight (Eq. 5: what = (s_O - 1) W_O; Eq. 1 per
- * output channel; Sec. 3.1 "computing what in real time"):
+ * Re-quantize the scaled outlier rows of the weight, every step (Eq. 5: what = (s_O - 1) W_O; Eq. 1 per
+ * output channel; Sec. 3.1):
  *   what[i][n] = (s_O[i] - 1) * W_O[i][n];  dw_O[n] = max_i|what[i][n]| / 127;
  *   wq_O[n][i] = round_to_nearest_even(what[i][n] * (127 / max_i|what[i][n]|)), 0 for i >= nO
  *   W_O [nO][N] bf16, ldwo (in);  s_O [nO] f32 (in)
@@ -204,13 +228,15 @@ quaff_status_t quaff_qlinear_fwd(int M, int K, int N,
  *   dA = X^T G  [K][r] f32 ;  dB = lora_scale * T^T dY  [r][N] f32   (nullable pair; accumulate != 0 adds)
  *   dY [M][N] bf16, lddy (lddy % 8 == 0);  T [M][r] bf16 from the forward
  *   Wq, wq_O: 16-byte aligned, ldwq_main and ldwq multiples of 16 (as in the forward)
+ *   G_out_opt [M][r] bf16 (dense, 16-byte aligned), optional: receives G (otherwise G lives in the workspace only)
  *   ws: QUAFF_WS_BWD bytes;  status_opt as in the forward.
- * Independent parts of the backward are forked onto two library-owned side streams per device (lowest priority) and
- * joined back into `stream` before the call returns its last launch: for the caller everything is still ordered on
+ * Independent parts of the backward are forked onto two library-owned side streams (lowest priority) and
+ * joined back into `stream` before the call returns: for the caller everything is still ordered on
  * `stream`.  The weight dequantization runs beside G in front of the grad-input GEMM; dA and dB are enqueued behind the
- * GEMM without depending on it, so that their split-K CTAs run in the SMs the GEMM's last wave leaves idle.  The side
- * streams are created by the first backward call on a device (make that call outside any stream capture); under
- * capture the forks become parallel branches of the captured graph.
+ * GEMM without depending on it, so that their split-K CTAs run in the SMs the GEMM's last wave leaves idle.  Each device
+ * has four sets of side streams, created by the first backward call on that device (make that call outside any stream
+ * capture).  Under capture the forks become parallel branches of the captured graph, and a set stays with its capture
+ * until the capture ends; with more than four captures open at once on one device, further calls run unforked.
  */
 quaff_status_t quaff_qlinear_bwd(int M, int K, int N,
                                  const quaff_bf16* dY, int64_t lddy,
@@ -220,7 +246,7 @@ quaff_status_t quaff_qlinear_bwd(int M, int K, int N,
                                  const quaff_bf16* X, int64_t ldx, const quaff_bf16* T,
                                  const quaff_bf16* A, const quaff_bf16* B, int r, float lora_scale,
                                  quaff_bf16* dX, int64_t lddx,
-                                 float* dA, float* dB, int accumulate,
+                                 float* dA, float* dB, int accumulate, quaff_bf16* G_out_opt,
                                  int32_t* status_opt, void* ws, size_t ws_bytes, quaff_stream_t stream);
 
 /*
@@ -234,9 +260,9 @@ quaff_status_t quaff_qlinear_bwd(int M, int K, int N,
  * scratch (column maxima and a block counter) lives in a fixed array compiled into the library, so
  * this entry point calls no cudaMalloc, cudaFree or allocating library routine.
  *
- *  - Limit: nO <= 4096 outlier channels (16 KB + 4 B of device memory, held by every GPU that loads
- *    the library until the process exits).  A larger nO returns QUAFF_ERR_UNSUPPORTED_SHAPE; use
- *    quaff_momentum_update with a workspace then.
+ *  - Limit: nO <= 4096 outlier channels, the limit of every entry point (16 KB + 4 B of device memory,
+ *    held by every GPU that loads the library until the process exits).  A larger nO returns
+ *    QUAFF_ERR_UNSUPPORTED_SHAPE here as in quaff_momentum_update.
  *  - The first call on each device looks up the array's device address (cudaGetSymbolAddress, with
  *    that device current) and caches it.  Make that first call outside any stream capture.
  *  - All calls on a device share the one array.  Each call clears what must start at zero, but two
@@ -249,16 +275,18 @@ quaff_status_t quaff_momentum_update_static(const quaff_bf16* X, int64_t ldx, in
                                             quaff_stream_t stream);
 
 /*
- * Measurement aids (no counterpart in the paper; process-wide state, not thread-safe).
+ * Measurement aids (no counterpart in the paper).  The two switches are PER HOST THREAD: they affect only later calls
+ * made by the thread that set them, so no other caller's kernel choice or stream contents can change under it.
  *
- * quaff_debug_launch_count: number of kernels this library has launched since it was loaded.
+ * quaff_debug_launch_count: number of kernels this library has launched since it was loaded (all threads).
  *
  * quaff_debug_force_fwd_tile: quaff_qlinear_fwd picks the output-column tile of its kernel (128, 192 or 256) by a
- * cost model; tile_n = 128 / 192 / 256 forces that kernel where the shape allows it (outlier set or LoRA present,
- * nOp <= 128), 0 gives the choice back to the cost model.  For tests and timing of each kernel on the same shape.
+ * cost model; tile_n = 128 / 192 / 256 forces that kernel for the calling thread where the shape allows it (outlier set
+ * or LoRA present, nOp <= 128), 0 gives the choice back to the cost model.  For tests and timing of each kernel on
+ * the same shape.
  *
  * quaff_debug_time_gemm: arm a one-shot pair of CUDA events (cudaEvent_t, created by the caller
- * with timing enabled) around the next launch of the forward (which = 0) or grad-input
+ * with timing enabled) around the calling thread's next launch of the forward (which = 0) or grad-input
  * (which = 1) tensor-core GEMM kernel: `start` is recorded on the launch stream right before the
  * kernel, `stop` right after, then the pair is disarmed.  Null events disarm.  If the stream is being
  * captured into a CUDA graph, the pair becomes two event-record nodes of that graph: every replay records

@@ -25,7 +25,7 @@ QUAFF_BF16, QUAFF_F32 = 0, 1
 QUAFF_WS_PREPARE, QUAFF_WS_MOMENTUM, QUAFF_WS_FWD, QUAFF_WS_BWD, QUAFF_WS_CALIBRATE, QUAFF_WS_HITS = 0, 1, 2, 3, 4, 5
 
 EXPORTS = ("quaff_status_string", "quaff_workspace_bytes", "quaff_debug_launch_count", "quaff_debug_force_fwd_tile", "quaff_debug_time_gemm", "quaff_prepare_weight", "quaff_momentum_update", "quaff_lora_down", "quaff_outlier_count", "quaff_select_outliers", "quaff_outlier_hits",
-           "quaff_momentum_update_static", "quaff_quant_act", "quaff_requant_weight_rows", "quaff_qlinear_fwd", "quaff_qlinear_bwd")
+           "quaff_momentum_update_static", "quaff_outlier_colmax", "quaff_momentum_apply", "quaff_quant_act", "quaff_requant_weight_rows", "quaff_qlinear_fwd", "quaff_qlinear_bwd")
 
 _lib = None
 _vp, _i64, _i32, _f32, _sz = ctypes.c_void_p, ctypes.c_int64, ctypes.c_int, ctypes.c_float, ctypes.c_size_t
@@ -60,6 +60,10 @@ def lib() -> ctypes.CDLL:
         L.quaff_momentum_update.argtypes = [_vp, _i64, _i32, _i32, _vp, _i32, _vp, _f32, _vp, _vp, _vp, _vp, _sz, _vp]
         L.quaff_momentum_update_static.restype = _i32
         L.quaff_momentum_update_static.argtypes = [_vp, _i64, _i32, _i32, _vp, _i32, _vp, _f32, _vp, _vp, _vp, _vp]
+        L.quaff_outlier_colmax.restype = _i32
+        L.quaff_outlier_colmax.argtypes = [_vp, _i64, _i32, _i32, _vp, _i32, _vp, _vp, _sz, _vp]
+        L.quaff_momentum_apply.restype = _i32
+        L.quaff_momentum_apply.argtypes = [_vp, _vp, _i32, _f32, _vp, _vp, _vp]
         L.quaff_quant_act.restype = _i32
         L.quaff_quant_act.argtypes = [_vp, _i64, _i32, _i32, _vp, _i32, _vp, _vp, _i64, _vp, _i64, _i32, _vp, _vp]
         L.quaff_requant_weight_rows.restype = _i32
@@ -77,7 +81,7 @@ def lib() -> ctypes.CDLL:
                                         _vp, _i64, _vp, _vp, _i32, _f32, _vp, _vp, _i32, _i64, _vp, _vp, _vp, _vp, _sz, _vp]
         L.quaff_qlinear_bwd.restype = _i32
         L.quaff_qlinear_bwd.argtypes = [_i32, _i32, _i32, _vp, _i64, _vp, _i64, _vp, _vp, _i64, _vp, _i32, _vp, _i32, _vp,
-                                        _vp, _i64, _vp, _vp, _vp, _i32, _f32, _vp, _i64, _vp, _vp, _i32, _vp, _vp, _sz, _vp]
+                                        _vp, _i64, _vp, _vp, _vp, _i32, _f32, _vp, _i64, _vp, _vp, _i32, _vp, _vp, _vp, _sz, _vp]
         L.quaff_debug_launch_count.restype = ctypes.c_uint64
         L.quaff_debug_launch_count.argtypes = []
         L.quaff_debug_force_fwd_tile.restype = None
@@ -176,6 +180,21 @@ def quaff_momentum_update_static(X, O_idx, wmax_O, gamma: float, s_O, colmax_O=N
            "quaff_momentum_update_static")
 
 
+def quaff_outlier_colmax(X, O_idx, colmax_O, ws) -> None:
+    """Column maxima of this GPU's rows over the outlier channels (first half of a token-sharded scale update)."""
+    M, K = X.shape
+    nO = 0 if O_idx is None else O_idx.numel()
+    _check(lib().quaff_outlier_colmax(_ptr(X), _ld(X), M, K, _ptr(O_idx), nO, _ptr(colmax_O), _ptr(ws),
+                                      ws.numel() * ws.element_size() if ws is not None else 0, _stream()), "quaff_outlier_colmax")
+
+
+def quaff_momentum_apply(colmax_O, wmax_O, gamma: float, s_O, beta_O=None) -> None:
+    """Eq. 8 and Eq. 7 from given (all-reduced) column maxima."""
+    nO = 0 if colmax_O is None else colmax_O.numel()
+    _check(lib().quaff_momentum_apply(_ptr(colmax_O), _ptr(wmax_O), nO, float(gamma), _ptr(s_O), _ptr(beta_O), _stream()),
+           "quaff_momentum_apply")
+
+
 def quaff_quant_act(X, O_idx, s_O, Xq, xq_O, dx) -> None:
     M, K = X.shape
     nO = 0 if O_idx is None else O_idx.numel()
@@ -217,7 +236,7 @@ def quaff_qlinear_fwd(Xq, xq_O, dx, Wq, dW, wq_O, dw_O, X, A, B, lora_scale: flo
 
 
 def quaff_qlinear_bwd(dY, Wq, dW, wq_O, dw_O, O_idx, s_O, X, T, A, B, lora_scale: float, dX, dA, dB,
-                      accumulate: bool, ws, status=None) -> None:
+                      accumulate: bool, ws, status=None, G_out=None) -> None:
     M, N = dY.shape
     K = Wq.shape[1]
     nOp = 0 if wq_O is None else wq_O.shape[1]
@@ -227,6 +246,6 @@ def quaff_qlinear_bwd(dY, Wq, dW, wq_O, dw_O, O_idx, s_O, X, T, A, B, lora_scale
                                    _ld(wq_O) if wq_O is not None else 0, _ptr(dw_O), nOp, _ptr(O_idx), nO, _ptr(s_O),
                                    _ptr(X), _ld(X) if X is not None else 0, _ptr(T), _ptr(A), _ptr(B), r,
                                    float(lora_scale), _ptr(dX), _ld(dX) if dX is not None else 0, _ptr(dA), _ptr(dB),
-                                   1 if accumulate else 0, _ptr(status), _ptr(ws),
+                                   1 if accumulate else 0, _ptr(G_out), _ptr(status), _ptr(ws),
                                    ws.numel() * ws.element_size() if ws is not None else 0, _stream()),
            "quaff_qlinear_bwd")

@@ -6,6 +6,7 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <atomic>
 #include <utility>
 
 #include "../../include/quaff.h"
@@ -22,11 +23,11 @@ inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 
 inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
 inline size_t round_up(size_t a, size_t b) { return (a + b - 1) / b * b; }
 
-extern unsigned long long g_launch_count;  // kernels launched by this library (diagnostics)
+extern std::atomic<unsigned long long> g_launch_count;  // kernels launched by this library (diagnostics)
 
 // Call right after every kernel launch: counts it and turns a launch error into a status.
 inline quaff_status_t launch_status() {
-    ++g_launch_count;
+    g_launch_count.fetch_add(1, std::memory_order_relaxed);
     return cudaGetLastError() == cudaSuccess ? QUAFF_OK : QUAFF_ERR_CUDA;
 }
 
@@ -120,22 +121,42 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
     return ok != 0;
 }
 
-// Bounded wait.  Every wait in these kernels goes through here: after `kWaitLimit` failed polls
-// (seconds of wall time) the waiter raises the CTA-wide abort flag and reports failure, so that a
-// broken pipeline ends with an error status instead of hanging the device.  Other waiters see the
-// flag and give up as well.
-constexpr uint32_t kWaitLimit = 1u << 24;
-static __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+// Bounded wait.  Every wait in these kernels goes through here.  The slow path gives up kWaitNs of wall time
+// (%globaltimer) after it was entered, or after kWaitLimit polls, whichever comes first: the waiter raises the abort
+// flag of its CTA - and, in a CTA pair, of its partner, through the partner's shared::cluster address - and reports
+// failure, so that a broken pipeline ends with an error status instead of hanging the device.  Every other waiter
+// of the CTA (pair) sees the flag within 1024 polls and gives up as well, so the pair drains together.
+struct AbortCtl {
+    int flag;            // set by whoever gave up
+    uint32_t peer;       // shared::cluster address of the partner CTA's `flag`, 0 outside a CTA pair
+};
+constexpr uint32_t kWaitLimit = 1u << 26;
+constexpr uint64_t kWaitNs = 2000000000ull;      // 2 s
+__device__ __forceinline__ uint64_t global_timer_ns() {
+    uint64_t t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+__device__ __forceinline__ void raise_abort(volatile AbortCtl* ctl) {
+    ctl->flag = 1;
+    const uint32_t peer = ctl->peer;
+    if (peer) asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(peer), "r"(1u) : "memory");
+}
+static __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile AbortCtl* ctl) {
+    const uint64_t t0 = global_timer_ns();
     for (uint32_t it = 0; it < kWaitLimit; ++it) {
         if (mbar_try_wait(bar, parity)) return true;
-        if ((it & 1023u) == 1023u && *abort_flag) return false;
+        if ((it & 1023u) == 1023u) {
+            if (ctl->flag) return false;
+            if (global_timer_ns() - t0 > kWaitNs) break;
+        }
     }
-    *abort_flag = 1;
+    raise_abort(ctl);
     return false;
 }
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile AbortCtl* ctl) {
     if (mbar_try_wait(bar, parity)) return true;   // fast path: keeps the issue loops of the single-thread roles short
-    return mbar_wait_slow(bar, parity, abort_flag);
+    return mbar_wait_slow(bar, parity, ctl);
 }
 
 // ------------------------------------------------------------------ PTX: TMA (no multicast anywhere)

@@ -37,7 +37,7 @@ struct Fwd192Smem {
     uint64_t empty[kMaxStages];
     uint64_t tmem_full, tmem_empty, aux_ready, aux_free;
     uint32_t tmem_base;
-    int abort_flag;
+    AbortCtl abort;
 };
 
 constexpr int kF192Fixed = 1024 + 256 + kF192ScaleBytes;      // alignment slack, barrier block (padded), scales
@@ -99,7 +99,7 @@ __global__ void __launch_bounds__(kF192Threads, 1) fwd192_kernel(const __grid_co
     unsigned char* aligned = smem_dyn + (tiles_base - raw);
     Fwd192Smem* sm = reinterpret_cast<Fwd192Smem*>(aligned + (size_t)kStages * kStageBytes);
     float* scales = reinterpret_cast<float*>(reinterpret_cast<unsigned char*>(sm) + 256);   // [2][dW | dw_O][TN]
-    volatile int* abort_flag = &sm->abort_flag;
+    volatile AbortCtl* abort_flag = &sm->abort;
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
@@ -122,7 +122,8 @@ __global__ void __launch_bounds__(kF192Threads, 1) fwd192_kernel(const __grid_co
         mbar_init(tmem_empty_bar, 8 * 2);       // eight epilogue warps in each CTA of the pair
         mbar_init(aux_ready_bar, 1);
         mbar_init(aux_free_bar, 8 * 2);
-        sm->abort_flag = 0;
+        sm->abort.flag = 0;
+        sm->abort.peer = mapa_shared(smem_u32(&sm->abort.flag), rank ^ 1u);
         fence_barrier_init();
     }
     if (warp == 1) {
@@ -333,7 +334,7 @@ __global__ void __launch_bounds__(kF192Threads, 1) fwd192_kernel(const __grid_co
     // ---------------------------------------------------------------------- common exit
     tc_fence_before();
     __syncthreads();
-    if (*abort_flag) {
+    if (abort_flag->flag) {
         for (int i = 0; i < 1000; ++i) __nanosleep(1000);   // let copies in flight land before the CTA retires
         if (threadIdx.x == 0 && p.status) atomicExch(p.status, (int)QUAFF_ERR_TIMEOUT);
         __syncthreads();

@@ -42,7 +42,7 @@ struct Fwd256Smem {
     uint64_t empty[kMaxStages];
     uint64_t tmem_full, tmem_empty, aux_ready, aux_free;
     uint32_t tmem_base;
-    int abort_flag;
+    AbortCtl abort;
 };
 
 constexpr int kF256Fixed = 1024 + 256 + kF256ScaleBytes;    // alignment slack, barrier block (padded), scales
@@ -79,7 +79,7 @@ __global__ void __launch_bounds__(kF256Threads, 1) fwd256_kernel(const __grid_co
     unsigned char* aligned = smem_dyn + (tiles_base - raw);
     Fwd256Smem* sm = reinterpret_cast<Fwd256Smem*>(aligned + (size_t)kStages * kStageBytes);
     float* scales = reinterpret_cast<float*>(reinterpret_cast<unsigned char*>(sm) + 256);   // [epilogue warp][dW | dw_O][round][32]
-    volatile int* abort_flag = &sm->abort_flag;
+    volatile AbortCtl* abort_flag = &sm->abort;
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
@@ -102,7 +102,8 @@ __global__ void __launch_bounds__(kF256Threads, 1) fwd256_kernel(const __grid_co
         mbar_init(tmem_empty_bar, kF256EpiWarps * 2);       // every epilogue warp of both CTAs
         mbar_init(aux_ready_bar, 1);
         mbar_init(aux_free_bar, kF256EpiWarps * 2);
-        sm->abort_flag = 0;
+        sm->abort.flag = 0;
+        sm->abort.peer = mapa_shared(smem_u32(&sm->abort.flag), rank ^ 1u);
         fence_barrier_init();
     }
     if (warp == 1) {
@@ -373,7 +374,7 @@ __global__ void __launch_bounds__(kF256Threads, 1) fwd256_kernel(const __grid_co
     // ---------------------------------------------------------------------- common exit
     tc_fence_before();
     __syncthreads();
-    if (*abort_flag) {
+    if (abort_flag->flag) {
         for (int i = 0; i < 1000; ++i) __nanosleep(1000);   // let copies in flight land before the CTA retires
         if (threadIdx.x == 0 && p.status) atomicExch(p.status, (int)QUAFF_ERR_TIMEOUT);
         __syncthreads();

@@ -4,6 +4,9 @@
 #include <stdlib.h>
 #include <string.h>
 
+#include <atomic>
+#include <mutex>
+
 #include "fwd256.cuh"
 
 namespace quaff {
@@ -14,14 +17,14 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
 static EncodeTiledFn encode_tiled_fn() {
-    static EncodeTiledFn fn = nullptr;
-    if (!fn) {
+    static const EncodeTiledFn fn = [] {      // initialised once, whichever thread comes first
         void* sym = nullptr;
         cudaDriverEntryPointQueryResult q;
         if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &q) == cudaSuccess &&
             q == cudaDriverEntryPointSuccess)
-            fn = reinterpret_cast<EncodeTiledFn>(sym);
-    }
+            return reinterpret_cast<EncodeTiledFn>(sym);
+        return static_cast<EncodeTiledFn>(nullptr);
+    }();
     return fn;
 }
 
@@ -43,53 +46,89 @@ quaff_status_t make_tmap_2d(CUtensorMap* map, const void* base, int elem_bytes, 
 
 // Side streams of the backward: work that does not depend on each other (the dequantization of the weight,
 // G = dY B^T, dB = T^T dY; later the outlier fix-up and dA = X^T G) is forked from the caller's stream onto
-// these and joined back with events, so the small kernels overlap instead of queueing.  One set per device,
-// created at the first backward call on that device; under stream capture the forks become parallel
-// branches of the graph.
-struct SideStreams {
+// these and joined back with events, so the small kernels overlap instead of queueing.  Each device has a small
+// pool of SETS (two streams and their events), created by the first backward call on that device.  A call takes
+// a set for the time it enqueues its work, under the device's mutex: outside stream capture any set will do (an
+// event may be re-recorded once the wait that refers to it has been enqueued); a set whose streams have been drawn
+// into a capture stays with that capture until it ends.  Calls from several host threads are therefore safe; they
+// are enqueued one after the other.
+constexpr int kSideSets = 4;
+struct SideSet {
     cudaStream_t s[2];
     cudaEvent_t fork[2], join[2], g_ready;
-    bool ok;
 };
-static SideStreams* side_streams() {
-    static SideStreams per_dev[64];
-    static bool tried[64] = {false};
+struct DeviceSide {
+    std::once_flag once;
+    std::mutex mu;          // held while a backward call enqueues its work
+    bool ok = false;
+    SideSet set[kSideSets];
+};
+static DeviceSide* device_side() {
+    static DeviceSide per_dev[64];
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
-    SideStreams& ss = per_dev[dev];
-    if (!tried[dev]) {
-        tried[dev] = true;
-        ss.ok = true;
+    DeviceSide& ds = per_dev[dev];
+    std::call_once(ds.once, [&ds] {
+        bool ok = true;
         // lowest priority, so that the side work never outranks the caller's stream (a default stream has the same
         // priority: there the launch order decides, which is why the backward enqueues dA and dB behind its GEMM)
         int least = 0, greatest = 0;
         cudaDeviceGetStreamPriorityRange(&least, &greatest);
-        ss.ok = ss.ok && cudaEventCreateWithFlags(&ss.g_ready, cudaEventDisableTiming) == cudaSuccess;
-        for (int i = 0; i < 2; ++i) {
-            ss.ok = ss.ok && cudaStreamCreateWithPriority(&ss.s[i], cudaStreamNonBlocking, least) == cudaSuccess;
-            ss.ok = ss.ok && cudaEventCreateWithFlags(&ss.fork[i], cudaEventDisableTiming) == cudaSuccess;
-            ss.ok = ss.ok && cudaEventCreateWithFlags(&ss.join[i], cudaEventDisableTiming) == cudaSuccess;
+        for (int k = 0; k < kSideSets; ++k) {
+            SideSet& ss = ds.set[k];
+            ok = ok && cudaEventCreateWithFlags(&ss.g_ready, cudaEventDisableTiming) == cudaSuccess;
+            for (int i = 0; i < 2; ++i) {
+                ok = ok && cudaStreamCreateWithPriority(&ss.s[i], cudaStreamNonBlocking, least) == cudaSuccess;
+                ok = ok && cudaEventCreateWithFlags(&ss.fork[i], cudaEventDisableTiming) == cudaSuccess;
+                ok = ok && cudaEventCreateWithFlags(&ss.join[i], cudaEventDisableTiming) == cudaSuccess;
+            }
         }
-        if (!ss.ok) cudaGetLastError();
+        if (!ok) cudaGetLastError();
+        ds.ok = ok;
+    });
+    return ds.ok ? &ds : nullptr;
+}
+// A set this call on stream `st` may use (the device's mutex is held): one whose streams belong to the capture `st`
+// is part of, else one that is in no capture; null if every set is tied to some other capture.
+static SideSet* pick_side_set(DeviceSide* ds, cudaStream_t st) {
+    cudaStreamCaptureStatus mine = cudaStreamCaptureStatusNone;
+    unsigned long long my_id = 0;
+    if (cudaStreamGetCaptureInfo(st, &mine, &my_id) != cudaSuccess) { cudaGetLastError(); return nullptr; }
+    SideSet* free_set = nullptr;
+    for (int k = 0; k < kSideSets; ++k) {
+        SideSet* ss = &ds->set[k];
+        bool in_capture = false, same = true;
+        for (int i = 0; i < 2; ++i) {
+            cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
+            unsigned long long id = 0;
+            if (cudaStreamGetCaptureInfo(ss->s[i], &cs, &id) != cudaSuccess) { cudaGetLastError(); in_capture = true; same = false; continue; }
+            if (cs != cudaStreamCaptureStatusNone) {
+                in_capture = true;
+                if (cs != cudaStreamCaptureStatusActive || mine != cudaStreamCaptureStatusActive || id != my_id) same = false;
+            }
+        }
+        if (in_capture && same) return ss;              // already part of this capture
+        if (!in_capture && !free_set) free_set = ss;
     }
-    return ss.ok ? &ss : nullptr;
+    return free_set;
 }
 // side stream i continues from the current end of `st` / `st` continues after side stream i
-static bool fork_to(SideStreams* ss, int i, cudaStream_t st) {
+static bool fork_to(SideSet* ss, int i, cudaStream_t st) {
     return cudaEventRecord(ss->fork[i], st) == cudaSuccess && cudaStreamWaitEvent(ss->s[i], ss->fork[i], 0) == cudaSuccess;
 }
-static bool join_from(SideStreams* ss, int i, cudaStream_t st) {
+static bool join_from(SideSet* ss, int i, cudaStream_t st) {
     return cudaEventRecord(ss->join[i], ss->s[i]) == cudaSuccess && cudaStreamWaitEvent(st, ss->join[i], 0) == cudaSuccess;
 }
 
-static cudaEvent_t g_time_start[2] = {nullptr, nullptr};
-static cudaEvent_t g_time_stop[2] = {nullptr, nullptr};
+// Measurement aids: per host thread, one-shot (see quaff.h)
+static thread_local cudaEvent_t g_time_start[2] = {nullptr, nullptr};
+static thread_local cudaEvent_t g_time_stop[2] = {nullptr, nullptr};
 
 // Tile-processing units (CTAs, or CTA pairs) that can be resident at once.
 template <int EPI, int CTAS, int TN>
 static int gemm_units(int dev) {
-    static int cached[64] = {0};
-    if (cached[dev]) return cached[dev];
+    static std::atomic<int> cached[64];
+    if (cached[dev].load()) return cached[dev].load();
     int units = sm_count() / CTAS;
     if (CTAS == 2) {
         cudaLaunchConfig_t cfg = {};
@@ -107,21 +146,21 @@ static int gemm_units(int dev) {
         else
             cudaGetLastError();
     }
-    cached[dev] = max(units, 1);
-    return cached[dev];
+    cached[dev].store(max(units, 1));     // every thread computes the same value
+    return cached[dev].load();
 }
 
 template <int EPI, int CTAS, int TN>
 static quaff_status_t launch_gemm(const GemmParams& p, cudaStream_t st) {
     using Cfg = GemmCfg<EPI, CTAS, TN>;
-    static bool configured[64] = {false};
+    static std::atomic<bool> configured[64];
     int dev = 0;
     cudaGetDevice(&dev);
     if (dev < 0 || dev >= 64) return QUAFF_ERR_CUDA;
-    if (!configured[dev]) {
+    if (!configured[dev].load()) {     // setting the attribute twice (two threads at once) is harmless
         if (cudaFuncSetAttribute(umma_gemm_kernel<EPI, CTAS, TN>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg::kSmemBytes) != cudaSuccess)
             return QUAFF_ERR_CUDA;
-        configured[dev] = true;
+        configured[dev].store(true);
     }
     const int ntiles = p.tiles_m * p.tiles_n;
     if (ntiles == 0) return QUAFF_OK;
@@ -146,15 +185,15 @@ static quaff_status_t launch_gemm(const GemmParams& p, cudaStream_t st) {
 
 // The wide forward kernels (fwd192.cuh, fwd256.cuh): which = 0 / 1
 static quaff_status_t launch_fwd_wide(int which, const FwdWideParams& p, cudaStream_t st) {
-    static bool configured[2][64] = {{false}};
-    static int units_of[2][64] = {{0}};
+    static std::atomic<bool> configured[2][64];
+    static std::atomic<int> units_of[2][64];
     void (*const kernel)(const FwdWideParams) = which ? fwd256_kernel : fwd192_kernel;
     const int threads = which ? kF256Threads : kF192Threads;
     const size_t smem = which ? kF256SmemBytes : kF192SmemBytes;
     int dev = 0;
     cudaGetDevice(&dev);
     if (dev < 0 || dev >= 64) return QUAFF_ERR_CUDA;
-    if (!configured[which][dev]) {
+    if (!configured[which][dev].load()) {
         if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return QUAFF_ERR_CUDA;
         int units = sm_count() / 2;
         cudaLaunchConfig_t cfg = {};
@@ -169,12 +208,12 @@ static quaff_status_t launch_fwd_wide(int which, const FwdWideParams& p, cudaStr
         int nclusters = 0;
         if (cudaOccupancyMaxActiveClusters(&nclusters, kernel, &cfg) == cudaSuccess && nclusters > 0) units = min(units, nclusters);
         else cudaGetLastError();
-        units_of[which][dev] = max(units, 1);
-        configured[which][dev] = true;
+        units_of[which][dev].store(max(units, 1));
+        configured[which][dev].store(true);
     }
     const int ntiles = p.tiles_m * p.tiles_n;
     if (ntiles == 0) return QUAFF_OK;
-    const int units = min(ntiles, units_of[which][dev]);
+    const int units = min(ntiles, units_of[which][dev].load());
     const bool timed = g_time_start[0] && g_time_stop[0];
     unsigned int ev_flags = cudaEventRecordDefault;
     if (timed) {
@@ -387,11 +426,13 @@ static void fill_phase(GemmPhase& ph, int is_i8, int kext, int acc_slot, int fre
 // part[s][row][j] (f32, row pitch r) = sum over the s-th slice of the contraction of A(row, :) * B(j, :).
 //   K-major  (mn_major = 0): A is [rows_out][kc] with pitch lda, B is [r][kc] with pitch ldb.
 //   MN-major (mn_major = 1): A is [kc][rows_out] with pitch lda, B is [kc][r] with pitch ldb.
-static quaff_status_t skinny_gemm(int mn_major, const void* A, int64_t lda, const void* B, int64_t ldb, int rows_out,
-                                  int kc, int r, float* part, int32_t* status, cudaStream_t st, int* S_out) {
+// skinny_prepare builds the launch parameters (tensor maps included; nothing is enqueued), skinny_launch enqueues.
+struct SkinnyGemm { GemmParams p; int S; };
+static quaff_status_t skinny_prepare(SkinnyGemm& g, int mn_major, const void* A, int64_t lda, const void* B, int64_t ldb, int rows_out,
+                                     int kc, int r, float* part, int32_t* status) {
     const SplitPlan sp = split_plan(rows_out, kc);
     const int rp = pad16(r);
-    GemmParams p;
+    GemmParams& p = g.p;
     memset(&p, 0, sizeof(p));
     GemmPhase& ph = p.ph[0];
     quaff_status_t rc;
@@ -410,11 +451,12 @@ static quaff_status_t skinny_gemm(int mn_major, const void* A, int64_t lda, cons
     p.band_m = p.tiles_m;
     p.status = status;
     p.part = part; p.part_ld = r; p.part_cols = r;
-    *S_out = sp.S;
-    return launch_gemm<EPI_PART, 1, 128>(p, st);
+    g.S = sp.S;
+    return QUAFF_OK;
 }
+static quaff_status_t skinny_launch(const SkinnyGemm& g, cudaStream_t st) { return launch_gemm<EPI_PART, 1, 128>(g.p, st); }
 
-static int g_force_fwd_tile = 0;   // quaff_debug_force_fwd_tile: 0 = the cost model decides
+static thread_local int g_force_fwd_tile = 0;   // quaff_debug_force_fwd_tile (per host thread): 0 = the cost model decides
 
 // Cost model of the three forward kernels, fitted to sweeps of the number of waves at fixed shapes (B200, clocks of
 // 1965 MHz): a tile of width W takes about  max(MMAs x kFwdMmaClk + kFwdTileOvh, kFwdTileMin)  clocks; the floor is
@@ -440,9 +482,8 @@ static FwdWorkspace fwd_workspace(int M, int K, int N, int r) {
 // Output-column tile of the grad-input GEMM: 128, 192 or 256.  A tcgen05.mma of a CTA pair costs about 60 + N/2
 // clocks (measured: N = 128: 125, 192: 165, 256: 190), so wide tiles are cheaper per column, while the width also
 // decides how full the last wave is.  Cost model: waves on the CTA pairs x cost of one MMA of that width; among equals
-// the wider tile (fewer tiles, fewer epilogues).  (The kernel takes any multiple of 16, but widths that are not a
-// multiple of 64 run far below this model - measured: 176 columns 208 clocks per MMA, 240 columns 215 - so they are
-// not candidates.)
+// the wider tile (fewer tiles, fewer epilogues).  (Widths that are not a multiple of 64 run far below this model -
+// measured: 176 columns 208 clocks per MMA, 240 columns 215 - so they are not candidates.)
 static int round_up32(int k) { return (k + 31) / 32 * 32; }
 static int bwd_tile_n(int M, int K, int nOp) {
     const int units = kPlanSMs / 2;
@@ -490,11 +531,12 @@ static quaff_status_t lora_down(const quaff_bf16* X, int64_t ldx, int M, int K, 
     float* part = reinterpret_cast<float*>(base + w.off_part);
     const int rp = pad16(r);
     quaff_status_t rc;
+    SkinnyGemm g;
+    if ((rc = skinny_prepare(g, 0, X, ldx, At, K, M, K, r, part, status_opt)) != QUAFF_OK) return rc;
     launch_pdl(transpose_pad_kernel, dim3(ceil_div(K * rp, 256)), dim3(256), 0, st, 1, A, K, r, At, K);   // At[j][k] = A[k][j]
     if ((rc = launch_status()) != QUAFF_OK) return rc;
-    int S = 1;
-    if ((rc = skinny_gemm(0, X, ldx, At, K, M, K, r, part, status_opt, st, &S)) != QUAFF_OK) return rc;
-    launch_pdl(reduce_parts_bf16_kernel, dim3(ceil_div(M * r / 8, 256)), dim3(256), 0, st, 1, part, S, M, r, 1.0f, T_out);
+    if ((rc = skinny_launch(g, st)) != QUAFF_OK) return rc;
+    launch_pdl(reduce_parts_bf16_kernel, dim3(ceil_div(M * r / 8, 256)), dim3(256), 0, st, 1, part, g.S, M, r, 1.0f, T_out);
     return launch_status();
 }
 
@@ -678,8 +720,8 @@ extern "C" quaff_status_t quaff_qlinear_bwd(int M, int K, int N, const quaff_bf1
                                             const float* dw_O, int nOp, const int32_t* O_idx, int nO, const float* s_O,
                                             const quaff_bf16* X, int64_t ldx, const quaff_bf16* T, const quaff_bf16* A,
                                             const quaff_bf16* B, int r, float lora_scale, quaff_bf16* dX, int64_t lddx,
-                                            float* dA, float* dB, int accumulate, int32_t* status_opt, void* ws,
-                                            size_t ws_bytes, quaff_stream_t stream) {
+                                            float* dA, float* dB, int accumulate, quaff_bf16* G_out_opt,
+                                            int32_t* status_opt, void* ws, size_t ws_bytes, quaff_stream_t stream) {
     QUAFF_RETURN_IF(M < 0 || K <= 0 || N <= 0 || nOp < 0 || nO < 0 || nO > nOp || r < 0, QUAFF_ERR_INVALID_ARG);
     QUAFF_RETURN_IF(!dY || lddy < N || !Wq || !dW || ldwq_main < K, QUAFF_ERR_INVALID_ARG);
     QUAFF_RETURN_IF(nOp > 0 && (!wq_O || !dw_O || ldwq < nOp), QUAFF_ERR_INVALID_ARG);
@@ -693,7 +735,7 @@ extern "C" quaff_status_t quaff_qlinear_bwd(int M, int K, int N, const quaff_bf1
     QUAFF_RETURN_IF(!aligned16(Wq) || (ldwq_main % 16), QUAFF_ERR_ALIGNMENT);
     QUAFF_RETURN_IF(nOp > 0 && (!aligned16(wq_O) || (ldwq % 16)), QUAFF_ERR_ALIGNMENT);
     QUAFF_RETURN_IF(dX && (!aligned16(dX) || (lddx % 8)), QUAFF_ERR_ALIGNMENT);
-    QUAFF_RETURN_IF(r > 0 && (!aligned16(A) || !aligned16(B)), QUAFF_ERR_ALIGNMENT);
+    QUAFF_RETURN_IF(r > 0 && (!aligned16(A) || !aligned16(B) || (G_out_opt && !aligned16(G_out_opt))), QUAFF_ERR_ALIGNMENT);
     QUAFF_RETURN_IF(r > 0 && dA && (!aligned16(X) || !aligned16(T) || !aligned16(dA) || !aligned16(dB) || (ldx % 8)), QUAFF_ERR_ALIGNMENT);
     const BwdWorkspace w = bwd_workspace(M, K, N, nOp, r);
     QUAFF_RETURN_IF(!ws || !aligned16(ws) || ws_bytes < w.total, QUAFF_ERR_WORKSPACE_TOO_SMALL);
@@ -701,44 +743,24 @@ extern "C" quaff_status_t quaff_qlinear_bwd(int M, int K, int N, const quaff_bf1
     cudaStream_t st = (cudaStream_t)stream;
     unsigned char* base = reinterpret_cast<unsigned char*>(ws);
     uint16_t* Wd = reinterpret_cast<uint16_t*>(base + w.off_wd);
-    uint16_t* G = reinterpret_cast<uint16_t*>(base + w.off_g);
+    uint16_t* G = (r > 0 && G_out_opt) ? G_out_opt : reinterpret_cast<uint16_t*>(base + w.off_g);
     float* P = reinterpret_cast<float*>(base + w.off_p);
     float* part = reinterpret_cast<float*>(base + w.off_part);
     float* part_a = reinterpret_cast<float*>(base + w.off_part_a);
     float* part_b = reinterpret_cast<float*>(base + w.off_part_b);
     quaff_status_t rc;
-    int S = 1;
     const bool want_dAB = r > 0 && dA && dB;
-    // Dependencies:  dB = T^T dY needs nothing computed here;  the weight dequantization neither;
-    // G = dY B^T feeds the grad-input GEMM and dA = X^T G;  the outlier fix-up follows the GEMM.
-    SideStreams* ss = side_streams();
-    cudaStream_t s_deq = ss ? ss->s[0] : st;       // dequantization, later dA
-    cudaStream_t s_db = ss ? ss->s[1] : st;        // dB
-    bool forked0 = false, forked1 = false;
-
-    // Launch order = the order in which the block scheduler hands out SM slots while everything below runs at once:
-    // the chain the grad-input GEMM waits for longest (G) first, then the bulk dequantization; dB and dA come behind
-    // the GEMM.  The side streams fork off before any of it, so that they depend on nothing launched here.
-    if (ss && want_dAB && !(forked1 = fork_to(ss, 1, st))) return QUAFF_ERR_CUDA;
-    if (ss && dX && !(forked0 = fork_to(ss, 0, st))) return QUAFF_ERR_CUDA;
-    if (r > 0) {   // G = bf16(lora_scale * dY B^T): B [r][N] is already K-major for this contraction over N
-        if ((rc = skinny_gemm(0, dY, lddy, B, N, M, N, r, part, status_opt, st, &S)) != QUAFF_OK) return rc;
-        launch_pdl(reduce_parts_bf16_kernel, dim3(ceil_div(M * r / 8, 256)), dim3(256), 0, st, 1, part, S, M, r, lora_scale, G);
-        if ((rc = launch_status()) != QUAFF_OK) return rc;
-        if (ss && cudaEventRecord(ss->g_ready, st) != cudaSuccess) return QUAFF_ERR_CUDA;
-    }
     constexpr int CTAS = 2;
     const int TN = w.tile_n, Kpad = w.Kpad;
     const int Kext = nOp > 0 ? Kpad + 2 * nOp : K;
-    if (dX) {
-        const int chunks = (Kpad + 2 * nOp) / 16;
-        launch_pdl(dequant_weight_kernel, dim3(N, ceil_div(chunks, 256)), dim3(256), 0, s_deq, 1, Wq, ldwq_main, dW, wq_O, ldwq, dw_O, O_idx,
-                   nO, nOp, K, Kpad, Wd, w.ldwd);
-        if ((rc = launch_status()) != QUAFF_OK) return rc;
+
+    // ---- every tensor map and launch parameter first: nothing has been enqueued when one of them fails
+    SkinnyGemm gemm_g, gemm_db, gemm_da;
+    GemmParams p;
+    if (r > 0) {   // G = bf16(lora_scale * dY B^T): B [r][N] is already K-major for this contraction over N
+        if ((rc = skinny_prepare(gemm_g, 0, dY, lddy, B, N, M, N, r, part, status_opt)) != QUAFF_OK) return rc;
     }
     if (dX) {
-        if (forked0 && !join_from(ss, 0, st)) return QUAFF_ERR_CUDA;     // the dequantized weight is ready
-        GemmParams p;
         memset(&p, 0, sizeof(p));
         int np = 0;
         {   // main: dY Wd over N; Wd [N][Kext] is MN-major for this contraction (rows = n)
@@ -766,43 +788,82 @@ extern "C" quaff_status_t quaff_qlinear_bwd(int M, int K, int N, const quaff_bf1
         p.status = status_opt;
         p.dX = dX; p.lddx = lddx; p.P = P; p.ldp = 2 * nOp;
         p.tile_n = TN;      // the 256-column instance serves every width above 128
-        rc = TN > 128 ? launch_gemm<EPI_BWD, CTAS, 256>(p, st) : launch_gemm<EPI_BWD, CTAS, 128>(p, st);
-        if (rc != QUAFF_OK) return rc;
     }
     if (want_dAB) {
-        // dB^T = dY^T T: the contraction runs over the tokens, the slow axis of dY and T: MN-major operands.  It needs
-        // nothing computed here, but it is held back (side stream 1 waits for the end of the dequantization) until the
+        // dB^T = dY^T T and dA = X^T G: the contraction runs over the tokens, the slow axis of all four matrices: MN-major operands
+        if ((rc = skinny_prepare(gemm_db, 1, dY, lddy, T, r, N, M, r, part_b, status_opt)) != QUAFF_OK) return rc;
+        if ((rc = skinny_prepare(gemm_da, 1, X, ldx, G, r, K, M, r, part_a, status_opt)) != QUAFF_OK) return rc;
+    }
+
+    // Dependencies:  dB = T^T dY needs nothing computed here;  the weight dequantization neither;
+    // G = dY B^T feeds the grad-input GEMM and dA = X^T G;  the outlier fix-up follows the GEMM.
+    DeviceSide* ds = device_side();
+    std::unique_lock<std::mutex> lock;
+    SideSet* ss = nullptr;
+    if (ds) {
+        lock = std::unique_lock<std::mutex>(ds->mu);
+        ss = pick_side_set(ds, st);
+    }
+    cudaStream_t s_deq = ss ? ss->s[0] : st;       // dequantization, later dA
+    cudaStream_t s_db = ss ? ss->s[1] : st;        // dB
+    bool forked0 = false, forked1 = false;
+    // From the first fork on, an error leaves through `leave`: whatever has been forked is joined back into the
+    // caller's stream, so that no branch stays open (a stream capture would otherwise be invalid, and a caller could
+    // reuse the workspace while a side stream still writes it).
+    auto leave = [&](quaff_status_t code) {
+        if (forked0 && !join_from(ss, 0, st) && code == QUAFF_OK) code = QUAFF_ERR_CUDA;
+        if (forked1 && !join_from(ss, 1, st) && code == QUAFF_OK) code = QUAFF_ERR_CUDA;
+        return code;
+    };
+
+    // Launch order = the order in which the block scheduler hands out SM slots while everything below runs at once:
+    // the chain the grad-input GEMM waits for longest (G) first, then the bulk dequantization; dB and dA come behind
+    // the GEMM.  The side streams fork off before any of it, so that they depend on nothing launched here.
+    if (ss && want_dAB && !(forked1 = fork_to(ss, 1, st))) return leave(QUAFF_ERR_CUDA);
+    if (ss && dX && !(forked0 = fork_to(ss, 0, st))) return leave(QUAFF_ERR_CUDA);
+    if (r > 0) {
+        if ((rc = skinny_launch(gemm_g, st)) != QUAFF_OK) return leave(rc);
+        launch_pdl(reduce_parts_bf16_kernel, dim3(ceil_div(M * r / 8, 256)), dim3(256), 0, st, 1, part, gemm_g.S, M, r, lora_scale, G);
+        if ((rc = launch_status()) != QUAFF_OK) return leave(rc);
+        if (ss && cudaEventRecord(ss->g_ready, st) != cudaSuccess) return leave(QUAFF_ERR_CUDA);
+    }
+    if (dX) {
+        const int chunks = (Kpad + 2 * nOp) / 16;
+        launch_pdl(dequant_weight_kernel, dim3(N, ceil_div(chunks, 256)), dim3(256), 0, s_deq, 1, Wq, ldwq_main, dW, wq_O, ldwq, dw_O, O_idx,
+                   nO, nOp, K, Kpad, Wd, w.ldwd);
+        if ((rc = launch_status()) != QUAFF_OK) return leave(rc);
+        if (forked0) {     // the dequantized weight is ready
+            forked0 = false;
+            if (!join_from(ss, 0, st)) return leave(QUAFF_ERR_CUDA);
+        }
+        rc = TN > 128 ? launch_gemm<EPI_BWD, CTAS, 256>(p, st) : launch_gemm<EPI_BWD, CTAS, 128>(p, st);
+        if (rc != QUAFF_OK) return leave(rc);
+    }
+    if (want_dAB) {
+        // dB needs nothing computed here, but it is held back (side stream 1 waits for the end of the dequantization) until the
         // grad-input GEMM is ready too and enqueued behind it: with the lowest priority it then runs in the SMs the GEMM
         // leaves free instead of competing with G and the dequantization for HBM in front of the GEMM.
-        if (ss && dX && cudaStreamWaitEvent(ss->s[1], ss->join[0], 0) != cudaSuccess) return QUAFF_ERR_CUDA;
-        if ((rc = skinny_gemm(1, dY, lddy, T, r, N, M, r, part_b, status_opt, s_db, &S)) != QUAFF_OK) return rc;
-        launch_pdl(reduce_parts_kernel, dim3(ceil_div(N * r / 4, 256)), dim3(256), 0, s_db, 1, part_b, S, N, r, lora_scale, 1, accumulate, dB);
-        if ((rc = launch_status()) != QUAFF_OK) return rc;
-    }
-    if (want_dAB) {
-        // dA = X^T G (MN-major operands) needs G, not the grad-input GEMM: on side stream 0 it follows the weight
-        // dequantization and waits for G only.  It is enqueued BEHIND the GEMM, so the persistent GEMM gets every SM
-        // first and the split-K CTAs of dA move in as the pairs that have no tile left in the last wave retire.
+        if (ss && dX && cudaStreamWaitEvent(ss->s[1], ss->join[0], 0) != cudaSuccess) return leave(QUAFF_ERR_CUDA);
+        if ((rc = skinny_launch(gemm_db, s_db)) != QUAFF_OK) return leave(rc);
+        launch_pdl(reduce_parts_kernel, dim3(ceil_div(N * r / 4, 256)), dim3(256), 0, s_db, 1, part_b, gemm_db.S, N, r, lora_scale, 1, accumulate, dB);
+        if ((rc = launch_status()) != QUAFF_OK) return leave(rc);
+        // dA needs G, not the grad-input GEMM: on side stream 0 it follows the weight dequantization and waits for G
+        // only.  It is enqueued BEHIND the GEMM, so the persistent GEMM gets every SM first and the split-K CTAs of dA
+        // move in as the pairs that have no tile left in the last wave retire.
         cudaStream_t s_da = st;
-        bool forked_da = false;
         if (ss && dX) {
-            if (cudaStreamWaitEvent(ss->s[0], ss->g_ready, 0) != cudaSuccess) return QUAFF_ERR_CUDA;
-            forked_da = true;
+            if (cudaStreamWaitEvent(ss->s[0], ss->g_ready, 0) != cudaSuccess) return leave(QUAFF_ERR_CUDA);
+            forked0 = true;
             s_da = ss->s[0];
         }
-        if ((rc = skinny_gemm(1, X, ldx, G, r, K, M, r, part_a, status_opt, s_da, &S)) != QUAFF_OK) return rc;
-        launch_pdl(reduce_parts_kernel, dim3(ceil_div(K * r / 4, 256)), dim3(256), 0, s_da, 1, part_a, S, K, r, 1.0f, 0, accumulate, dA);
-        if ((rc = launch_status()) != QUAFF_OK) return rc;
-        forked0 = forked_da;
-    } else {
-        forked0 = false;
+        if ((rc = skinny_launch(gemm_da, s_da)) != QUAFF_OK) return leave(rc);
+        launch_pdl(reduce_parts_kernel, dim3(ceil_div(K * r / 4, 256)), dim3(256), 0, s_da, 1, part_a, gemm_da.S, K, r, 1.0f, 0, accumulate, dA);
+        if ((rc = launch_status()) != QUAFF_OK) return leave(rc);
     }
     if (dX && nO > 0) {
         launch_pdl(bwd_fixup_kernel, dim3(ceil_div(M * nO, 256)), dim3(256), 0, st, 1, P, (int64_t)(2 * nOp), M, nO, nOp, O_idx, s_O, G, A, r,
                    dX, lddx);
-        if ((rc = launch_status()) != QUAFF_OK) return rc;
+        if ((rc = launch_status()) != QUAFF_OK) return leave(rc);
     }
-    if (forked0 && !join_from(ss, 0, st)) return QUAFF_ERR_CUDA;
-    if (forked1 && !join_from(ss, 1, st)) return QUAFF_ERR_CUDA;
-    return QUAFF_OK;
+    return leave(QUAFF_OK);
 }

@@ -9,19 +9,19 @@
 
 namespace quaff {
 
-unsigned long long g_launch_count = 0;
+std::atomic<unsigned long long> g_launch_count{0};
 
 int sm_count() {
-    static int cached[64] = {0};
+    static std::atomic<int> cached[64];
     int dev = 0;
     cudaGetDevice(&dev);
     if (dev < 0 || dev >= 64) dev = 0;
-    if (cached[dev] == 0) {
-        int n = 0;
+    int n = cached[dev].load();
+    if (n == 0) {
         if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
-        cached[dev] = n;
+        cached[dev].store(n);
     }
-    return cached[dev];
+    return n;
 }
 
 // =====================================================================================
@@ -266,56 +266,62 @@ static quaff_status_t quant_act_dispatch(const uint16_t* X, int64_t ldx, int M, 
 // channel, warp = row), reduces in shared memory and merges with an integer atomicMax on the
 // fp32 bit pattern (non-negative floats order like integers, so the result is exact and
 // order-free).  The last block to finish derives beta and updates s.
+// colmax_in != null: the maxima are given (one block; nothing is scanned).  apply = 0: the maxima are only
+// written to colmax_opt (Eq. 8 and Eq. 7 are left to a later call).
 __global__ void __launch_bounds__(256) momentum_kernel(const uint16_t* __restrict__ X, int64_t ldx, int M,
                                                        const int32_t* __restrict__ O_idx, int nO,
                                                        const float* __restrict__ wmax_O, float gamma,
                                                        float* __restrict__ s_O, float* __restrict__ colmax_opt,
-                                                       float* __restrict__ beta_opt, unsigned int* __restrict__ ws) {
+                                                       float* __restrict__ beta_opt, unsigned int* __restrict__ ws,
+                                                       const float* __restrict__ colmax_in, int apply) {
     pdl_launch_dependents();
     pdl_wait();
     __shared__ unsigned int red[8][32];
     __shared__ int is_last;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int rows_per_block = (M + gridDim.x - 1) / gridDim.x;
-    const int r0 = blockIdx.x * rows_per_block;
-    const int r1 = min(M, r0 + rows_per_block);
+    if (!colmax_in) {
+        const int rows_per_block = (M + gridDim.x - 1) / gridDim.x;
+        const int r0 = blockIdx.x * rows_per_block;
+        const int r1 = min(M, r0 + rows_per_block);
 
-    for (int c0 = 0; c0 < nO; c0 += 32) {
-        const int i = c0 + lane;
-        unsigned int best = 0;
-        if (i < nO) {
-            const uint16_t* xc = X + O_idx[i];
-            int m = r0 + warp;
-            for (; m + 24 < r1; m += 32) {     // four independent gathers in flight per thread
-                const unsigned int a = __ldg(xc + (int64_t)m * ldx), b = __ldg(xc + (int64_t)(m + 8) * ldx);
-                const unsigned int c = __ldg(xc + (int64_t)(m + 16) * ldx), d = __ldg(xc + (int64_t)(m + 24) * ldx);
-                best = max(best, max(max(a & 0x7FFFu, b & 0x7FFFu), max(c & 0x7FFFu, d & 0x7FFFu)));
+        for (int c0 = 0; c0 < nO; c0 += 32) {
+            const int i = c0 + lane;
+            unsigned int best = 0;
+            if (i < nO) {
+                const uint16_t* xc = X + O_idx[i];
+                int m = r0 + warp;
+                for (; m + 24 < r1; m += 32) {     // four independent gathers in flight per thread
+                    const unsigned int a = __ldg(xc + (int64_t)m * ldx), b = __ldg(xc + (int64_t)(m + 8) * ldx);
+                    const unsigned int c = __ldg(xc + (int64_t)(m + 16) * ldx), d = __ldg(xc + (int64_t)(m + 24) * ldx);
+                    best = max(best, max(max(a & 0x7FFFu, b & 0x7FFFu), max(c & 0x7FFFu, d & 0x7FFFu)));
+                }
+                for (; m < r1; m += 8) best = max(best, (unsigned int)__ldg(xc + (int64_t)m * ldx) & 0x7FFFu);
+                best <<= 16;                       // |x| as fp32 bits
             }
-            for (; m < r1; m += 8) best = max(best, (unsigned int)__ldg(xc + (int64_t)m * ldx) & 0x7FFFu);
-            best <<= 16;                       // |x| as fp32 bits
-        }
-        red[warp][lane] = best;
-        __syncthreads();
-        if (warp == 0) {
+            red[warp][lane] = best;
+            __syncthreads();
+            if (warp == 0) {
 #pragma unroll
-            for (int w = 1; w < 8; ++w) best = max(best, red[w][lane]);
-            if (i < nO && best) atomicMax(&ws[i], best);
+                for (int w = 1; w < 8; ++w) best = max(best, red[w][lane]);
+                if (i < nO && best) atomicMax(&ws[i], best);
+            }
+            __syncthreads();
         }
+        __threadfence();
+        if (tid == 0) is_last = (atomicAdd(&ws[nO], 1u) == gridDim.x - 1);
         __syncthreads();
+        if (!is_last) return;
+        __threadfence();
     }
-    __threadfence();
-    if (tid == 0) is_last = (atomicAdd(&ws[nO], 1u) == gridDim.x - 1);
-    __syncthreads();
-    if (!is_last) return;
-    __threadfence();
     const float one_minus_gamma = __fsub_rn(1.0f, gamma);
     for (int i = tid; i < nO; i += blockDim.x) {
-        const float cmax = __uint_as_float(*reinterpret_cast<volatile unsigned int*>(&ws[i]));
+        const float cmax = colmax_in ? colmax_in[i] : __uint_as_float(*reinterpret_cast<volatile unsigned int*>(&ws[i]));
+        if (colmax_opt) colmax_opt[i] = cmax;
+        if (!apply) continue;
         const float wmax = wmax_O[i];
         float beta = 1.0f;
         if (wmax > 0.0f) beta = fmaxf(1.0f, __fsqrt_rn(__fdiv_rn(cmax, wmax)));   // Eq. 8
         s_O[i] = __fadd_rn(__fmul_rn(gamma, s_O[i]), __fmul_rn(one_minus_gamma, beta));  // Eq. 7
-        if (colmax_opt) colmax_opt[i] = cmax;
         if (beta_opt) beta_opt[i] = beta;
     }
 }
@@ -410,9 +416,20 @@ __global__ void __launch_bounds__(256) gather_outlier_rows_kernel(const uint16_t
 constexpr int kStaticMaxNO = 4096;
 static __device__ __align__(256) unsigned int g_momentum_scratch[kStaticMaxNO + 1];
 
-static bool valid_outlier_args(const int32_t* O_idx, int nO, int K) {
-    return nO >= 0 && nO <= K && nO <= 4096 && (nO == 0 || O_idx != nullptr);
+// The outlier set of every entry point: 0 <= nO <= K, at most kStaticMaxNO channels (the row kernels stage O and
+// s_O in shared memory; the paper's largest budget, 10 % of an 11008-wide layer, is 1100).
+static quaff_status_t check_outlier_args(const int32_t* O_idx, int nO, int K) {
+    if (nO < 0 || nO > K || (nO > 0 && O_idx == nullptr)) return QUAFF_ERR_INVALID_ARG;
+    if (nO > kStaticMaxNO) return QUAFF_ERR_UNSUPPORTED_SHAPE;
+    return QUAFF_OK;
 }
+#define QUAFF_CHECK_OUTLIERS(O_idx, nO, K)                              \
+    do {                                                                \
+        const quaff_status_t rc_ = check_outlier_args(O_idx, nO, K);    \
+        if (rc_ != QUAFF_OK) return rc_;                                \
+    } while (0)
+
+static int momentum_grid(int M) { return max(1, min(ceil_div(M, 16), sm_count() * 2)); }
 
 }  // namespace quaff
 
@@ -422,7 +439,8 @@ extern "C" quaff_status_t quaff_quant_act(const quaff_bf16* X, int64_t ldx, int 
                                           const float* s_O, int8_t* Xq, int64_t ldxq, int8_t* xq_O, int64_t ldxo,
                                           int nOp, float* dx, quaff_stream_t stream) {
     QUAFF_RETURN_IF(!X || !Xq || !dx || M < 0 || K <= 0, QUAFF_ERR_INVALID_ARG);
-    QUAFF_RETURN_IF(!valid_outlier_args(O_idx, nO, K) || (nO > 0 && !s_O), QUAFF_ERR_INVALID_ARG);
+    QUAFF_CHECK_OUTLIERS(O_idx, nO, K);
+    QUAFF_RETURN_IF(nO > 0 && !s_O, QUAFF_ERR_INVALID_ARG);
     QUAFF_RETURN_IF(nOp < nO || (nOp > 0 && !xq_O) || ldx < K || ldxq < K || (nOp > 0 && ldxo < nOp), QUAFF_ERR_INVALID_ARG);
     QUAFF_RETURN_IF(!aligned16(X) || !aligned16(Xq) || (ldx % 8) || (ldxq % 16), QUAFF_ERR_ALIGNMENT);
     if (M == 0) return QUAFF_OK;
@@ -434,16 +452,41 @@ extern "C" quaff_status_t quaff_momentum_update(const quaff_bf16* X, int64_t ldx
                                                 float* colmax_O_opt, float* beta_O_opt, void* ws, size_t ws_bytes,
                                                 quaff_stream_t stream) {
     QUAFF_RETURN_IF(!X || M < 0 || K <= 0 || ldx < K, QUAFF_ERR_INVALID_ARG);
-    QUAFF_RETURN_IF(!valid_outlier_args(O_idx, nO, K), QUAFF_ERR_INVALID_ARG);
+    QUAFF_CHECK_OUTLIERS(O_idx, nO, K);
     QUAFF_RETURN_IF(!(gamma >= 0.0f && gamma <= 1.0f), QUAFF_ERR_INVALID_ARG);
     if (nO == 0) return QUAFF_OK;
     QUAFF_RETURN_IF(!wmax_O || !s_O, QUAFF_ERR_INVALID_ARG);
     QUAFF_RETURN_IF(!ws || ws_bytes < quaff_workspace_bytes(QUAFF_WS_MOMENTUM, M, K, 0, nO, 0), QUAFF_ERR_WORKSPACE_TOO_SMALL);
     cudaStream_t st = (cudaStream_t)stream;
     if (cudaMemsetAsync(ws, 0, (size_t)(nO + 1) * 4, st) != cudaSuccess) return QUAFF_ERR_CUDA;
-    const int grid = max(1, min(ceil_div(M, 16), sm_count() * 2));
-    launch_pdl(momentum_kernel, dim3(grid), dim3(256), 0, st, 1, X, ldx, M, O_idx, nO, wmax_O, gamma, s_O, colmax_O_opt, beta_O_opt,
-               reinterpret_cast<unsigned int*>(ws));
+    launch_pdl(momentum_kernel, dim3(momentum_grid(M)), dim3(256), 0, st, 1, X, ldx, M, O_idx, nO, wmax_O, gamma, s_O, colmax_O_opt,
+               beta_O_opt, reinterpret_cast<unsigned int*>(ws), (const float*)nullptr, 1);
+    return launch_status();
+}
+
+extern "C" quaff_status_t quaff_outlier_colmax(const quaff_bf16* X, int64_t ldx, int M, int K, const int32_t* O_idx, int nO,
+                                               float* colmax_O, void* ws, size_t ws_bytes, quaff_stream_t stream) {
+    QUAFF_RETURN_IF(!X || M < 0 || K <= 0 || ldx < K, QUAFF_ERR_INVALID_ARG);
+    QUAFF_CHECK_OUTLIERS(O_idx, nO, K);
+    if (nO == 0) return QUAFF_OK;
+    QUAFF_RETURN_IF(!colmax_O, QUAFF_ERR_INVALID_ARG);
+    QUAFF_RETURN_IF(!ws || ws_bytes < quaff_workspace_bytes(QUAFF_WS_MOMENTUM, M, K, 0, nO, 0), QUAFF_ERR_WORKSPACE_TOO_SMALL);
+    cudaStream_t st = (cudaStream_t)stream;
+    if (cudaMemsetAsync(ws, 0, (size_t)(nO + 1) * 4, st) != cudaSuccess) return QUAFF_ERR_CUDA;
+    launch_pdl(momentum_kernel, dim3(momentum_grid(M)), dim3(256), 0, st, 1, X, ldx, M, O_idx, nO, (const float*)nullptr, 0.0f,
+               (float*)nullptr, colmax_O, (float*)nullptr, reinterpret_cast<unsigned int*>(ws), (const float*)nullptr, 0);
+    return launch_status();
+}
+
+extern "C" quaff_status_t quaff_momentum_apply(const float* colmax_O, const float* wmax_O, int nO, float gamma, float* s_O,
+                                               float* beta_O_opt, quaff_stream_t stream) {
+    QUAFF_RETURN_IF(nO < 0, QUAFF_ERR_INVALID_ARG);
+    QUAFF_RETURN_IF(!(gamma >= 0.0f && gamma <= 1.0f), QUAFF_ERR_INVALID_ARG);
+    QUAFF_RETURN_IF(nO > kStaticMaxNO, QUAFF_ERR_UNSUPPORTED_SHAPE);
+    if (nO == 0) return QUAFF_OK;
+    QUAFF_RETURN_IF(!colmax_O || !wmax_O || !s_O, QUAFF_ERR_INVALID_ARG);
+    launch_pdl(momentum_kernel, dim3(1), dim3(256), 0, (cudaStream_t)stream, 1, (const uint16_t*)nullptr, (int64_t)0, 0,
+               (const int32_t*)nullptr, nO, wmax_O, gamma, s_O, (float*)nullptr, beta_O_opt, (unsigned int*)nullptr, colmax_O, 1);
     return launch_status();
 }
 
@@ -464,7 +507,7 @@ extern "C" quaff_status_t quaff_prepare_weight(const quaff_bf16* Wt, int64_t ldw
                                                int nO, int8_t* Wq, int64_t ldwq, float* dW, quaff_bf16* W_O,
                                                int64_t ldwo, float* wmax_O, quaff_stream_t stream) {
     QUAFF_RETURN_IF(!Wt || !Wq || !dW || N <= 0 || K <= 0 || ldw < K || ldwq < K, QUAFF_ERR_INVALID_ARG);
-    QUAFF_RETURN_IF(!valid_outlier_args(O_idx, nO, K), QUAFF_ERR_INVALID_ARG);
+    QUAFF_CHECK_OUTLIERS(O_idx, nO, K);
     QUAFF_RETURN_IF(nO > 0 && (!W_O || !wmax_O || ldwo < N), QUAFF_ERR_INVALID_ARG);
     QUAFF_RETURN_IF(!aligned16(Wt) || !aligned16(Wq) || (ldw % 8) || (ldwq % 16), QUAFF_ERR_ALIGNMENT);
     cudaStream_t st = (cudaStream_t)stream;
@@ -483,27 +526,27 @@ extern "C" quaff_status_t quaff_momentum_update_static(const quaff_bf16* X, int6
                                                        float* s_O, float* colmax_O_opt, float* beta_O_opt,
                                                        quaff_stream_t stream) {
     QUAFF_RETURN_IF(!X || M < 0 || K <= 0 || ldx < K, QUAFF_ERR_INVALID_ARG);
-    QUAFF_RETURN_IF(nO < 0 || nO > K || (nO > 0 && !O_idx), QUAFF_ERR_INVALID_ARG);
+    QUAFF_CHECK_OUTLIERS(O_idx, nO, K);    // nO > 4096: more outlier channels than the built-in scratch (or any entry point) takes
     QUAFF_RETURN_IF(!(gamma >= 0.0f && gamma <= 1.0f), QUAFF_ERR_INVALID_ARG);
-    QUAFF_RETURN_IF(nO > kStaticMaxNO, QUAFF_ERR_UNSUPPORTED_SHAPE);  // more outlier channels than the built-in scratch holds
     if (nO == 0) return QUAFF_OK;
     QUAFF_RETURN_IF(!wmax_O || !s_O, QUAFF_ERR_INVALID_ARG);
 
     // In host code `g_momentum_scratch` is only a stand-in for the device array; the address a kernel
     // may use comes from cudaGetSymbolAddress, once per device, with that device current.
-    static unsigned int* scratch_of_device[64] = {nullptr};
+    static std::atomic<unsigned int*> scratch_of_device[64];
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return QUAFF_ERR_CUDA;
-    if (!scratch_of_device[dev]) {
+    unsigned int* scratch = scratch_of_device[dev].load();
+    if (!scratch) {
         void* ptr = nullptr;
         if (cudaGetSymbolAddress(&ptr, g_momentum_scratch) != cudaSuccess || !ptr) return QUAFF_ERR_CUDA;
-        scratch_of_device[dev] = static_cast<unsigned int*>(ptr);
+        scratch = static_cast<unsigned int*>(ptr);
+        scratch_of_device[dev].store(scratch);      // the same address whichever thread gets here first
     }
-    unsigned int* scratch = scratch_of_device[dev];
     cudaStream_t st = (cudaStream_t)stream;
     // the array keeps the previous call's maxima and ticket count: both must start at zero
     if (cudaMemsetAsync(scratch, 0, (size_t)(nO + 1) * sizeof(unsigned int), st) != cudaSuccess) return QUAFF_ERR_CUDA;
-    const int grid = max(1, min(ceil_div(M, 16), sm_count() * 2));
-    launch_pdl(momentum_kernel, dim3(grid), dim3(256), 0, st, 1, X, ldx, M, O_idx, nO, wmax_O, gamma, s_O, colmax_O_opt, beta_O_opt, scratch);
+    launch_pdl(momentum_kernel, dim3(momentum_grid(M)), dim3(256), 0, st, 1, X, ldx, M, O_idx, nO, wmax_O, gamma, s_O, colmax_O_opt,
+               beta_O_opt, scratch, (const float*)nullptr, 1);
     return launch_status();
 }

@@ -95,7 +95,7 @@ struct GemmParams {
     int M, N;            // output extent (rows, columns)
     int tiles_m, tiles_n;
     int band_m;          // row tiles per band of the tile order (tiles_m: one band)
-    int tile_n;          // EPI_BWD: output columns per tile, any multiple of 16 up to TN (0: TN); other epilogues: TN
+    int tile_n;          // EPI_BWD: output columns per tile, a multiple of 64 up to TN (0: TN); other epilogues: TN
     int32_t* status;
     // forward epilogue (Eq. 9 + LoRA)
     const float* dx;     // [M]
@@ -128,7 +128,7 @@ struct GemmSmem {
     uint64_t tmem_full;
     uint64_t tmem_empty;
     uint32_t tmem_base;
-    int abort_flag;
+    AbortCtl abort;
 };
 
 template <int EPI, int CTAS, int TN>
@@ -196,7 +196,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) umma_gemm_kernel(const __grid
     unsigned char* aligned = smem_dyn + (tiles_base - raw);
     GemmSmem* sm = reinterpret_cast<GemmSmem*>(aligned + (size_t)kStages * kStageBytes);
     float* scales = reinterpret_cast<float*>(sm + 1);                 // EPI_FWD only: [2][2][TN]
-    volatile int* abort_flag = &sm->abort_flag;
+    volatile AbortCtl* abort_flag = &sm->abort;
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
@@ -219,7 +219,8 @@ __global__ void __launch_bounds__(kGemmThreads, 1) umma_gemm_kernel(const __grid
         }
         mbar_init(tmem_full_bar, 1);
         mbar_init(tmem_empty_bar, 4 * CTAS);
-        sm->abort_flag = 0;
+        sm->abort.flag = 0;
+        sm->abort.peer = CTAS == 2 ? mapa_shared(smem_u32(&sm->abort.flag), rank ^ 1u) : 0u;
         fence_barrier_init();
     }
     if (warp == 1) {
@@ -379,26 +380,14 @@ __global__ void __launch_bounds__(kGemmThreads, 1) umma_gemm_kernel(const __grid
                     }
                 }
             } else if (EPI == EPI_BWD) {
-                if ((tn_cols & 31) == 0) {
 #pragma unroll 1
-                    for (int c = 0; c < tn_cols; c += 32) {
-                        const int nc = n0 + c;
-                        if (nc >= p.N) break;            // uniform across the warp
-                        uint32_t r0[32];
-                        tmem_ld_32x32(lane_addr + (uint32_t)(buf * kAccStride + c), r0);
-                        tmem_ld_wait();
-                        if (m < p.M) bwd_store_chunk<32>(p, m, nc, r0);
-                    }
-                } else {                                 // a tile width that is a multiple of 16 only
-#pragma unroll 1
-                    for (int c = 0; c < tn_cols; c += 16) {
-                        const int nc = n0 + c;
-                        if (nc >= p.N) break;
-                        uint32_t r0[16];
-                        tmem_ld_32x16(lane_addr + (uint32_t)(buf * kAccStride + c), r0);
-                        tmem_ld_wait();
-                        if (m < p.M) bwd_store_chunk<16>(p, m, nc, r0);
-                    }
+                for (int c = 0; c < tn_cols; c += 32) {
+                    const int nc = n0 + c;
+                    if (nc >= p.N) break;            // uniform across the warp
+                    uint32_t r0[32];
+                    tmem_ld_32x32(lane_addr + (uint32_t)(buf * kAccStride + c), r0);
+                    tmem_ld_wait();
+                    if (m < p.M) bwd_store_chunk<32>(p, m, nc, r0);
                 }
             } else {
 #pragma unroll 1
@@ -467,7 +456,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) umma_gemm_kernel(const __grid
     // ---------------------------------------------------------------------- common exit
     tc_fence_before();
     __syncthreads();
-    if (*abort_flag) {
+    if (abort_flag->flag) {
         for (int i = 0; i < 1000; ++i) __nanosleep(1000);   // let copies in flight land before the CTA retires
         if (threadIdx.x == 0 && p.status) atomicExch(p.status, (int)QUAFF_ERR_TIMEOUT);
         __syncthreads();

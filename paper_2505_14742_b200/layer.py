@@ -24,7 +24,7 @@ class QuaffLinear:
 
     def __init__(self, Wt: torch.Tensor, O_idx: Optional[torch.Tensor], A: Optional[torch.Tensor],
                  B: Optional[torch.Tensor], lora_scale: float, gamma: float, max_tokens: int,
-                 y_dtype: torch.dtype = torch.bfloat16, debug_acc: bool = False):
+                 y_dtype: torch.dtype = torch.bfloat16, debug_acc: bool = False, keep_G: bool = False):
         dev = Wt.device
         self.N, self.K = Wt.shape
         self.nO = 0 if O_idx is None else int(O_idx.numel())
@@ -56,6 +56,8 @@ class QuaffLinear:
         self.dB = torch.zeros((r, N), dtype=f32, device=dev) if r else None
         self.acc_main = torch.empty((M, N), dtype=torch.int32, device=dev) if debug_acc else None
         self.acc_out = torch.empty((M, N), dtype=torch.int32, device=dev) if debug_acc else None
+        # G = bf16(lora_scale dY B^T) of the last backward, kept on request (otherwise it lives in the workspace)
+        self.G = torch.empty((M, r), dtype=bf, device=dev) if (keep_G and r) else None
         self.status = torch.zeros(4, dtype=torch.int32, device=dev)
         ws_bytes = max(Q.workspace_bytes(Q.QUAFF_WS_MOMENTUM, M, K, N, nOp, r),
                        Q.workspace_bytes(Q.QUAFF_WS_FWD, M, K, N, nOp, r),
@@ -101,7 +103,8 @@ class QuaffLinear:
         dX = self.dX[:M] if need_dX else None
         T = self.T[:M] if self.r else None
         Q.quaff_qlinear_bwd(dY, self.Wq, self.dW, self.wq_O, self.dw_O, self.O_idx, self.s_O, self._X, T, self.A, self.B,
-                            self.lora_scale, dX, self.dA, self.dB, accumulate, self.ws, self.status)
+                            self.lora_scale, dX, self.dA, self.dB, accumulate, self.ws, self.status,
+                            self.G[:M] if self.G is not None else None)
         return dX, self.dA, self.dB
 
 

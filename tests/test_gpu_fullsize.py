@@ -11,7 +11,7 @@ import pytest
 
 import oracle
 from paper_2505_14742_b200 import synth
-from util import TOL_BF16, dev, dev_bf16, f32, flip_slack, host, host_bits, max_rel_err
+from util import TOL_BF16, check_bf16_intermediate, dev, dev_bf16, dx_floor, host, host_bits, max_rel_err
 
 pytestmark = pytest.mark.gpu
 
@@ -26,7 +26,8 @@ def _run_layer(wl, li, steps, nsample, check_acc, full_grads=True):
     M, K, N, r = wl.M, sp.K, sp.N, sp.r
     scale = wl.lora_alpha / r
     nOp = synth.pad_to(sp.nO, 32)
-    layer = QuaffLinear(dev_bf16(lin.W), dev(lin.O_idx), dev_bf16(lin.A), dev_bf16(lin.B), scale, wl.gamma, M)
+    # keep_G: the backward writes G into a buffer of the layer instead of its workspace (same kernels, same launches)
+    layer = QuaffLinear(dev_bf16(lin.W), dev(lin.O_idx), dev_bf16(lin.A), dev_bf16(lin.B), scale, wl.gamma, M, keep_G=True)
     Xd = torch.empty((M, K), dtype=torch.bfloat16, device="cuda")
     dYd = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
 
@@ -39,6 +40,7 @@ def _run_layer(wl, li, steps, nsample, check_acc, full_grads=True):
     s = np.ones(sp.nO, np.float32)
     graph = None
     rng = np.random.default_rng(wl.seed + li)
+    none_O, none_s, none_wq = np.zeros(0, np.int32), np.zeros(0, np.float32), np.zeros((1, 0), np.int8)
     for step in range(steps):
         X, dY = synth.step_inputs(wl, li, step, lin)
         Xd.copy_(dev_bf16(X)); dYd.copy_(dev_bf16(dY))
@@ -60,35 +62,34 @@ def _run_layer(wl, li, steps, nsample, check_acc, full_grads=True):
         rows = np.sort(rng.choice(M, nsample, replace=False))
         rows[0], rows[-1] = 0, M - 1                       # first and last row of the first and last tile
         Xs, dYs = np.ascontiguousarray(X[rows]), np.ascontiguousarray(dY[rows])
+        Tg, Gg = host_bits(layer.T), host_bits(layer.G)
+        # the bf16 intermediates of the sampled rows: at most one ulp from the oracle's; everything downstream is
+        # compared with the oracle evaluated on the GPU's own T and G bits, with no allowance
         oY, oT, o1, o2 = oracle.qlinear_fwd(Xq[rows], xqo[rows], dx[rows], Wq, dW, wq, dw, Xs, lin.A, lin.B, scale)
-        Tg = host_bits(layer.T)
-        assert max_rel_err(f32(Tg[rows]), f32(oT)) <= TOL_BF16, "T"
-        err = max_rel_err(host(layer.Y)[rows], oY, flip_slack(f32(oT).T, f32(lin.B), scale))
+        check_bf16_intermediate(Tg[rows], oT, f"T rows, step {step}")
+        oY = oracle.qlinear_fwd(Xq[rows], xqo[rows], dx[rows], Wq, dW, wq, dw, Xs, lin.A, lin.B, scale, T_in=Tg[rows])[0]
+        err = max_rel_err(host(layer.Y)[rows], oY)
         assert err <= TOL_BF16, f"Y rows, step {step}: {err:.3e}"
-        odX, _, _, oGs = oracle.qlinear_bwd(dYs, Wq, dW, wq, dw, lin.O_idx, s, Xs, oT, lin.A, lin.B, scale, want_dAB=False)
-        err = max_rel_err(host(layer.dX)[rows], odX, flip_slack(f32(oGs).T, f32(lin.A).T))
+        oGs = oracle.qlinear_bwd(dYs, Wq, dW, wq, dw, lin.O_idx, s, Xs, Tg[rows], lin.A, lin.B, scale, want_dX=False, want_dAB=False)[3]
+        check_bf16_intermediate(Gg[rows], oGs, f"G rows, step {step}")
+        odX = oracle.qlinear_bwd(dYs, Wq, dW, wq, dw, lin.O_idx, s, Xs, Tg[rows], lin.A, lin.B, scale, want_dAB=False, G_in=Gg[rows])[0]
+        err = max_rel_err(host(layer.dX)[rows], odX, dx_floor(N))
         assert err <= TOL_BF16, f"dX rows, step {step}: {err:.3e}"
-        # LoRA gradients contract over all tokens: T and G of the whole batch from the oracle
-        oT_full = oracle.lora_down(X, lin.A)
+        # LoRA gradients contract over all tokens
         if full_grads:
-            _, odA, odB, oG_full = oracle.qlinear_bwd(dY, Wq, dW, wq, dw, lin.O_idx, s, X, oT_full, lin.A, lin.B, scale,
-                                                      want_dX=False)
-            assert max_rel_err(host(layer.dA), odA, flip_slack(f32(oG_full), f32(X)).T) <= TOL_BF16, "dA"
-            assert max_rel_err(host(layer.dB), odB, flip_slack(f32(oT_full), f32(dY), scale)) <= TOL_BF16, "dB"
+            check_bf16_intermediate(Tg, oracle.lora_down(X, lin.A), f"T, step {step}")
+            _, odA, odB, _ = oracle.qlinear_bwd(dY, Wq, dW, wq, dw, lin.O_idx, s, X, Tg, lin.A, lin.B, scale, want_dX=False, G_in=Gg)
+            ea, eb = max_rel_err(host(layer.dA), odA), max_rel_err(host(layer.dB), odB)
         else:
-            # too large for the oracle's loops: dA = X^T G and dB = scale T^T dY on sampled rows / columns, the
-            # contraction over all tokens by a float64 matrix product of the oracle's rounded G and T
-            Gf = np.empty((M, r), np.float64)
-            for m0 in range(0, M, 1024):      # G = bf16(scale dY B^T) from the oracle, a slab of tokens at a time
-                sl = slice(m0, min(M, m0 + 1024))
-                Gf[sl] = f32(oracle.qlinear_bwd(dY[sl], Wq, dW, wq, dw, lin.O_idx, s, X[sl], oT_full[sl], lin.A, lin.B, scale,
-                                                want_dX=False, want_dAB=False)[3])
-            ks = np.sort(rng.choice(K, 96, replace=False)); ks[:len(lin.O_idx[:8])] = lin.O_idx[:8]
-            ns = np.sort(rng.choice(N, 96, replace=False))
-            odA = f32(X[:, ks]).astype(np.float64).T @ Gf
-            odB = scale * (f32(oT_full).astype(np.float64).T @ f32(dY[:, ns]).astype(np.float64))
-            assert max_rel_err(host(layer.dA)[ks], odA, flip_slack(Gf, f32(X[:, ks])).T) <= TOL_BF16, "dA rows"
-            assert max_rel_err(host(layer.dB)[:, ns], odB, flip_slack(f32(oT_full), f32(dY[:, ns]), scale)) <= TOL_BF16, "dB columns"
+            # too large for the oracle's loops in full: dA[k][:] depends on column k of X only and dB[:][n] on column n of
+            # dY only, so the oracle computes sampled rows of dA and sampled columns of dB over ALL tokens
+            ks = np.sort(rng.choice(K, 64, replace=False)); ks[:len(lin.O_idx[:8])] = lin.O_idx[:8]; ks = np.unique(ks)
+            ns = np.sort(rng.choice(N, 64, replace=False))
+            _, odA, odB, _ = oracle.qlinear_bwd(np.ascontiguousarray(dY[:, ns]), np.zeros((len(ns), len(ks)), np.int8), dW[ns], none_wq,
+                                                dw[ns], none_O, none_s, np.ascontiguousarray(X[:, ks]), Tg, np.ascontiguousarray(lin.A[ks]),
+                                                np.ascontiguousarray(lin.B[:, ns]), scale, want_dX=False, G_in=Gg)
+            ea, eb = max_rel_err(host(layer.dA)[ks], odA), max_rel_err(host(layer.dB)[:, ns], odB)
+        assert ea <= TOL_BF16 and eb <= TOL_BF16, f"dA {ea:.3e} dB {eb:.3e}, step {step}"
         if check_acc and step == 0:
             # INT32 accumulators of the same rows through the C ABI's debug dumps (a separate call: the dumps are
             # not on the timed path)
@@ -112,8 +113,16 @@ def test_phi3_attn_o_proj_full_size():
     _run_layer(synth.WORKLOADS["phi3_attn"], 1, steps=1, nsample=48, check_acc=True)
 
 
-def test_llama7b_down_proj_full_size():
-    _run_layer(synth.WORKLOADS["llama7b_block"], 6, steps=1, nsample=24, check_acc=True, full_grads=False)
+# LLaMA-2-7B block, 8192 tokens: one layer of each shape (q/k/v/o are 4096 -> 4096, gate/up 4096 -> 11008)
+@pytest.mark.parametrize("li", [0, 4, 6], ids=["q_proj", "gate_proj", "down_proj"])
+def test_llama7b_block_layers_full_size(li):
+    _run_layer(synth.WORKLOADS["llama7b_block"], li, steps=1, nsample=24, check_acc=True, full_grads=False)
+
+
+# Phi-3 MLP, 4096 tokens: fused gate_up 3072 -> 16384 and down 8192 -> 3072, one forward + backward step each
+@pytest.mark.parametrize("li", [0, 1], ids=["gate_up_proj", "down_proj"])
+def test_phi3_mlp_layers_full_size(li):
+    _run_layer(synth.WORKLOADS["phi3_mlp"], li, steps=1, nsample=24, check_acc=True, full_grads=False)
 
 
 def test_phi3_mlp_late_outliers_momentum_adaptation():
@@ -161,9 +170,24 @@ def test_phi3_mlp_late_outliers_momentum_adaptation():
             assert np.all(s[-sp.late:] > 25.0), "the late outlier channels (20-100x) have been picked up by the momentum update"
 
 
-@pytest.mark.parametrize("M,K,N,r,frac", [(512, 2048, 4096, 8, 0.05), (2048, 8192, 2048, 32, 0.01), (32768, 2048, 2048, 64, 0.005)])
+# Twelve points of the shape sweep (tokens x K x N x rank x outlier fraction): together they take every value of every
+# axis - M in {512, 2048, 8192, 32768}, K and N in {2048, 4096, 8192}, rank in {8, 32, 64}, 0.5 / 1 / 5 % outlier
+# channels.  5 % of 8192 is nO = 410 (nOp = 416 > 128: the forward with all three accumulators resident), 5 % of
+# 2048 is nO = 102 (nOp = 128).
+SWEEP_POINTS = [(512, 2048, 4096, 8, 0.05), (2048, 8192, 2048, 32, 0.01), (32768, 2048, 2048, 64, 0.005),
+                (8192, 8192, 4096, 8, 0.05), (512, 4096, 8192, 64, 0.01), (2048, 4096, 4096, 32, 0.005),
+                (8192, 2048, 8192, 32, 0.05), (32768, 4096, 2048, 8, 0.01), (512, 8192, 8192, 32, 0.005),
+                (2048, 2048, 2048, 64, 0.05), (8192, 4096, 2048, 64, 0.005), (32768, 8192, 4096, 32, 0.01)]
+
+
+def test_sweep_points_cover_every_axis_value():
+    for axis, want in ((0, {512, 2048, 8192, 32768}), (1, {2048, 4096, 8192}), (2, {2048, 4096, 8192}), (3, {8, 32, 64}),
+                       (4, {0.005, 0.01, 0.05})):
+        assert {p[axis] for p in SWEEP_POINTS} == want
+
+
+@pytest.mark.parametrize("M,K,N,r,frac", SWEEP_POINTS)
 def test_shape_sweep_points(M, K, N, r, frac):
-    """Points of the shape sweep (tokens x K x N x rank x outlier fraction), one step each; 5 % of 2048 channels is
-    nO = 102 (the 128-column forward with nOp = 128)."""
+    """One forward + backward step of a sweep point through the graph-replayed layer, against the oracle."""
     wl = synth.sweep_point(M, K, N, r, frac)
     _run_layer(wl, 0, steps=1, nsample=16, check_acc=True, full_grads=False)

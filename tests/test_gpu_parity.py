@@ -6,7 +6,7 @@ import pytest
 
 import oracle
 from paper_2505_14742_b200 import synth
-from util import TOL_BF16, TOL_F32, bf, dev, dev_bf16, f32, flip_slack, host, host_bits, max_rel_err
+from util import TOL_BF16, TOL_F32, bf, check_bf16_intermediate, dev, dev_bf16, dx_floor, f32, host, host_bits, max_rel_err
 
 pytestmark = pytest.mark.gpu
 
@@ -196,11 +196,13 @@ def _check_fwd(Q, M, K, N, nO, r, y_f32, y_pad=0):
     assert np.array_equal(host(a1), o1), "main INT32 accumulator"
     assert np.array_equal(host(a2), o2), "outlier INT32 accumulator"
     if r:
-        assert max_rel_err(f32(host_bits(T)), f32(oT)) <= TOL_BF16, "LoRA down-projection T"
+        # T: at most one bf16 ulp from the oracle's, entry by entry; Y is then checked against the oracle's
+        # up-projection of the GPU's own T bits, so that no allowance for a differing rounding of T is needed
+        Tg = host_bits(T)
+        check_bf16_intermediate(Tg, oT, "LoRA down-projection T")
+        oY = oracle.qlinear_fwd(Xq, xqo, dx, Wq, dW, wq, dw, X, A, B, 0.5, T_in=Tg)[0]
     tol = TOL_F32 if (y_f32 and r == 0) else TOL_BF16
-    # Y[m][n] += scale * sum_j T[m][j] B[j][n]: allowance for a differing rounding decision on T
-    slack = flip_slack(f32(oT).T, f32(B), 0.5) if r else None
-    err = max_rel_err(host(Y), oY, slack)
+    err = max_rel_err(host(Y), oY)
     assert err <= tol, f"max rel err {err:.3e}"
     assert bool((Ybuf[M:, :] == SENT).all()) and bool((Ybuf[:, N:] == SENT).all()), "write outside Y"
 
@@ -244,23 +246,25 @@ def test_qlinear_bwd(Q, M, K, N, nO, r):
     args = (dev_bf16(dY), Wq_d[:, :K], dev(dW), dev(wq) if nOp else None, dev(dw), dev(O) if nO else None,
             dev(s) if nO else None, dev_bf16(X), dev_bf16(oT) if r else None, dev_bf16(A) if r else None,
             dev_bf16(B) if r else None, 0.5, dX, dA, dB)
-    Q.quaff_qlinear_bwd(*args, False, ws, st)
+    Gd = torch.full((M, r), float("nan"), dtype=torch.bfloat16, device="cuda") if r else None
+    Q.quaff_qlinear_bwd(*args, False, ws, st, Gd)
     torch.cuda.synchronize()
     assert host(st)[0] == 0
-    # allowances for a differing bf16 rounding decision on G (dX += G A^T, dA = X^T G) or T (dB = scale T^T dY)
-    Gf = f32(oG) if r else None
-    sl_dX = flip_slack(Gf.T, f32(A).T) if r else None                # [M][K]
-    sl_dA = flip_slack(Gf, f32(X)).T if r else None                  # [K][r]
-    sl_dB = flip_slack(f32(oT), f32(dY), 0.5) if r else None         # [r][N]
-    err = max_rel_err(host(dX), odX, sl_dX)
+    if r:
+        # G: at most one bf16 ulp from the oracle's, entry by entry; everything downstream of G is then compared with
+        # the oracle evaluated on the GPU's own G bits (T is the oracle's on both sides already): no allowance
+        Gg = host_bits(Gd)
+        check_bf16_intermediate(Gg, oG, "G = bf16(scale dY B^T)")
+        odX, odA, odB, _ = oracle.qlinear_bwd(dY, Wq, dW, wq, dw, O, s, X, oT, A, B, 0.5, G_in=Gg)
+    err = max_rel_err(host(dX), odX, dx_floor(N))
     assert err <= TOL_BF16, f"dX max rel err {err:.3e}"
     assert bool((dXbuf[M:, :] == -777.0).all()) and bool((dXbuf[:, K:] == -777.0).all()), "write outside dX"
     if nO:
-        err_o = max_rel_err(host(dX)[:, O], odX[:, O], sl_dX[:, O] if r else None)
+        err_o = max_rel_err(host(dX)[:, O], odX[:, O], dx_floor(N))
         assert err_o <= TOL_BF16, f"dX outlier columns max rel err {err_o:.3e}"
     if r:
-        assert max_rel_err(host(dA), odA, sl_dA) <= TOL_BF16
-        assert max_rel_err(host(dB), odB, sl_dB) <= TOL_BF16
+        err_a, err_b = max_rel_err(host(dA), odA), max_rel_err(host(dB), odB)
+        assert err_a <= TOL_BF16 and err_b <= TOL_BF16, f"dA {err_a:.3e} dB {err_b:.3e}"
     # the two halves of the call on their own (other stream layout inside the library): the same kernels, the same bits
     dX2 = torch.full((M, K), float("nan"), dtype=torch.bfloat16, device="cuda")
     Q.quaff_qlinear_bwd(*args[:12], dX2, None, None, False, ws, st)            # dX only
@@ -274,8 +278,8 @@ def test_qlinear_bwd(Q, M, K, N, nO, r):
         # gradient accumulation: a second call with accumulate adds the same gradients again
         Q.quaff_qlinear_bwd(*args, True, ws, st)
         torch.cuda.synchronize()
-        assert max_rel_err(host(dA), 2 * odA, 2 * sl_dA) <= TOL_BF16
-        assert max_rel_err(host(dB), 2 * odB, 2 * sl_dB) <= TOL_BF16
+        assert max_rel_err(host(dA), 2 * odA) <= TOL_BF16
+        assert max_rel_err(host(dB), 2 * odB) <= TOL_BF16
 
 
 # ----------------------------------------------------------------------------- whole path, several steps
@@ -290,7 +294,7 @@ def test_tiny_workload_all_steps(Q):
     sp = lin.spec
     scale = wl.lora_alpha / sp.r
     layer = QuaffLinear(dev_bf16(lin.W), dev(lin.O_idx), dev_bf16(lin.A), dev_bf16(lin.B), scale, wl.gamma, wl.M,
-                        y_dtype=torch.bfloat16, debug_acc=True)
+                        y_dtype=torch.bfloat16, debug_acc=True, keep_G=True)
     Wq, dW, W_O, wmax = oracle.prepare_weight(lin.W, lin.O_idx)
     s = np.ones(sp.nO, np.float32)
     nOp = _pad32(sp.nO)
@@ -304,7 +308,12 @@ def test_tiny_workload_all_steps(Q):
         Xq, xqo, dx = oracle.quant_act(X, lin.O_idx, s, nOp)
         wq, dw = oracle.requant_weight_rows(W_O, s, nOp)
         oY, oT, o1, o2 = oracle.qlinear_fwd(Xq, xqo, dx, Wq, dW, wq, dw, X, lin.A, lin.B, scale)
-        odX, odA, odB, _ = oracle.qlinear_bwd(dY, Wq, dW, wq, dw, lin.O_idx, s, X, oT, lin.A, lin.B, scale)
+        _, _, _, oG = oracle.qlinear_bwd(dY, Wq, dW, wq, dw, lin.O_idx, s, X, oT, lin.A, lin.B, scale, want_dX=False, want_dAB=False)
+        Tg, Gg = host_bits(layer.T), host_bits(layer.G)
+        check_bf16_intermediate(Tg, oT, f"T at step {step}")
+        check_bf16_intermediate(Gg, oG, f"G at step {step}")
+        oY = oracle.qlinear_fwd(Xq, xqo, dx, Wq, dW, wq, dw, X, lin.A, lin.B, scale, T_in=Tg)[0]
+        odX, odA, odB, _ = oracle.qlinear_bwd(dY, Wq, dW, wq, dw, lin.O_idx, s, X, Tg, lin.A, lin.B, scale, G_in=Gg)
         assert np.array_equal(host(layer.s_O), s), f"s_O at step {step}"
         assert np.array_equal(host(layer.Xq), Xq) and np.array_equal(host(layer.xq_O), xqo)
         assert np.array_equal(host(layer.dx), dx)
@@ -336,3 +345,98 @@ def test_argument_validation(Q):
         Q.quaff_momentum_update(X, O[:4], dx, 0.5, dx, torch.zeros(8, dtype=torch.uint8, device="cuda"))
     assert e.value.code == Q.QUAFF_ERR_WORKSPACE_TOO_SMALL
     torch.cuda.synchronize()
+
+
+# ----------------------------------------------------------------------------- split scale update (token shards)
+def test_split_momentum_update_matches_the_whole_batch(Q):
+    """Column maxima per shard (quaff_outlier_colmax), elementwise maximum (what a MAX all-reduce does), then
+    quaff_momentum_apply: the same s_O, bit for bit, as quaff_momentum_update on the whole batch and as the oracle."""
+    import torch
+    M, K, nO, gamma = 1000, 768, 37, 0.2
+    O, X, Wt, _, _, _ = _mk_inputs(901, M, K, 16, nO, 0)
+    _, _, _, wmax = oracle.prepare_weight(Wt, O)
+    Xd, Od, wd = dev_bf16(X), dev(O), dev(wmax)
+    ws = torch.empty(Q.workspace_bytes(Q.QUAFF_WS_MOMENTUM, M, K, 16, _pad32(nO), 0), dtype=torch.uint8, device="cuda")
+    s_whole, s_split = dev(np.full(nO, 1.5, np.float32)), dev(np.full(nO, 1.5, np.float32))
+    cm_whole = torch.empty(nO, dtype=torch.float32, device="cuda")
+    Q.quaff_momentum_update(Xd, Od, wd, gamma, s_whole, ws, cm_whole)
+    shards = [(0, 300), (300, 301), (301, M)]
+    cms = []
+    for a, b in shards:
+        cm = torch.full((nO,), -1.0, dtype=torch.float32, device="cuda")
+        Q.quaff_outlier_colmax(Xd[a:b], Od, cm, ws)
+        torch.cuda.synchronize()
+        assert np.array_equal(host(cm), oracle.outlier_colmax(X[a:b], O))
+        cms.append(cm)
+    combined = torch.maximum(torch.maximum(cms[0], cms[1]), cms[2])
+    be = torch.empty(nO, dtype=torch.float32, device="cuda")
+    Q.quaff_momentum_apply(combined, wd, gamma, s_split, be)
+    torch.cuda.synchronize()
+    assert np.array_equal(host(combined), host(cm_whole))
+    assert np.array_equal(host(s_split), host(s_whole))
+    s_or, _, be_or = oracle.momentum_update(X, O, wmax, gamma, np.full(nO, 1.5, np.float32))
+    assert np.array_equal(host(s_split), s_or) and np.array_equal(host(be), be_or)
+
+
+# ----------------------------------------------------------------------------- two host threads, two streams
+def test_backward_from_two_host_threads_is_bit_identical_to_serial(Q):
+    """Two host threads, each with its own stream, buffers and workspace, call forward + backward at the same time
+    (the library's lazily created per-device resources and the side streams of the backward are shared): every
+    output equals the serial run's, bit for bit."""
+    import threading
+    import torch
+    M, K, N, nO, r = 640, 1024, 1536, 12, 16
+    cases = []
+    for seed in (31, 32):
+        O, X, Wt, A, B, dY = _mk_inputs(seed, M, K, N, nO, r)
+        Wq, dW, W_O, wmax, s, Xq, xqo, dx, wq, dw = _oracle_state(O, X, Wt)
+        nOp = _pad32(nO)
+        d = dict(Xq=dev(Xq), xqo=dev(xqo), dx=dev(dx), Wq=dev(Wq), dW=dev(dW), wq=dev(wq), dw=dev(dw), X=dev_bf16(X), A=dev_bf16(A),
+                 B=dev_bf16(B), dY=dev_bf16(dY), O=dev(O), s=dev(s),
+                 ws=torch.empty(max(Q.workspace_bytes(Q.QUAFF_WS_FWD, M, K, N, nOp, r), Q.workspace_bytes(Q.QUAFF_WS_BWD, M, K, N, nOp, r)),
+                                dtype=torch.uint8, device="cuda"),
+                 st=torch.zeros(4, dtype=torch.int32, device="cuda"))
+        cases.append(d)
+
+    def run(d, out):
+        T = torch.empty((M, r), dtype=torch.bfloat16, device="cuda")
+        Y = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
+        dX = torch.empty((M, K), dtype=torch.bfloat16, device="cuda")
+        dA = torch.empty((K, r), dtype=torch.float32, device="cuda")
+        dB = torch.empty((r, N), dtype=torch.float32, device="cuda")
+        for _ in range(out["reps"]):
+            Q.quaff_qlinear_fwd(d["Xq"], d["xqo"], d["dx"], d["Wq"], d["dW"], d["wq"], d["dw"], d["X"], d["A"], d["B"], 0.5, T, Y, d["ws"],
+                                None, None, d["st"])
+            Q.quaff_qlinear_bwd(d["dY"], d["Wq"], d["dW"], d["wq"], d["dw"], d["O"], d["s"], d["X"], T, d["A"], d["B"], 0.5, dX, dA, dB,
+                                False, d["ws"], d["st"])
+        out["res"] = (Y, dX, dA, dB)
+
+    serial = []
+    for d in cases:
+        o = {"reps": 1}
+        run(d, o)
+        torch.cuda.synchronize()
+        serial.append([host(t) for t in o["res"]])
+
+    outs = [{"reps": 20}, {"reps": 20}]
+    errors = []
+
+    def worker(i):
+        try:
+            with torch.cuda.stream(torch.cuda.Stream()):
+                run(cases[i], outs[i])
+                torch.cuda.current_stream().synchronize()
+        except Exception as e:  # noqa: BLE001
+            errors.append(e)
+
+    threads = [threading.Thread(target=worker, args=(i,)) for i in range(2)]
+    for t in threads:
+        t.start()
+    for t in threads:
+        t.join()
+    torch.cuda.synchronize()
+    assert not errors, errors
+    for i in range(2):
+        assert host(cases[i]["st"])[0] == 0
+        for got, ref in zip(outs[i]["res"], serial[i]):
+            assert np.array_equal(host(got), ref)

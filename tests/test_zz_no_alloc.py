@@ -2,10 +2,12 @@
 (a plug-in in a framework that owns the memory budget, a step that must not hit cudaMalloc's
 device-wide synchronisation) - must give exactly what quaff_momentum_update gives with a
 caller-supplied workspace.  Checked on two calls in a row, because the built-in scratch array keeps
-the previous call's contents and the entry point has to clear it itself.  Collected last on purpose."""
+the previous call's contents and the entry point has to clear it itself; both are also compared with the
+CPU oracle's update.  Collected last on purpose."""
 import numpy as np
 import pytest
 
+import oracle
 from util import bf, dev, dev_bf16, host
 
 pytestmark = pytest.mark.gpu
@@ -23,6 +25,7 @@ def test_static_scratch_variant_matches_workspace_variant_twice_in_a_row():
     s_st = dev(np.ones(nO, np.float32))
     out = {k: torch.empty(nO, dtype=torch.float32, device="cuda") for k in ("cm_ws", "be_ws", "cm_st", "be_st")}
     ws = torch.empty(Q.workspace_bytes(Q.QUAFF_WS_MOMENTUM, M, K, 16, 64, 0), dtype=torch.uint8, device="cuda")
+    s_or = np.ones(nO, np.float32)
     for call in range(2):
         x = rng.standard_normal((M, K)).astype(np.float32)
         x[:, O] *= rng.uniform(20, 100, nO).astype(np.float32) / (1 + 3 * call)   # second call: smaller maxima
@@ -34,6 +37,10 @@ def test_static_scratch_variant_matches_workspace_variant_twice_in_a_row():
         assert np.array_equal(host(out["cm_st"]), host(out["cm_ws"])), f"column maxima, call {call}"
         assert np.array_equal(host(out["be_st"]), host(out["be_ws"])), f"beta, call {call}"
         assert np.array_equal(host(s_st), host(s_ws)), f"s_O, call {call}"
+        # and both against the oracle (Eq. 8, Eq. 7), state carried over the two calls
+        s_or, cm_or, be_or = oracle.momentum_update(bf(x), O, wmax, gamma, s_or)
+        assert np.array_equal(host(out["cm_st"]), cm_or) and np.array_equal(host(out["be_st"]), be_or), f"oracle, call {call}"
+        assert np.array_equal(host(s_st), s_or), f"s_O against the oracle, call {call}"
     assert (host(s_st) > 1.0).all()
 
 
