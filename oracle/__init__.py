@@ -37,6 +37,7 @@ def _load():
         _lib.qo_num_threads.restype = ctypes.c_int
         _lib.qo_int_gemm.restype = ctypes.c_int64
         _lib.qo_qlinear_fwd.restype = ctypes.c_int64
+        _lib.qo_qlinear_bwd_int8.restype = ctypes.c_int64
     return _lib
 
 
@@ -233,6 +234,52 @@ def qlinear_bwd(dY, Wq, dW, wq_O, dw_O, O_idx, s_O, X, T, A, B, lora_scale: floa
                            _p(X), I64(K), _p(T_), _p(A_), _p(B_), I32(r), F32(lora_scale),
                            _p(dX), _p(dA), _p(dB), _p(G), _p(G_in_))
     return dX, dA, dB, G[:, :r]
+
+
+def quant_grad(dY: np.ndarray, dW: np.ndarray):
+    """INT8 grad-input variant: Z = dY * dW[n] quantized per token.  Returns (Zq[M,N] int8, dz[M] f32)."""
+    dY = _c(dY, np.uint16)
+    dW = _c(dW, np.float32)
+    M, N = dY.shape
+    Zq = np.empty((M, N), np.int8)
+    dz = np.empty(M, np.float32)
+    _load().qo_quant_grad(_p(dY), I64(N), I32(M), I32(N), _p(dW), _p(Zq), I64(N), _p(dz))
+    return Zq, dz
+
+
+def qlinear_bwd_int8(dY, Wq, dW, wq_O, dw_O, O_idx, s_O, X, T, A, B, lora_scale: float, want_dAB: bool = True, G_in=None):
+    """The INT8 grad-input variant (not the paper's method).  Returns (dX[M,K] f64, dA | None, dB | None, G bf16 bits,
+    Zq[M,N] int8, dz[M] f32, acc[M,K] int32)."""
+    dY = _c(dY, np.uint16)
+    M, N = dY.shape
+    Wq = _c(Wq, np.int8)
+    K = Wq.shape[1]
+    O_idx = _c(O_idx, np.int32)
+    nO = O_idx.shape[0]
+    nOp = wq_O.shape[1]
+    wq_O = _c(wq_O if nOp else np.zeros((N, 1), np.int8), np.int8)
+    dW = _c(dW, np.float32)
+    dw_O = _c(dw_O, np.float32)
+    s_O = _c(s_O, np.float32)
+    r = 0 if A is None else A.shape[1]
+    X = _c(X, np.uint16)
+    T_ = _c(T, np.uint16) if r else None
+    A_ = _c(A, np.uint16) if r else None
+    B_ = _c(B, np.uint16) if r else None
+    dX = np.empty((M, K), np.float64)
+    dA = np.empty((K, r), np.float64) if (want_dAB and r) else None
+    dB = np.empty((r, N), np.float64) if (want_dAB and r) else None
+    G = np.zeros((M, max(r, 1)), np.uint16)
+    G_in_ = _c(G_in, np.uint16) if (G_in is not None and r) else None
+    Zq = np.empty((M, N), np.int8)
+    dz = np.empty(M, np.float32)
+    acc = np.empty((M, K), np.int32)
+    ov = _load().qo_qlinear_bwd_int8(I32(M), I32(K), I32(N), _p(dY), I64(N), _p(Wq), I64(K), _p(dW),
+                                     _p(wq_O), I64(wq_O.shape[1]), _p(dw_O), I32(nOp), _p(O_idx), I32(nO), _p(s_O),
+                                     _p(X), I64(K), _p(T_), _p(A_), _p(B_), I32(r), F32(lora_scale),
+                                     _p(dX), _p(dA), _p(dB), _p(G), _p(G_in_), _p(Zq), _p(dz), _p(acc))
+    assert ov == 0, "integer accumulator overflow"
+    return dX, dA, dB, G[:, :r], Zq, dz, acc
 
 
 def outlier_count(X: np.ndarray, thr: int, xi: np.ndarray) -> np.ndarray:

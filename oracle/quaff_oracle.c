@@ -395,6 +395,97 @@ void qo_qlinear_bwd(int M, int K, int N,
     free(G);
 }
 
+/* ---------------------------------------------------------------- INT8 grad-input variant (NOT the paper's method)
+ * The paper quantizes no gradient (Sec. 4.1 keeps the model in floating point; Sec. 3.3 gives a forward only).  This
+ * variant exists to put the largest GEMM of the step on the INT8 tensor path; it is selected by its own entry point
+ * and reported separately.  Per-output-channel step sizes Delta_W[n] lie on the contraction axis of the backward, so
+ * they are folded into dY before a per-token quantization (Eq. 1 applied to the rows of Z):
+ *   Z[m][n]   = dY[m][n] * Delta_W[n]                       (fp32, one rounding)
+ *   Dz[m]     = max_n |Z[m][n]| / 127 ;  Zq[m][n] = [Z[m][n] / Dz[m]]          (ties to even, as everywhere)
+ *   acc[m][k] = sum_n Zq[m][n] * Wq[n][k]                   (integers)
+ *   dXhat[m][k] = Dz[m] * acc[m][k]                         for k outside O
+ * The nO outlier columns stay on the floating-point path of qo_qlinear_bwd (they are few, and they are the ones
+ * divided by s):  dXhat[m][O_i] = (sum_n dY[m][n] Wd[n][O_i] + sum_n dY[m][n] wd[n][i]) / s_i.
+ * G, dX = dXhat + G A^T, dA and dB are those of qo_qlinear_bwd.
+ */
+void qo_quant_grad(const uint16_t* dY, int64_t lddy, int M, int N, const float* dW, int8_t* Zq, int64_t ldz, float* dz) {
+#pragma omp parallel for schedule(static)
+    for (int m = 0; m < M; ++m) {
+        float* z = (float*)malloc(sizeof(float) * (size_t)(N > 0 ? N : 1));
+        float amax = 0.0f;
+        for (int n = 0; n < N; ++n) {
+            z[n] = bf2f(dY[(int64_t)m * lddy + n]) * dW[n];
+            float a = fabsf(z[n]);
+            if (a > amax) amax = a;
+        }
+        dz[m] = amax / 127.0f;
+        float rinv = amax > 0.0f ? 127.0f / amax : 0.0f;
+        for (int n = 0; n < N; ++n) Zq[(int64_t)m * ldz + n] = quant_code(z[n], rinv);
+        free(z);
+    }
+}
+
+/* dX [M][K] double (required); dA, dB, G_out, G_in as in qo_qlinear_bwd; Zq_out [M][N], dz_out [M], acc_out [M][K] int32
+ * (nullable dumps).  Returns the number of accumulators outside int32 (must be 0). */
+int64_t qo_qlinear_bwd_int8(int M, int K, int N,
+                            const uint16_t* dY, int64_t lddy,
+                            const int8_t* Wq, int64_t ldwq_main, const float* dW,
+                            const int8_t* wq_O, int64_t ldwq, const float* dw_O, int nOp,
+                            const int32_t* O_idx, int nO, const float* s_O,
+                            const uint16_t* X, int64_t ldx, const uint16_t* T, const uint16_t* A, const uint16_t* B,
+                            int r, float lora_scale,
+                            double* dX, double* dA, double* dB, uint16_t* G_out, const uint16_t* G_in,
+                            int8_t* Zq_out, float* dz_out, int32_t* acc_out) {
+    /* G, dA, dB: exactly the floating-point routine with the grad-input switched off */
+    uint16_t* G = (uint16_t*)malloc(sizeof(uint16_t) * (size_t)M * (size_t)(r > 0 ? r : 1));
+    qo_qlinear_bwd(M, K, N, dY, lddy, Wq, ldwq_main, dW, wq_O, ldwq, dw_O, nOp, O_idx, nO, s_O, X, ldx, T, A, B, r, lora_scale,
+                   NULL, dA, dB, G, G_in);
+    if (G_out && r > 0) memcpy(G_out, G, sizeof(uint16_t) * (size_t)M * (size_t)r);
+    int8_t* Zq = (int8_t*)malloc((size_t)M * (size_t)N);
+    float* dz = (float*)malloc(sizeof(float) * (size_t)M);
+    qo_quant_grad(dY, lddy, M, N, dW, Zq, N, dz);
+    if (Zq_out) memcpy(Zq_out, Zq, (size_t)M * (size_t)N);
+    if (dz_out) memcpy(dz_out, dz, sizeof(float) * (size_t)M);
+    int64_t overflow = 0;
+#pragma omp parallel for schedule(static) reduction(+ : overflow)
+    for (int m = 0; m < M; ++m) {
+        double* row = dX + (int64_t)m * K;
+        int64_t* acc = (int64_t*)calloc((size_t)K, sizeof(int64_t));
+        for (int n = 0; n < N; ++n) {
+            int64_t z = (int64_t)Zq[(int64_t)m * N + n];
+            const int8_t* w = Wq + (int64_t)n * ldwq_main;
+            for (int k = 0; k < K; ++k) acc[k] += z * (int64_t)w[k];
+        }
+        for (int k = 0; k < K; ++k) {
+            if (acc[k] > INT32_MAX || acc[k] < INT32_MIN) overflow++;
+            if (acc_out) acc_out[(int64_t)m * K + k] = (int32_t)acc[k];
+            row[k] = (double)dz[m] * (double)acc[k];
+        }
+        free(acc);
+        /* outlier columns: floating-point path, through the bf16-dequantized codes */
+        for (int i = 0; i < nO; ++i) {
+            double o = 0.0;
+            for (int n = 0; n < N; ++n) {
+                double g = (double)bf2f(dY[(int64_t)m * lddy + n]);
+                double wd_main = (double)bf2f(f2bf((float)Wq[(int64_t)n * ldwq_main + O_idx[i]] * dW[n]));
+                double wd_out = (double)bf2f(f2bf((float)wq_O[(int64_t)n * ldwq + i] * dw_O[n]));
+                o += g * wd_main + g * wd_out;
+            }
+            row[O_idx[i]] = o / (double)s_O[i];
+        }
+        if (r > 0)
+            for (int k = 0; k < K; ++k) {
+                double l = 0.0;
+                for (int j = 0; j < r; ++j) l += (double)bf2f(G[(int64_t)m * r + j]) * (double)bf2f(A[(int64_t)k * r + j]);
+                row[k] += l;
+            }
+    }
+    free(Zq);
+    free(dz);
+    free(G);
+    return overflow;
+}
+
 /* ---------------------------------------------------------------- calibration, Eq. 6
  * One calibration sample X^i [M][K]:  xi[o] += 1  if  max_m |X[m][o]| > thr * mean(|X|).
  * So that the indicator is one well-defined integer decision, |x| is taken in units of 2^-16,

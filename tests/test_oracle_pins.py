@@ -474,6 +474,87 @@ def test_lora_gradients_by_finite_differences_of_the_forward():
     assert np.linalg.norm(dB - dB_true) / np.linalg.norm(dB_true) < 4e-3
 
 
+# ----------------------------------------------------------------------------- INT8 grad-input variant (not the paper's method)
+def test_quant_grad_hand_examples():
+    # Z = dY * Delta_W[n], then Eq. 1 per token.  Row 0: Z = (2.5, 3.5, -0.5, 127) -> amax 127, codes (2, 4, 0, 127): three ties.
+    # Row 1: the column scales change which entry is the row maximum: dY = (1, -2, 0.5, 4), Delta_W = (0.5, 0.5, 0.5, 0.5)
+    # -> Z = (0.5, -1, 0.25, 2) -> r = 63.5 -> (31.75 -> 32, -63.5 -> -64, 15.875 -> 16, 127).
+    dY = bf([[5.0, 7.0, -1.0, 254.0], [1.0, -2.0, 0.5, 4.0], [0.0, 0.0, 0.0, 0.0]])
+    dW = np.full(4, 0.5, np.float32)
+    Zq, dz = oracle.quant_grad(dY, dW)
+    assert Zq.tolist() == [[2, 4, 0, 127], [32, -64, 16, 127], [0, 0, 0, 0]]
+    assert dz.tolist() == [1.0, np.float32(2.0) / np.float32(127.0), 0.0]
+    # unequal column scales: dY = (8, 1), Delta_W = (0.125, 4) -> Z = (1, 4): the SECOND entry carries the maximum
+    Zq, dz = oracle.quant_grad(bf([[8.0, 1.0]]), np.array([0.125, 4.0], np.float32))
+    assert Zq.tolist() == [[32, 127]] and dz[0] == np.float32(4.0) / np.float32(127.0)
+
+
+def test_int8_backward_accumulators_brute_force_and_shared_parts():
+    rng = np.random.default_rng(51)
+    M, K, N, nO, r = 5, 24, 12, 2, 4
+    O, X, Wt, A, B, Wq, dW, W_O, wmax, s = _setup(rng, M, K, N, nO, r)
+    wq, dw = oracle.requant_weight_rows(W_O, s, 4)
+    T = oracle.lora_down(X, A)
+    dY = rand_bf(rng, (M, N), 1e-2)
+    dX8, dA8, dB8, G8, Zq, dz, acc = oracle.qlinear_bwd_int8(dY, Wq, dW, wq, dw, O, s, X, T, A, B, 0.5)
+    Zq2, dz2 = oracle.quant_grad(dY, dW)
+    assert np.array_equal(Zq, Zq2) and np.array_equal(dz, dz2)
+    for m in range(M):
+        for k in range(K):
+            assert int(acc[m, k]) == sum(int(Zq[m, n]) * int(Wq[n, k]) for n in range(N))
+    dX, dA, dB, G = oracle.qlinear_bwd(dY, Wq, dW, wq, dw, O, s, X, T, A, B, 0.5)
+    # G, dA, dB and the outlier columns are those of the floating-point backward
+    assert np.array_equal(G8, G) and np.array_equal(dA8, dA) and np.array_equal(dB8, dB)
+    assert np.allclose(dX8[:, O], dX[:, O], rtol=1e-12, atol=1e-18)
+    # the other columns: Dz[m] * acc + G A^T
+    rest = np.setdiff1d(np.arange(K), O)
+    lora = f32(G).astype(np.float64) @ f32(A).astype(np.float64).T
+    assert np.allclose(dX8[:, rest], (dz[:, None].astype(np.float64) * acc.astype(np.float64) + lora)[:, rest], rtol=1e-12, atol=1e-18)
+
+
+def test_int8_backward_is_exact_when_the_gradient_quantization_is_lossless():
+    """Integer-valued weight with column maxima 127 (codes = values, Delta_W = 1) and integer-valued dY with row maxima
+    127 (Zq = dY, Dz = 1): the INT8 variant then computes dY W^T exactly, and so does the floating-point backward."""
+    rng = np.random.default_rng(52)
+    M, K, N = 6, 20, 16
+    W = rng.integers(-127, 128, (N, K)).astype(np.float32)
+    W[:, 0] = 127.0                                                    # every output channel (row of Wt) has maximum 127
+    g = rng.integers(-127, 128, (M, N)).astype(np.float32)
+    g[:, 3] = -127.0
+    Wt, dY = bf(W), bf(g)
+    assert np.array_equal(f32(Wt), W) and np.array_equal(f32(dY), g)
+    O = np.zeros(0, np.int32)
+    Wq, dW, W_O, wmax = oracle.prepare_weight(Wt, O)
+    assert np.array_equal(Wq, W.astype(np.int8)) and (dW == 1.0).all()
+    none = np.zeros((N, 0), np.int8)
+    X = bf(np.zeros((M, K), np.float32))
+    dX8, _, _, _, Zq, dz, acc = oracle.qlinear_bwd_int8(dY, Wq, dW, none, np.zeros(N, np.float32), O, np.zeros(0, np.float32), X, None, None, None, 0.0)
+    assert np.array_equal(Zq, g.astype(np.int8)) and (dz == 1.0).all()
+    exact = g.astype(np.float64) @ W.astype(np.float64)
+    assert np.array_equal(dX8, exact)
+    dX = oracle.qlinear_bwd(dY, Wq, dW, none, np.zeros(N, np.float32), O, np.zeros(0, np.float32), X, None, None, None, 0.0)[0]
+    assert np.array_equal(dX, exact)
+
+
+def test_int8_backward_error_bound_against_the_floating_point_backward():
+    """Element by element: |dX_int8 - dX_fp| <= (Dz[m] / 2) sum_n |Wq[n][k]|  (rounding of Zq, Eq. 1)
+    + 2^-8 sum_n |Z[m][n] Wq[n][k]|  (the bf16 rounding of the dequantized weight on the other side, and of Z in fp32)."""
+    rng = np.random.default_rng(53)
+    M, K, N, nO = 16, 96, 64, 3
+    O, X, Wt, A, B, Wq, dW, W_O, wmax, s = _setup(rng, M, K, N, nO, 0)
+    wq, dw = oracle.requant_weight_rows(W_O, s, 4)
+    dY = rand_bf(rng, (M, N), 1e-2)
+    dX8, _, _, _, Zq, dz, acc = oracle.qlinear_bwd_int8(dY, Wq, dW, wq, dw, O, s, X, None, None, None, 0.0)
+    dX = oracle.qlinear_bwd(dY, Wq, dW, wq, dw, O, s, X, None, None, None, 0.0)[0]
+    Z = np.abs(f32(dY).astype(np.float64) * dW[None, :].astype(np.float64))
+    aW = np.abs(Wq.astype(np.float64))
+    bound = 0.5 * dz[:, None].astype(np.float64) * aW.sum(axis=0)[None, :] * (1 + 1e-6) + 2.0 ** -8 * (Z @ aW)
+    assert (np.abs(dX8 - dX) <= bound).all()
+    # and it is an approximation of the same thing: a few per cent of the gradient's norm
+    rest = np.setdiff1d(np.arange(K), O)
+    assert np.linalg.norm((dX8 - dX)[:, rest]) / np.linalg.norm(dX[:, rest]) < 3e-2
+
+
 # ----------------------------------------------------------------------------- generator sanity
 def test_synthetic_workload_shapes_and_outliers():
     wl = synth.WORKLOADS["tiny"]
