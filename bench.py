@@ -225,7 +225,7 @@ def run_gpu(args, wl):
         for li, lin in enumerate(lins):
             sp = lin.spec
             layer = QuaffLinear(to_bf16(lin.W), torch.from_numpy(lin.O_idx).cuda(), to_bf16(lin.A), to_bf16(lin.B),
-                                wl.lora_alpha / sp.r, wl.gamma, M)
+                                wl.lora_alpha / sp.r, wl.gamma, M, int8_grad=args.int8_grad)
             X, dY = synth.step_inputs(wl, li, qdist.batch_index(rep, rank), lin)
             layers.append(layer)
             xs.append(to_bf16(X)); dys.append(to_bf16(dY))
@@ -425,6 +425,9 @@ def run_gpu(args, wl):
     peak_note = f"{peaks['source']} cuBLAS bf16 {'sustained' if sustained else 'burst'}"
     per_layer = []
     dominant = None
+    # the grad-input GEMM runs in bf16 (the paper quantizes no gradient); with --int8-grad it is the INT8 variant's kernel
+    bwd_peak = bf16_peak * (2.0 if args.int8_grad else 1.0)
+    bwd_unit = "TOP/s" if args.int8_grad else "TFLOP/s"
     for li, sp in enumerate(wl.layers):
         nOp = synth.pad_to(sp.nO, 32)
         f_ms, b_ms = gemm_ms[li]
@@ -438,7 +441,7 @@ def run_gpu(args, wl):
                  "bwd_gemm_ms": b_ms, "bwd_bf16_tflops": b_tflops,
                  "bwd_pct_of_bf16_nominal_2250": 100.0 * b_tflops / 2.25e3,
                  "bwd_pct_of_int8_nominal_4500": 100.0 * b_tflops / 4.5e3,
-                 "bwd_roofline": {"bound": "tensor", "achieved": b_tflops, "peak": bf16_peak, "unit": "TFLOP/s", "frac": b_tflops / bf16_peak,
+                 "bwd_roofline": {"bound": "tensor", "achieved": b_tflops, "peak": bwd_peak, "unit": bwd_unit, "frac": b_tflops / bwd_peak,
                                   "traffic": ncu_traffic.get(("bwd_bf16_gemm", M, sp.K, sp.N, sp.nO, sp.r))}}
         per_layer.append(entry)
         for kind, ms, work in (("fwd_int8_gemm", f_ms, fwd_int8 + fwd_lora), ("bwd_bf16_gemm", b_ms, bwd_bf16)):
@@ -446,16 +449,19 @@ def run_gpu(args, wl):
                 dominant = (sp.name, kind, ms, work, ncu_traffic.get((kind, M, sp.K, sp.N, sp.nO, sp.r)))
     name, kind, ms, work, traffic = dominant
     achieved = work / (ms * 1e-3) / 1e12
-    peak = bf16_peak * (2.0 if kind == "fwd_int8_gemm" else 1.0)
-    roofline = {"bound": "tensor", "kernel": f"{'forward INT8 GEMM (Eq. 9 + LoRA)' if kind == 'fwd_int8_gemm' else 'umma_gemm_kernel<EPI_BWD> grad-input GEMM'} ({name})",
-                "achieved": achieved, "peak": peak, "unit": "TFLOP/s" if kind == "bwd_bf16_gemm" else "TOP/s",
+    int8_kernel = kind == "fwd_int8_gemm" or args.int8_grad
+    peak = bf16_peak * (2.0 if int8_kernel else 1.0)
+    kname = ("forward INT8 GEMM (Eq. 9 + LoRA)" if kind == "fwd_int8_gemm" else
+             "INT8 grad-input GEMM (variant, not the paper's method)" if args.int8_grad else "umma_gemm_kernel<EPI_BWD> grad-input GEMM")
+    roofline = {"bound": "tensor", "kernel": f"{kname} ({name})",
+                "achieved": achieved, "peak": peak, "unit": "TOP/s" if int8_kernel else "TFLOP/s",
                 "frac": achieved / peak, "traffic": traffic,
-                "peak_source": peak_note + (" x2 (nominal int8:bf16 ratio)" if kind == "fwd_int8_gemm" else "")
+                "peak_source": peak_note + (" x2 (nominal int8:bf16 ratio)" if int8_kernel else "")
                                + f"; the timed region ran {timed_total_ms:.0f} ms",
                 "avg_launch_ms": ms,
                 "timing": f"CUDA event pair around the kernel in an instrumented pass over the same steps ({inst_steps} steps, "
                           f"{inst_ms_per_step:.4f} ms per step with the event nodes in the graph)"}
-    if kind == "bwd_bf16_gemm":
+    if kind == "bwd_bf16_gemm" and not args.int8_grad:
         # Inside the step the grad-input GEMM shares the SMs: the split-K GEMMs of dA and dB are scheduled into the SMs
         # its last wave leaves idle, which shortens the step and lengthens the GEMM.  The same kernel alone (a backward
         # call for dX only on the same layer's buffers, L2 flushed before it) is reported beside it.
@@ -487,9 +493,11 @@ def run_gpu(args, wl):
             "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
             "repeats": {"n": args.repeats, "ms_per_step_min": float(np.min(region_ms)) / args.steps,
                         "ms_per_step_max": float(np.max(region_ms)) / args.steps, "ms_per_step_median": ms_per_step},
-            "vs_baseline": None, "dtype": "int8 forward (int32 accumulate), bf16 backward (f32 accumulate)",
+            "vs_baseline": None, "dtype": "int8 forward (int32 accumulate), " + ("int8 grad-input (variant)" if args.int8_grad else "bf16 backward (f32 accumulate)"),
             "data": "synthetic",
             "config": {"workload": wl.name, "tokens_per_gpu": M,
+                       "backward": "INT8 grad-input variant (NOT the paper's method; reported separately)" if args.int8_grad
+                                   else "bf16 grad-input through the dequantized INT8 weight (the paper quantizes no gradient)",
                        "layers": [f"{l.name} {l.K}->{l.N} nO={l.nO} r={l.r}" for l in wl.layers], "gamma": wl.gamma,
                        "l2": f"rotating {REPLICAS} full buffer sets (weights, activations, outputs); one set alone exceeds the 126 MB L2",
                        "launch": "eager" if args.eager else "one CUDA graph replay per step"},
@@ -703,6 +711,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--micro-rank", type=int, default=64, help="LoRA rank of --micro fwd / bwd")
     ap.add_argument("--workload", default="llama7b_block", choices=sorted(synth.WORKLOADS) + ["sweep"])
+    ap.add_argument("--int8-grad", action="store_true",
+                    help="run the backward through quaff_qlinear_bwd_int8, the INT8 grad-input variant (not the paper's method)")
     ap.add_argument("--sweep-quick", action="store_true", help="--workload sweep on a 2 x 2 x 2 corner of the (M, K, N) grid only")
     ap.add_argument("--repeats", type=int, default=30, help="how often the timed region of --steps steps is repeated (median reported)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])

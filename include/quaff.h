@@ -62,7 +62,8 @@ enum { /* `which` of quaff_workspace_bytes */
     QUAFF_WS_FWD = 2,
     QUAFF_WS_BWD = 3,
     QUAFF_WS_CALIBRATE = 4,  /* quaff_outlier_count and quaff_select_outliers (depends on K only) */
-    QUAFF_WS_HITS = 5        /* quaff_outlier_hits (depends on K only) */
+    QUAFF_WS_HITS = 5,       /* quaff_outlier_hits (depends on K only) */
+    QUAFF_WS_BWD_INT8 = 6    /* quaff_qlinear_bwd_int8 */
 };
 
 const char* quaff_status_string(quaff_status_t s);
@@ -248,6 +249,33 @@ quaff_status_t quaff_qlinear_bwd(int M, int K, int N,
                                  quaff_bf16* dX, int64_t lddx,
                                  float* dA, float* dB, int accumulate, quaff_bf16* G_out_opt,
                                  int32_t* status_opt, void* ws, size_t ws_bytes, quaff_stream_t stream);
+
+/*
+ * INT8 grad-input variant of the backward.  NOT the paper's method: the paper quantizes no gradient (Sec. 4.1 keeps the
+ * model in floating point, Sec. 3.3 states a forward only), so this entry point is never what quaff_qlinear_bwd does
+ * and its results are reported separately.  It puts the grad-input GEMM, the largest cost of a step, on the INT8
+ * tensor path: the per-output-channel step sizes lie on the backward's contraction axis, so they are folded into dY
+ * before a per-token quantization,
+ *   Z[m][n] = dY[m][n] * dW[n] ;  dz[m] = max_n |Z[m][n]| / 127 ;  Zq[m][n] = round_to_nearest_even(Z[m][n] * (127 / max_n|Z[m][n]|))
+ *   dXhat[m][k] = dz[m] * sum_n Zq[m][n] * Wq[n][k]                      (INT8 x INT8 -> INT32, Wq read in place)
+ * for every k outside O; the nO outlier columns keep the floating-point path of quaff_qlinear_bwd,
+ *   dXhat[m][O_i] = (sum_n dY[m][n] (Wd[n][O_i] + wd[n][i])) / s_O[i].
+ * G, dX = dXhat + G A^T, dA, dB and all other arguments are those of quaff_qlinear_bwd; dX is required; N must be a
+ * multiple of 16; dbg_acc_opt: optional dense [M][K] int32 dump of sum_n Zq Wq (parity checks);  ws: QUAFF_WS_BWD_INT8 bytes.
+ * quaff_quant_grad is the quantization step on its own (Zq [M][N] int8 with ldz % 16 == 0, dz [M] f32).
+ */
+quaff_status_t quaff_quant_grad(const quaff_bf16* dY, int64_t lddy, int M, int N, const float* dW, int8_t* Zq, int64_t ldz,
+                                float* dz, quaff_stream_t stream);
+quaff_status_t quaff_qlinear_bwd_int8(int M, int K, int N,
+                                      const quaff_bf16* dY, int64_t lddy,
+                                      const int8_t* Wq, int64_t ldwq_main, const float* dW,
+                                      const int8_t* wq_O, int64_t ldwq, const float* dw_O, int nOp,
+                                      const int32_t* O_idx, int nO, const float* s_O,
+                                      const quaff_bf16* X, int64_t ldx, const quaff_bf16* T,
+                                      const quaff_bf16* A, const quaff_bf16* B, int r, float lora_scale,
+                                      quaff_bf16* dX, int64_t lddx,
+                                      float* dA, float* dB, int accumulate, quaff_bf16* G_out_opt, int32_t* dbg_acc_opt,
+                                      int32_t* status_opt, void* ws, size_t ws_bytes, quaff_stream_t stream);
 
 /*
  * quaff_momentum_update without a caller-supplied workspace (the paper has no counterpart: this

@@ -22,10 +22,10 @@ QUAFF_ERR_WORKSPACE_TOO_SMALL = 4
 QUAFF_ERR_CUDA = 5
 QUAFF_ERR_TIMEOUT = 6
 QUAFF_BF16, QUAFF_F32 = 0, 1
-QUAFF_WS_PREPARE, QUAFF_WS_MOMENTUM, QUAFF_WS_FWD, QUAFF_WS_BWD, QUAFF_WS_CALIBRATE, QUAFF_WS_HITS = 0, 1, 2, 3, 4, 5
+QUAFF_WS_PREPARE, QUAFF_WS_MOMENTUM, QUAFF_WS_FWD, QUAFF_WS_BWD, QUAFF_WS_CALIBRATE, QUAFF_WS_HITS, QUAFF_WS_BWD_INT8 = 0, 1, 2, 3, 4, 5, 6
 
 EXPORTS = ("quaff_status_string", "quaff_workspace_bytes", "quaff_debug_launch_count", "quaff_debug_force_fwd_tile", "quaff_debug_time_gemm", "quaff_prepare_weight", "quaff_momentum_update", "quaff_lora_down", "quaff_outlier_count", "quaff_select_outliers", "quaff_outlier_hits",
-           "quaff_momentum_update_static", "quaff_outlier_colmax", "quaff_momentum_apply", "quaff_quant_act", "quaff_requant_weight_rows", "quaff_qlinear_fwd", "quaff_qlinear_bwd")
+           "quaff_momentum_update_static", "quaff_outlier_colmax", "quaff_momentum_apply", "quaff_quant_act", "quaff_requant_weight_rows", "quaff_qlinear_fwd", "quaff_qlinear_bwd", "quaff_quant_grad", "quaff_qlinear_bwd_int8")
 
 _lib = None
 _vp, _i64, _i32, _f32, _sz = ctypes.c_void_p, ctypes.c_int64, ctypes.c_int, ctypes.c_float, ctypes.c_size_t
@@ -82,6 +82,11 @@ def lib() -> ctypes.CDLL:
         L.quaff_qlinear_bwd.restype = _i32
         L.quaff_qlinear_bwd.argtypes = [_i32, _i32, _i32, _vp, _i64, _vp, _i64, _vp, _vp, _i64, _vp, _i32, _vp, _i32, _vp,
                                         _vp, _i64, _vp, _vp, _vp, _i32, _f32, _vp, _i64, _vp, _vp, _i32, _vp, _vp, _vp, _sz, _vp]
+        L.quaff_qlinear_bwd_int8.restype = _i32
+        L.quaff_qlinear_bwd_int8.argtypes = [_i32, _i32, _i32, _vp, _i64, _vp, _i64, _vp, _vp, _i64, _vp, _i32, _vp, _i32, _vp,
+                                             _vp, _i64, _vp, _vp, _vp, _i32, _f32, _vp, _i64, _vp, _vp, _i32, _vp, _vp, _vp, _vp, _sz, _vp]
+        L.quaff_quant_grad.restype = _i32
+        L.quaff_quant_grad.argtypes = [_vp, _i64, _i32, _i32, _vp, _vp, _i64, _vp, _vp]
         L.quaff_debug_launch_count.restype = ctypes.c_uint64
         L.quaff_debug_launch_count.argtypes = []
         L.quaff_debug_force_fwd_tile.restype = None
@@ -249,3 +254,26 @@ def quaff_qlinear_bwd(dY, Wq, dW, wq_O, dw_O, O_idx, s_O, X, T, A, B, lora_scale
                                    1 if accumulate else 0, _ptr(G_out), _ptr(status), _ptr(ws),
                                    ws.numel() * ws.element_size() if ws is not None else 0, _stream()),
            "quaff_qlinear_bwd")
+
+
+def quaff_quant_grad(dY, dW, Zq, dz) -> None:
+    """Z = dY * dW[n] quantized per token (the INT8 grad-input variant's first step)."""
+    M, N = dY.shape
+    _check(lib().quaff_quant_grad(_ptr(dY), _ld(dY), M, N, _ptr(dW), _ptr(Zq), _ld(Zq), _ptr(dz), _stream()), "quaff_quant_grad")
+
+
+def quaff_qlinear_bwd_int8(dY, Wq, dW, wq_O, dw_O, O_idx, s_O, X, T, A, B, lora_scale: float, dX, dA, dB,
+                           accumulate: bool, ws, status=None, G_out=None, dbg_acc=None) -> None:
+    """The INT8 grad-input variant of the backward (not the paper's method)."""
+    M, N = dY.shape
+    K = Wq.shape[1]
+    nOp = 0 if wq_O is None else wq_O.shape[1]
+    nO = 0 if O_idx is None else O_idx.numel()
+    r = 0 if A is None else A.shape[1]
+    _check(lib().quaff_qlinear_bwd_int8(M, K, N, _ptr(dY), _ld(dY), _ptr(Wq), _ld(Wq), _ptr(dW), _ptr(wq_O),
+                                        _ld(wq_O) if wq_O is not None else 0, _ptr(dw_O), nOp, _ptr(O_idx), nO, _ptr(s_O),
+                                        _ptr(X), _ld(X) if X is not None else 0, _ptr(T), _ptr(A), _ptr(B), r,
+                                        float(lora_scale), _ptr(dX), _ld(dX), _ptr(dA), _ptr(dB),
+                                        1 if accumulate else 0, _ptr(G_out), _ptr(dbg_acc), _ptr(status), _ptr(ws),
+                                        ws.numel() * ws.element_size() if ws is not None else 0, _stream()),
+           "quaff_qlinear_bwd_int8")

@@ -33,6 +33,10 @@ inline quaff_status_t launch_status() {
 
 int sm_count();  // SMs of the current device (cached)
 
+// Z = dY * colscale[n] quantized per token (the INT8 grad-input variant): Zq [M][N] int8, dz [M]; N a multiple of 16
+quaff_status_t quant_grad_dispatch(const uint16_t* dY, int64_t lddy, int M, int N, const float* colscale, int8_t* Zq, int64_t ldz,
+                                   float* dz, cudaStream_t st);
+
 // Every kernel of this library is launched with programmatic stream serialization: it may be scheduled
 // while its predecessor in the stream is still running, and it orders itself behind that predecessor with
 // griddepcontrol.wait (pdl_wait) before its first access to global memory.  The launch latency, the CTA

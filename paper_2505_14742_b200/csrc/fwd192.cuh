@@ -64,6 +64,9 @@ struct FwdWideParams {
     int y_f32;
     int32_t* dbg_main;
     int32_t* dbg_out;
+    // fwd256_kernel only (the INT8 grad-input variant runs through it with the roles of the matrices exchanged):
+    int wq_mn;                       // 1: map_wq is [contraction][output columns] (MN-major B operand), boxes of 128 x 128 bytes
+    int lora_kmajor;                 // 1: map_bt is [output columns][contraction] bf16 (K-major), boxes of 64 rows x 64 elements
 };
 
 // The ring schedule of one CTA pair: calls main_fn(t, tile, b) for every main k-block and aux_fn(t, tile, j)

@@ -67,6 +67,10 @@ __device__ __forceinline__ void for_each_item256(int unit, int nunits, int ntile
 
 // Parameters: FwdWideParams with the boxes of map_wq 128 rows and of map_wo 64 rows high;
 // map_bt is LoRA B [r][N] itself, boxes of rp contraction rows x 64 columns.
+// The INT8 grad-input variant uses the same kernel with the matrices in other roles (A operand = the quantized
+// gradient Zq [M][N], contraction over N): its weight operand is Wq [N][K] read IN PLACE with the contraction index as
+// the row (p.wq_mn: an MN-major INT8 operand, one box = 128 contraction rows x 128 output columns, so a CTA's half of
+// the tile is exactly one box), its LoRA operand is A [K][r] (p.lora_kmajor), and a null p.dW means column scale 1.
 __global__ void __launch_bounds__(kF256Threads, 1) fwd256_kernel(const __grid_constant__ FwdWideParams p) {
     constexpr int TN = kF256TN;
     constexpr int kStages = kF256Stages;
@@ -137,12 +141,15 @@ __global__ void __launch_bounds__(kF256Threads, 1) fwd256_kernel(const __grid_co
                 return true;
             };
             const uint32_t tx_main = kABytes + (TN / 2) * 128, tx_aux = kABytes + (kF256Round / 2) * 128;
-            const uint32_t tx_lora = kABytes + (uint32_t)p.nmma_l * 16u * 128u;      // B: one box of 64 columns x rp contraction rows
+            // LoRA B: one box of 64 columns x rp contraction rows (MN-major), or of 64 output columns x 64 elements (K-major)
+            const uint32_t tx_lora = kABytes + (p.lora_kmajor ? 64u * 128u : (uint32_t)p.nmma_l * 16u * 128u);
             int tm = 0, tn = 0;
             for_each_item256(unit, nunits, ntiles, p.nblk,
                 [&](int, int tile, int b) -> bool {
                     if (b == 0) tile_coords(tile, p.tiles_m, p.tiles_n, p.band_m, tm, tn);   // once per tile: this loop is the issue path
-                    return load_stage(&p.map_xq, &p.map_wq, b * 128, tm * 256 + (int)rank * kTileM, tn * TN + (int)rank * (TN / 2), tx_main);
+                    const int nb0 = tn * TN + (int)rank * (TN / 2);
+                    if (p.wq_mn) return load_stage(&p.map_xq, &p.map_wq, b * 128, tm * 256 + (int)rank * kTileM, b * 128, tx_main, nb0);
+                    return load_stage(&p.map_xq, &p.map_wq, b * 128, tm * 256 + (int)rank * kTileM, nb0, tx_main);
                 },
                 [&](int, int tile, int j) -> bool {
                     int tm, tn;
@@ -151,7 +158,8 @@ __global__ void __launch_bounds__(kF256Threads, 1) fwd256_kernel(const __grid_co
                     const int nr = tn * TN + j * kF256Round + (int)rank * (kF256Round / 2);
                     if (p.nmma_o && !load_stage(&p.map_xo, &p.map_wo, 0, m0, nr, tx_aux)) return false;
                     // LoRA B [r][N] is read in place: MN-major, coordinates (column, contraction row)
-                    if (p.nmma_l && !load_stage(&p.map_t, &p.map_bt, 0, m0, 0, tx_lora, nr)) return false;
+                    if (p.nmma_l && !(p.lora_kmajor ? load_stage(&p.map_t, &p.map_bt, 0, m0, nr, tx_lora)
+                                                    : load_stage(&p.map_t, &p.map_bt, 0, m0, 0, tx_lora, nr))) return false;
                     return true;
                 });
         }
@@ -159,20 +167,22 @@ __global__ void __launch_bounds__(kF256Threads, 1) fwd256_kernel(const __grid_co
         // ------------------------------------------------------------------ MMA issuer (the leader's, for the pair)
         if (rank == 0 && elect_one()) {
             uint32_t stage = 0, phase = 0;
-            const uint32_t idesc_main = umma_idesc(kCFmtS32, kFmtS8, 256, TN);
+            const uint32_t idesc_main = umma_idesc(kCFmtS32, kFmtS8, 256, TN) | (p.wq_mn ? (1u << 16) : 0u);
             const uint32_t idesc_o = umma_idesc(kCFmtS32, kFmtS8, 256, kF256Round);
-            const uint32_t idesc_l = umma_idesc(kCFmtF32, kFmtBF16, 256, kF256Round) | (1u << 16);     // B is MN-major
+            const uint32_t idesc_l = umma_idesc(kCFmtF32, kFmtBF16, 256, kF256Round) | (p.lora_kmajor ? 0u : (1u << 16));   // bit 16: B is MN-major
             // consume one ring stage with `nmma` MMAs of 32 contraction bytes each
             // (K-major operands advance 32 bytes inside the swizzled row per MMA; the MN-major B of the LoRA round
             // advances 16 contraction rows = 2048 bytes, its leading byte offset - the distance between boxes of 64
             // columns - is not used with a single box)
-            auto mma_stage = [&](uint32_t acc, uint32_t idesc, bool i8, int nmma, uint32_t& accumulate) -> bool {
+            // b_mn: the B operand of this stage is MN-major.  One MMA then consumes 32 bytes of contraction = 16 rows of
+            // bf16 or 32 rows of INT8, rows being 128 bytes apart: an advance of 2048 resp. 4096 bytes.
+            auto mma_stage = [&](uint32_t acc, uint32_t idesc, bool i8, bool b_mn, int nmma, uint32_t& accumulate) -> bool {
                 if (!mbar_wait(full0 + 8u * stage, phase, abort_flag)) return false;
                 tc_fence_after();
                 const uint32_t s_lo = ((tiles_base + stage * kStageBytes) & 0x3FFFFu) >> 4;
                 const uint32_t a_lo = s_lo | (1u << 16);
-                const uint32_t b_lo = i8 ? a_lo + (kABytes >> 4) : ((s_lo + (kABytes >> 4)) | ((uint32_t)(kAtomBytes >> 4) << 16));
-                const uint32_t b_adv = i8 ? 2u : (2048u >> 4);
+                const uint32_t b_lo = !b_mn ? a_lo + (kABytes >> 4) : ((s_lo + (kABytes >> 4)) | ((uint32_t)(kAtomBytes >> 4) << 16));
+                const uint32_t b_adv = !b_mn ? 2u : (i8 ? (4096u >> 4) : (2048u >> 4));
 #pragma unroll
                 for (int k = 0; k < 4; ++k) {
                     if (k < nmma) {
@@ -189,7 +199,7 @@ __global__ void __launch_bounds__(kF256Threads, 1) fwd256_kernel(const __grid_co
             for_each_item256(unit, nunits, ntiles, p.nblk,
                 [&](int, int, int b) -> bool {
                     if (b == 0) acc_main = 0u;
-                    return mma_stage(tmem_base, idesc_main, true, b == p.nblk - 1 ? p.nmma_last : 4, acc_main);
+                    return mma_stage(tmem_base, idesc_main, true, p.wq_mn != 0, b == p.nblk - 1 ? p.nmma_last : 4, acc_main);
                 },
                 [&](int t, int, int j) -> bool {
                     if (j == 0) {
@@ -203,9 +213,9 @@ __global__ void __launch_bounds__(kF256Threads, 1) fwd256_kernel(const __grid_co
                     }
                     tc_fence_after();
                     uint32_t acc = 0u;
-                    if (p.nmma_o && !mma_stage(tmem_base + kColAuxO, idesc_o, true, p.nmma_o, acc)) return false;
+                    if (p.nmma_o && !mma_stage(tmem_base + kColAuxO, idesc_o, true, false, p.nmma_o, acc)) return false;
                     acc = 0u;
-                    if (p.nmma_l && !mma_stage(tmem_base + kColAuxL, idesc_l, false, p.nmma_l, acc)) return false;
+                    if (p.nmma_l && !mma_stage(tmem_base + kColAuxL, idesc_l, false, !p.lora_kmajor, p.nmma_l, acc)) return false;
                     umma_commit<2>(j == 0 ? tmem_full_bar : aux_ready_bar);
                     return true;
                 });
@@ -295,7 +305,7 @@ __global__ void __launch_bounds__(kF256Threads, 1) fwd256_kernel(const __grid_co
 #pragma unroll
             for (int jj = 0; jj < 2; ++jj) {
                 const int n = n0 + jj * kF256Round + cq * 32 + lane;
-                scale_w[jj * 32 + lane] = n < p.N ? __ldg(p.dW + n) : 0.0f;
+                scale_w[jj * 32 + lane] = n < p.N ? (p.dW ? __ldg(p.dW + n) : 1.0f) : 0.0f;
                 scale_o[jj * 32 + lane] = (n < p.N && has_o) ? __ldg(p.dw_O + n) : 0.0f;
             }
             __syncwarp();

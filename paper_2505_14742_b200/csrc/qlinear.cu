@@ -184,7 +184,7 @@ static quaff_status_t launch_gemm(const GemmParams& p, cudaStream_t st) {
 }
 
 // The wide forward kernels (fwd192.cuh, fwd256.cuh): which = 0 / 1
-static quaff_status_t launch_fwd_wide(int which, const FwdWideParams& p, cudaStream_t st) {
+static quaff_status_t launch_fwd_wide(int which, const FwdWideParams& p, cudaStream_t st, int time_slot = 0) {
     static std::atomic<bool> configured[2][64];
     static std::atomic<int> units_of[2][64];
     void (*const kernel)(const FwdWideParams) = which ? fwd256_kernel : fwd192_kernel;
@@ -214,18 +214,18 @@ static quaff_status_t launch_fwd_wide(int which, const FwdWideParams& p, cudaStr
     const int ntiles = p.tiles_m * p.tiles_n;
     if (ntiles == 0) return QUAFF_OK;
     const int units = min(ntiles, units_of[which][dev].load());
-    const bool timed = g_time_start[0] && g_time_stop[0];
+    const bool timed = g_time_start[time_slot] && g_time_stop[time_slot];
     unsigned int ev_flags = cudaEventRecordDefault;
     if (timed) {
         cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
         if (cudaStreamIsCapturing(st, &cap) == cudaSuccess && cap == cudaStreamCaptureStatusActive) ev_flags = cudaEventRecordExternal;
-        cudaEventRecordWithFlags(g_time_start[0], st, ev_flags);
+        cudaEventRecordWithFlags(g_time_start[time_slot], st, ev_flags);
     }
     launch_pdl(kernel, dim3(units * 2), dim3(threads), smem, st, 2, p);
     const quaff_status_t rc = launch_status();
     if (timed) {
-        cudaEventRecordWithFlags(g_time_stop[0], st, ev_flags);
-        g_time_start[0] = g_time_stop[0] = nullptr;
+        cudaEventRecordWithFlags(g_time_stop[time_slot], st, ev_flags);
+        g_time_start[time_slot] = g_time_stop[time_slot] = nullptr;
     }
     return rc;
 }
@@ -523,6 +523,24 @@ static BwdWorkspace bwd_workspace(int M, int K, int N, int nOp, int r) {
     return w;
 }
 
+// INT8 grad-input variant: the quantized gradient Zq [M][N], its step sizes, the dequantized outlier columns
+// Wd_O [N][2 nOp] (the only bf16 weight data: the outlier columns stay on the floating-point path), G, P, split-K partials.
+struct BwdInt8Workspace { size_t off_zq, off_dz, off_wdo, off_g, off_p, off_part, off_part_a, off_part_b, total; };
+static BwdInt8Workspace bwd_int8_workspace(int M, int K, int N, int nOp, int r) {
+    BwdInt8Workspace w;
+    size_t off = 0;
+    w.off_zq = off;   off += round_up((size_t)M * (size_t)N, 256);
+    w.off_dz = off;   off += round_up((size_t)M * 4, 256);
+    w.off_wdo = off;  off += round_up((size_t)N * (size_t)max(2 * nOp, 1) * 2, 256);
+    w.off_g = off;    off += round_up((size_t)M * (size_t)max(r, 1) * 2, 256);
+    w.off_p = off;    off += round_up((size_t)M * (size_t)max(2 * nOp, 1) * 4, 256);
+    w.off_part = off;   off += round_up(split_part_bytes(M, N, r), 256);
+    w.off_part_a = off; off += round_up(split_part_bytes(K, M, r), 256);
+    w.off_part_b = off; off += round_up(split_part_bytes(N, M, r), 256);
+    w.total = off;
+    return w;
+}
+
 // T = bf16(X A): At = A^T (K-major operand), split-K tensor-core GEMM over K, reduction to bf16
 static quaff_status_t lora_down(const quaff_bf16* X, int64_t ldx, int M, int K, const quaff_bf16* A, int r, quaff_bf16* T_out,
                                 const FwdWorkspace& w, void* ws, int32_t* status_opt, cudaStream_t st) {
@@ -585,6 +603,7 @@ extern "C" size_t quaff_workspace_bytes(int which, int M, int K, int N, int nOp,
         case QUAFF_WS_MOMENTUM: return round_up((size_t)(nOp + 1) * 4, 256);
         case QUAFF_WS_FWD: return fwd_workspace(M, K, N, r).total;
         case QUAFF_WS_BWD: return bwd_workspace(M, K, N, nOp, r).total;
+        case QUAFF_WS_BWD_INT8: return bwd_int8_workspace(M, K, N, nOp, r).total;
         case QUAFF_WS_CALIBRATE: return round_up((size_t)max(K, 0) * 4, 256) + 256;   // column maxima / flags, sum, ticket
         case QUAFF_WS_HITS: return 2 * round_up((size_t)max(K, 0) * 4, 256) + 256;    // the same, then this batch's indicator
     }
@@ -861,6 +880,155 @@ extern "C" quaff_status_t quaff_qlinear_bwd(int M, int K, int N, const quaff_bf1
         if ((rc = launch_status()) != QUAFF_OK) return leave(rc);
     }
     if (dX && nO > 0) {
+        launch_pdl(bwd_fixup_kernel, dim3(ceil_div(M * nO, 256)), dim3(256), 0, st, 1, P, (int64_t)(2 * nOp), M, nO, nOp, O_idx, s_O, G, A, r,
+                   dX, lddx);
+        if ((rc = launch_status()) != QUAFF_OK) return leave(rc);
+    }
+    return leave(QUAFF_OK);
+}
+
+// The INT8 grad-input variant (not the paper's method; see quaff.h).  Kernels: quant_grad (Z = dY Delta_W quantized per
+// token), the 256-column INT8 kernel of the forward with the frozen codes Wq [N][K] read in place as an MN-major operand
+// (contraction over N) and G A^T in its LoRA rounds, and - for the nO outlier columns only - the floating-point path of
+// quaff_qlinear_bwd on the dequantized outlier columns (a grad-input GEMM with 2 nOp output columns, then the fix-up).
+extern "C" quaff_status_t quaff_qlinear_bwd_int8(int M, int K, int N, const quaff_bf16* dY, int64_t lddy, const int8_t* Wq,
+                                                 int64_t ldwq_main, const float* dW, const int8_t* wq_O, int64_t ldwq,
+                                                 const float* dw_O, int nOp, const int32_t* O_idx, int nO, const float* s_O,
+                                                 const quaff_bf16* X, int64_t ldx, const quaff_bf16* T, const quaff_bf16* A,
+                                                 const quaff_bf16* B, int r, float lora_scale, quaff_bf16* dX, int64_t lddx,
+                                                 float* dA, float* dB, int accumulate, quaff_bf16* G_out_opt,
+                                                 int32_t* dbg_acc_opt, int32_t* status_opt, void* ws, size_t ws_bytes,
+                                                 quaff_stream_t stream) {
+    QUAFF_RETURN_IF(M < 0 || K <= 0 || N <= 0 || nOp < 0 || nO < 0 || nO > nOp || r < 0, QUAFF_ERR_INVALID_ARG);
+    QUAFF_RETURN_IF(!dY || lddy < N || !Wq || !dW || ldwq_main < K || !dX || lddx < K, QUAFF_ERR_INVALID_ARG);
+    QUAFF_RETURN_IF(nOp > 0 && (!wq_O || !dw_O || ldwq < nOp), QUAFF_ERR_INVALID_ARG);
+    QUAFF_RETURN_IF(nO > 0 && (!O_idx || !s_O), QUAFF_ERR_INVALID_ARG);
+    QUAFF_RETURN_IF(r > 0 && (!A || !B), QUAFF_ERR_INVALID_ARG);
+    QUAFF_RETURN_IF(r > 0 && (dA || dB) && (!dA || !dB || !X || !T || ldx < K), QUAFF_ERR_INVALID_ARG);
+    QUAFF_RETURN_IF((nOp % 32) || (r % 8) || r > 64 || (N % 16), QUAFF_ERR_UNSUPPORTED_SHAPE);
+    QUAFF_RETURN_IF(!aligned16(dY) || (lddy % 8) || !aligned16(dW), QUAFF_ERR_ALIGNMENT);
+    QUAFF_RETURN_IF(!aligned16(Wq) || (ldwq_main % 16), QUAFF_ERR_ALIGNMENT);
+    QUAFF_RETURN_IF(nOp > 0 && (!aligned16(wq_O) || (ldwq % 16)), QUAFF_ERR_ALIGNMENT);
+    QUAFF_RETURN_IF(!aligned16(dX) || (lddx % 8), QUAFF_ERR_ALIGNMENT);
+    QUAFF_RETURN_IF(r > 0 && (!aligned16(A) || !aligned16(B) || (G_out_opt && !aligned16(G_out_opt))), QUAFF_ERR_ALIGNMENT);
+    QUAFF_RETURN_IF(r > 0 && dA && (!aligned16(X) || !aligned16(T) || !aligned16(dA) || !aligned16(dB) || (ldx % 8)), QUAFF_ERR_ALIGNMENT);
+    const BwdInt8Workspace w = bwd_int8_workspace(M, K, N, nOp, r);
+    QUAFF_RETURN_IF(!ws || !aligned16(ws) || ws_bytes < w.total, QUAFF_ERR_WORKSPACE_TOO_SMALL);
+    if (M == 0) return QUAFF_OK;
+    cudaStream_t st = (cudaStream_t)stream;
+    unsigned char* base = reinterpret_cast<unsigned char*>(ws);
+    int8_t* Zq = reinterpret_cast<int8_t*>(base + w.off_zq);
+    float* dz = reinterpret_cast<float*>(base + w.off_dz);
+    uint16_t* WdO = reinterpret_cast<uint16_t*>(base + w.off_wdo);
+    uint16_t* G = (r > 0 && G_out_opt) ? G_out_opt : reinterpret_cast<uint16_t*>(base + w.off_g);
+    float* P = reinterpret_cast<float*>(base + w.off_p);
+    float* part = reinterpret_cast<float*>(base + w.off_part);
+    float* part_a = reinterpret_cast<float*>(base + w.off_part_a);
+    float* part_b = reinterpret_cast<float*>(base + w.off_part_b);
+    quaff_status_t rc;
+    const bool want_dAB = r > 0 && dA && dB;
+    constexpr int CTAS = 2;
+
+    // ---- every tensor map and launch parameter first
+    SkinnyGemm gemm_g, gemm_db, gemm_da;
+    if (r > 0 && (rc = skinny_prepare(gemm_g, 0, dY, lddy, B, N, M, N, r, part, status_opt)) != QUAFF_OK) return rc;
+    FwdWideParams q;                                  // main: acc = Zq Wq over N; epilogue dX = dz[m] acc + G A^T
+    memset(&q, 0, sizeof(q));
+    if ((rc = make_tmap_2d(&q.map_xq, Zq, 1, M, N, N, kTileM, 128)) != QUAFF_OK) return rc;
+    if ((rc = make_tmap_2d(&q.map_wq, Wq, 1, N, K, ldwq_main, 128, 128)) != QUAFF_OK) return rc;     // rows = contraction index n
+    q.wq_mn = 1;
+    q.nblk = ceil_div(N, 128);
+    q.nmma_last = ceil_div(N - (q.nblk - 1) * 128, 32);
+    if (r > 0) {
+        if ((rc = make_tmap_2d(&q.map_t, G, 2, M, r, r, kTileM, 64)) != QUAFF_OK) return rc;
+        if ((rc = make_tmap_2d(&q.map_bt, A, 2, K, r, r, kF256Round / 2, 64)) != QUAFF_OK) return rc;
+        q.lora_kmajor = 1;
+        q.nmma_l = pad16(r) / 16;
+    }
+    q.M = M; q.N = K;
+    q.tiles_m = ceil_div(M, 2 * kTileM); q.tiles_n = ceil_div(K, kF256TN);
+    q.band_m = band_rows(q.tiles_m, q.tiles_n, 2 * kTileM, (size_t)N);
+    q.status = status_opt;
+    q.dx = dz; q.dW = nullptr; q.dw_O = nullptr; q.lora_scale = 1.0f;
+    q.Y = dX; q.ldy = lddx; q.y_f32 = 0;
+    q.dbg_main = dbg_acc_opt; q.dbg_out = nullptr;
+    GemmParams p;                                     // outlier columns: P = dY [Wd[:,O] | wd] over N, floating point
+    const int TNP = 2 * nOp > 128 ? 256 : 128;
+    if (nO > 0) {
+        memset(&p, 0, sizeof(p));
+        GemmPhase& ph = p.ph[0];
+        if ((rc = make_tmap_2d(&ph.map_a, dY, 2, M, N, lddy, kTileM, 64)) != QUAFF_OK) return rc;
+        if ((rc = make_tmap_2d(&ph.map_b, WdO, 2, N, 2 * nOp, 2 * nOp, 64, 64)) != QUAFF_OK) return rc;
+        fill_phase(ph, 0, N, 0, 1, 1 << 30, TNP, CTAS, 0, 1, 64, TNP);
+        p.nphases = 1;
+        p.M = M; p.N = 2 * nOp;
+        p.n_split = 0; p.p_col0 = 0;                  // every column is an outlier partial product
+        p.tiles_m = ceil_div(M, kTileM * CTAS); p.tiles_n = ceil_div(p.N, TNP);
+        p.band_m = p.tiles_m;
+        p.status = status_opt;
+        p.dX = nullptr; p.lddx = 0; p.P = P; p.ldp = 2 * nOp;
+        p.tile_n = TNP;
+    }
+    if (want_dAB) {
+        if ((rc = skinny_prepare(gemm_db, 1, dY, lddy, T, r, N, M, r, part_b, status_opt)) != QUAFF_OK) return rc;
+        if ((rc = skinny_prepare(gemm_da, 1, X, ldx, G, r, K, M, r, part_a, status_opt)) != QUAFF_OK) return rc;
+    }
+
+    DeviceSide* ds = device_side();
+    std::unique_lock<std::mutex> lock;
+    SideSet* ss = nullptr;
+    if (ds) {
+        lock = std::unique_lock<std::mutex>(ds->mu);
+        ss = pick_side_set(ds, st);
+    }
+    bool forked0 = false, forked1 = false;
+    auto leave = [&](quaff_status_t code) {
+        if (forked0 && !join_from(ss, 0, st) && code == QUAFF_OK) code = QUAFF_ERR_CUDA;
+        if (forked1 && !join_from(ss, 1, st) && code == QUAFF_OK) code = QUAFF_ERR_CUDA;
+        return code;
+    };
+    // side stream 0: the gradient quantization (beside G); later dA.  side stream 1: dB, enqueued behind the GEMMs.
+    if (ss && want_dAB && !(forked1 = fork_to(ss, 1, st))) return leave(QUAFF_ERR_CUDA);
+    if (ss && !(forked0 = fork_to(ss, 0, st))) return leave(QUAFF_ERR_CUDA);
+    cudaStream_t s_q = ss ? ss->s[0] : st;
+    if (r > 0) {
+        if ((rc = skinny_launch(gemm_g, st)) != QUAFF_OK) return leave(rc);
+        launch_pdl(reduce_parts_bf16_kernel, dim3(ceil_div(M * r / 8, 256)), dim3(256), 0, st, 1, part, gemm_g.S, M, r, lora_scale, G);
+        if ((rc = launch_status()) != QUAFF_OK) return leave(rc);
+        if (ss && cudaEventRecord(ss->g_ready, st) != cudaSuccess) return leave(QUAFF_ERR_CUDA);
+    }
+    if ((rc = quant_grad_dispatch(dY, lddy, M, N, dW, Zq, N, dz, s_q)) != QUAFF_OK) return leave(rc);
+    if (nO > 0) {
+        launch_pdl(dequant_weight_kernel, dim3(N, ceil_div(2 * nOp / 16, 256)), dim3(256), 0, s_q, 1, Wq, ldwq_main, dW, wq_O, ldwq, dw_O, O_idx,
+                   nO, nOp, 0, 0, WdO, (int64_t)(2 * nOp));
+        if ((rc = launch_status()) != QUAFF_OK) return leave(rc);
+    }
+    if (forked0) {
+        forked0 = false;
+        if (!join_from(ss, 0, st)) return leave(QUAFF_ERR_CUDA);
+    }
+    if ((rc = launch_fwd_wide(1, q, st, 1)) != QUAFF_OK) return leave(rc);      // timed as the grad-input GEMM
+    if (nO > 0) {
+        rc = TNP > 128 ? launch_gemm<EPI_BWD, CTAS, 256>(p, st) : launch_gemm<EPI_BWD, CTAS, 128>(p, st);
+        if (rc != QUAFF_OK) return leave(rc);
+    }
+    if (want_dAB) {
+        if (ss && cudaStreamWaitEvent(ss->s[1], ss->join[0], 0) != cudaSuccess) return leave(QUAFF_ERR_CUDA);
+        cudaStream_t s_db = ss ? ss->s[1] : st;
+        if ((rc = skinny_launch(gemm_db, s_db)) != QUAFF_OK) return leave(rc);
+        launch_pdl(reduce_parts_kernel, dim3(ceil_div(N * r / 4, 256)), dim3(256), 0, s_db, 1, part_b, gemm_db.S, N, r, lora_scale, 1, accumulate, dB);
+        if ((rc = launch_status()) != QUAFF_OK) return leave(rc);
+        cudaStream_t s_da = st;
+        if (ss) {
+            if (cudaStreamWaitEvent(ss->s[0], ss->g_ready, 0) != cudaSuccess) return leave(QUAFF_ERR_CUDA);
+            forked0 = true;
+            s_da = ss->s[0];
+        }
+        if ((rc = skinny_launch(gemm_da, s_da)) != QUAFF_OK) return leave(rc);
+        launch_pdl(reduce_parts_kernel, dim3(ceil_div(K * r / 4, 256)), dim3(256), 0, s_da, 1, part_a, gemm_da.S, K, r, 1.0f, 0, accumulate, dA);
+        if ((rc = launch_status()) != QUAFF_OK) return leave(rc);
+    }
+    if (nO > 0) {
         launch_pdl(bwd_fixup_kernel, dim3(ceil_div(M * nO, 256)), dim3(256), 0, st, 1, P, (int64_t)(2 * nOp), M, nO, nOp, O_idx, s_O, G, A, r,
                    dX, lddx);
         if ((rc = launch_status()) != QUAFF_OK) return leave(rc);

@@ -260,6 +260,115 @@ static quaff_status_t quant_act_dispatch(const uint16_t* X, int64_t ldx, int M, 
 }
 
 // =====================================================================================
+// INT8 grad-input variant: Z = dY * Delta_W[n], per-token quantization (one pass over dY)
+// =====================================================================================
+// The same row scheme as quant_act_kernel: a small CTA owns one row at a time and keeps it in registers as packed
+// bf16 (J units of 16 columns per thread), the CTA's next row is in flight while this one is processed.  The column
+// scales are re-read per row through the read-only path (all rows share them: L1 / L2 hits).  z = x * scale is one
+// fp32 product with one rounding, evaluated twice with the same operands (absmax pass, rounding pass).
+__device__ __forceinline__ void scaled8(const uint4& a, const float4& s0, const float4& s1, float (&z)[8]) {
+    z[0] = __fmul_rn(bf16_lo(a.x), s0.x); z[1] = __fmul_rn(bf16_hi(a.x), s0.y);
+    z[2] = __fmul_rn(bf16_lo(a.y), s0.z); z[3] = __fmul_rn(bf16_hi(a.y), s0.w);
+    z[4] = __fmul_rn(bf16_lo(a.z), s1.x); z[5] = __fmul_rn(bf16_hi(a.z), s1.y);
+    z[6] = __fmul_rn(bf16_lo(a.w), s1.z); z[7] = __fmul_rn(bf16_hi(a.w), s1.w);
+}
+template <int J>
+__global__ void __launch_bounds__(256, 2) quant_grad_kernel(const uint16_t* __restrict__ dY, int64_t lddy, int M, int N,
+                                                            const float* __restrict__ colscale, int8_t* __restrict__ Zq,
+                                                            int64_t ldz, float* __restrict__ dz) {
+    pdl_launch_dependents();
+    pdl_wait();
+    __shared__ float red[2][8];
+    const int tid = threadIdx.x, T = blockDim.x;
+    const int lane = tid & 31, warp = tid >> 5, nwarps = T >> 5;
+    uint4 raw[J][2];
+    int m = blockIdx.x;
+    if (m < M) load_row<J, false>(raw, dY + (int64_t)m * lddy, tid, T, N);
+    int parity = 0;
+    for (; m < M; m += gridDim.x, parity ^= 1) {
+        uint4 nxt[J][2];
+        const int mn = m + gridDim.x;
+        if (mn < M) load_row<J, false>(nxt, dY + (int64_t)mn * lddy, tid, T, N);
+        float amax = 0.0f;
+#pragma unroll
+        for (int j = 0; j < J; ++j) {
+            const int k0 = (tid + j * T) << 4;
+            if (k0 >= N) continue;
+            const float4* sc = reinterpret_cast<const float4*>(colscale + k0);
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                float z[8];
+                scaled8(raw[j][h], __ldg(sc + 2 * h), __ldg(sc + 2 * h + 1), z);
+#pragma unroll
+                for (int e = 0; e < 8; ++e) amax = fmaxf(amax, fabsf(z[e]));
+            }
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+        if (nwarps > 1) {
+            if (lane == 0) red[parity][warp] = amax;
+            __syncthreads();
+            amax = red[parity][0];
+            for (int w = 1; w < nwarps; ++w) amax = fmaxf(amax, red[parity][w]);
+        }
+        const float rinv = amax > 0.0f ? __fdiv_rn(127.0f, amax) : 0.0f;
+        if (tid == 0) dz[m] = __fdiv_rn(amax, 127.0f);
+        int8_t* qrow = Zq + (int64_t)m * ldz;
+#pragma unroll
+        for (int j = 0; j < J; ++j) {
+            const int k0 = (tid + j * T) << 4;
+            if (k0 >= N) continue;
+            const float4* sc = reinterpret_cast<const float4*>(colscale + k0);
+            uint32_t out[4];
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                float z[8];
+                scaled8(raw[j][h], __ldg(sc + 2 * h), __ldg(sc + 2 * h + 1), z);
+                uint32_t c[8];
+#pragma unroll
+                for (int e = 0; e < 8; ++e) c[e] = code_bits(z[e], rinv);
+                out[2 * h] = __byte_perm(__byte_perm(c[0], c[1], 0x0040), __byte_perm(c[2], c[3], 0x0040), 0x5410);
+                out[2 * h + 1] = __byte_perm(__byte_perm(c[4], c[5], 0x0040), __byte_perm(c[6], c[7], 0x0040), 0x5410);
+            }
+            *reinterpret_cast<uint4*>(qrow + k0) = make_uint4(out[0], out[1], out[2], out[3]);
+        }
+#pragma unroll
+        for (int j = 0; j < J; ++j) {
+            raw[j][0] = nxt[j][0];
+            raw[j][1] = nxt[j][1];
+        }
+    }
+}
+
+template <int J>
+static quaff_status_t launch_quant_grad(int T, const uint16_t* dY, int64_t lddy, int M, int N, const float* colscale, int8_t* Zq,
+                                        int64_t ldz, float* dz, cudaStream_t st) {
+    int per_sm = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, quant_grad_kernel<J>, T, 0) != cudaSuccess || per_sm < 1) per_sm = 1;
+    const int grid = min(M, sm_count() * per_sm);
+    launch_pdl(quant_grad_kernel<J>, dim3(grid), dim3(T), 0, st, 1, dY, lddy, M, N, colscale, Zq, ldz, dz);
+    return launch_status();
+}
+
+quaff_status_t quant_grad_dispatch(const uint16_t* dY, int64_t lddy, int M, int N, const float* colscale, int8_t* Zq, int64_t ldz,
+                                   float* dz, cudaStream_t st) {
+    const int nunits = N / 16;
+    if ((N % 16) || nunits > 8 * 256) return QUAFF_ERR_UNSUPPORTED_SHAPE;
+    // units per thread: small CTAs (128 threads or fewer) up to 4 units; rows beyond 8192 columns take 256 threads
+    // rather than 8 units (the row and the prefetched next row would no longer fit the registers)
+    int J = 1;
+    while (J < 4 && ceil_div(nunits, J) > kQuantActMaxThreads) J *= 2;
+    if (ceil_div(nunits, J) > 256) J = 8;
+    const int T = min(256, ceil_div(ceil_div(nunits, J), 32) * 32);
+    switch (J) {
+        case 1: return launch_quant_grad<1>(T, dY, lddy, M, N, colscale, Zq, ldz, dz, st);
+        case 2: return launch_quant_grad<2>(T, dY, lddy, M, N, colscale, Zq, ldz, dz, st);
+        case 4: return launch_quant_grad<4>(T, dY, lddy, M, N, colscale, Zq, ldz, dz, st);
+        default: return launch_quant_grad<8>(T, dY, lddy, M, N, colscale, Zq, ldz, dz, st);
+    }
+}
+
+// =====================================================================================
 // Momentum scale update (Eq. 8 then Eq. 7), only over the channels of O
 // =====================================================================================
 // Column maxima of |X| over the nO outlier columns: each block scans a slice of rows (lane =
@@ -549,4 +658,13 @@ extern "C" quaff_status_t quaff_momentum_update_static(const quaff_bf16* X, int6
     launch_pdl(momentum_kernel, dim3(momentum_grid(M)), dim3(256), 0, st, 1, X, ldx, M, O_idx, nO, wmax_O, gamma, s_O, colmax_O_opt,
                beta_O_opt, scratch, (const float*)nullptr, 1);
     return launch_status();
+}
+
+extern "C" quaff_status_t quaff_quant_grad(const quaff_bf16* dY, int64_t lddy, int M, int N, const float* dW, int8_t* Zq,
+                                           int64_t ldz, float* dz, quaff_stream_t stream) {
+    QUAFF_RETURN_IF(!dY || !dW || !Zq || !dz || M < 0 || N <= 0 || lddy < N || ldz < N, QUAFF_ERR_INVALID_ARG);
+    QUAFF_RETURN_IF(N % 16, QUAFF_ERR_UNSUPPORTED_SHAPE);
+    QUAFF_RETURN_IF(!aligned16(dY) || !aligned16(Zq) || !aligned16(dW) || (lddy % 8) || (ldz % 16), QUAFF_ERR_ALIGNMENT);
+    if (M == 0) return QUAFF_OK;
+    return quant_grad_dispatch(dY, lddy, M, N, dW, Zq, ldz, dz, (cudaStream_t)stream);
 }

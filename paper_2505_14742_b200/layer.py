@@ -24,7 +24,8 @@ class QuaffLinear:
 
     def __init__(self, Wt: torch.Tensor, O_idx: Optional[torch.Tensor], A: Optional[torch.Tensor],
                  B: Optional[torch.Tensor], lora_scale: float, gamma: float, max_tokens: int,
-                 y_dtype: torch.dtype = torch.bfloat16, debug_acc: bool = False, keep_G: bool = False):
+                 y_dtype: torch.dtype = torch.bfloat16, debug_acc: bool = False, keep_G: bool = False,
+                 int8_grad: bool = False):
         dev = Wt.device
         self.N, self.K = Wt.shape
         self.nO = 0 if O_idx is None else int(O_idx.numel())
@@ -59,9 +60,11 @@ class QuaffLinear:
         # G = bf16(lora_scale dY B^T) of the last backward, kept on request (otherwise it lives in the workspace)
         self.G = torch.empty((M, r), dtype=bf, device=dev) if (keep_G and r) else None
         self.status = torch.zeros(4, dtype=torch.int32, device=dev)
+        # int8_grad: the backward runs the INT8 grad-input variant (quaff_qlinear_bwd_int8) - not the paper's method
+        self.int8_grad = bool(int8_grad)
         ws_bytes = max(Q.workspace_bytes(Q.QUAFF_WS_MOMENTUM, M, K, N, nOp, r),
                        Q.workspace_bytes(Q.QUAFF_WS_FWD, M, K, N, nOp, r),
-                       Q.workspace_bytes(Q.QUAFF_WS_BWD, M, K, N, nOp, r), 256)
+                       Q.workspace_bytes(Q.QUAFF_WS_BWD_INT8 if int8_grad else Q.QUAFF_WS_BWD, M, K, N, nOp, r), 256)
         self.ws = torch.empty(ws_bytes, dtype=torch.uint8, device=dev)
         # the LoRA down-projection runs beside the quantization chain, on its own stream and workspace
         self.ws_lora = torch.empty(max(Q.workspace_bytes(Q.QUAFF_WS_FWD, M, K, N, nOp, r), 256), dtype=torch.uint8, device=dev) if r else None
@@ -102,9 +105,13 @@ class QuaffLinear:
         M = dY.shape[0]
         dX = self.dX[:M] if need_dX else None
         T = self.T[:M] if self.r else None
+        G = self.G[:M] if self.G is not None else None
+        if self.int8_grad:
+            Q.quaff_qlinear_bwd_int8(dY, self.Wq, self.dW, self.wq_O, self.dw_O, self.O_idx, self.s_O, self._X, T, self.A, self.B,
+                                     self.lora_scale, self.dX[:M], self.dA, self.dB, accumulate, self.ws, self.status, G)
+            return self.dX[:M], self.dA, self.dB
         Q.quaff_qlinear_bwd(dY, self.Wq, self.dW, self.wq_O, self.dw_O, self.O_idx, self.s_O, self._X, T, self.A, self.B,
-                            self.lora_scale, dX, self.dA, self.dB, accumulate, self.ws, self.status,
-                            self.G[:M] if self.G is not None else None)
+                            self.lora_scale, dX, self.dA, self.dB, accumulate, self.ws, self.status, G)
         return dX, self.dA, self.dB
 
 

@@ -16,7 +16,7 @@ from util import TOL_BF16, check_bf16_intermediate, dev, dev_bf16, dx_floor, hos
 pytestmark = pytest.mark.gpu
 
 
-def _run_layer(wl, li, steps, nsample, check_acc, full_grads=True):
+def _run_layer(wl, li, steps, nsample, check_acc, full_grads=True, int8_grad=False):
     import torch
     from paper_2505_14742_b200 import build
     from paper_2505_14742_b200.layer import QuaffLinear, StepGraph
@@ -27,7 +27,8 @@ def _run_layer(wl, li, steps, nsample, check_acc, full_grads=True):
     scale = wl.lora_alpha / r
     nOp = synth.pad_to(sp.nO, 32)
     # keep_G: the backward writes G into a buffer of the layer instead of its workspace (same kernels, same launches)
-    layer = QuaffLinear(dev_bf16(lin.W), dev(lin.O_idx), dev_bf16(lin.A), dev_bf16(lin.B), scale, wl.gamma, M, keep_G=True)
+    layer = QuaffLinear(dev_bf16(lin.W), dev(lin.O_idx), dev_bf16(lin.A), dev_bf16(lin.B), scale, wl.gamma, M, keep_G=True,
+                        int8_grad=int8_grad)
     Xd = torch.empty((M, K), dtype=torch.bfloat16, device="cuda")
     dYd = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
 
@@ -72,7 +73,10 @@ def _run_layer(wl, li, steps, nsample, check_acc, full_grads=True):
         assert err <= TOL_BF16, f"Y rows, step {step}: {err:.3e}"
         oGs = oracle.qlinear_bwd(dYs, Wq, dW, wq, dw, lin.O_idx, s, Xs, Tg[rows], lin.A, lin.B, scale, want_dX=False, want_dAB=False)[3]
         check_bf16_intermediate(Gg[rows], oGs, f"G rows, step {step}")
-        odX = oracle.qlinear_bwd(dYs, Wq, dW, wq, dw, lin.O_idx, s, Xs, Tg[rows], lin.A, lin.B, scale, want_dAB=False, G_in=Gg[rows])[0]
+        if int8_grad:    # the INT8 grad-input variant against its own oracle function
+            odX = oracle.qlinear_bwd_int8(dYs, Wq, dW, wq, dw, lin.O_idx, s, Xs, Tg[rows], lin.A, lin.B, scale, want_dAB=False, G_in=Gg[rows])[0]
+        else:
+            odX = oracle.qlinear_bwd(dYs, Wq, dW, wq, dw, lin.O_idx, s, Xs, Tg[rows], lin.A, lin.B, scale, want_dAB=False, G_in=Gg[rows])[0]
         err = max_rel_err(host(layer.dX)[rows], odX, dx_floor(N))
         assert err <= TOL_BF16, f"dX rows, step {step}: {err:.3e}"
         # LoRA gradients contract over all tokens
@@ -117,6 +121,12 @@ def test_phi3_attn_o_proj_full_size():
 @pytest.mark.parametrize("li", [0, 4, 6], ids=["q_proj", "gate_proj", "down_proj"])
 def test_llama7b_block_layers_full_size(li):
     _run_layer(synth.WORKLOADS["llama7b_block"], li, steps=1, nsample=24, check_acc=True, full_grads=False)
+
+
+# The INT8 grad-input variant (not the paper's method) at full size, against its own oracle function
+@pytest.mark.parametrize("wl_name,li", [("llama7b_block", 4), ("phi3_attn", 0)], ids=["llama_gate_proj", "phi3_qkv"])
+def test_int8_grad_variant_full_size(wl_name, li):
+    _run_layer(synth.WORKLOADS[wl_name], li, steps=1, nsample=24, check_acc=False, full_grads=False, int8_grad=True)
 
 
 # Phi-3 MLP, 4096 tokens: fused gate_up 3072 -> 16384 and down 8192 -> 3072, one forward + backward step each

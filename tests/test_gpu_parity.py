@@ -440,3 +440,69 @@ def test_backward_from_two_host_threads_is_bit_identical_to_serial(Q):
         assert host(cases[i]["st"])[0] == 0
         for got, ref in zip(outs[i]["res"], serial[i]):
             assert np.array_equal(host(got), ref)
+
+
+# ----------------------------------------------------------------------------- INT8 grad-input variant (not the paper's method)
+@pytest.mark.parametrize("M,N", [(1, 16), (37, 144), (300, 3072), (64, 11008), (19, 16384), (5, 20000)])
+def test_quant_grad_bit_exact(Q, M, N):
+    import torch
+    rng = np.random.default_rng(700 + M)
+    dY = bf(rng.standard_normal((M, N)).astype(np.float32) * 1e-2)
+    if M > 3:
+        dY[2] = 0
+    dW = (rng.random(N).astype(np.float32) + 0.01) * 1e-3
+    ld = N + 16
+    Zq = torch.full((M, ld), -128, dtype=torch.int8, device="cuda")
+    dz = torch.full((M,), -1.0, dtype=torch.float32, device="cuda")
+    Q.quaff_quant_grad(dev_bf16(dY), dev(dW), Zq[:, :N], dz)
+    torch.cuda.synchronize()
+    oZq, odz = oracle.quant_grad(dY, dW)
+    assert np.array_equal(host(Zq[:, :N]), oZq)
+    assert (host(Zq[:, N:]) == -128).all(), "wrote outside the row"
+    assert np.array_equal(host(dz), odz)
+
+
+BWD8_SHAPES = [(1, 128, 64, 0, 0), (128, 128, 128, 32, 16), (200, 320, 144, 5, 8), (256, 512, 512, 8, 8),
+               (384, 640, 1024, 40, 16), (130, 304, 2048, 33, 64), (100, 256, 256, 3, 0), (520, 1032, 3072, 32, 16),
+               (300, 2056, 528, 70, 32), (200, 11008, 528, 1100, 16), (2048, 1000, 1536, 20, 64)]
+
+
+@pytest.mark.parametrize("M,K,N,nO,r", BWD8_SHAPES)
+def test_qlinear_bwd_int8(Q, M, K, N, nO, r):
+    """quaff_qlinear_bwd_int8 against its own oracle function: INT32 accumulators bit for bit, G within one ulp, dX, dA,
+    dB against the oracle evaluated on the GPU's G bits."""
+    import torch
+    K = (K + 7) // 8 * 8
+    O, X, Wt, A, B, dY = _mk_inputs(800 + M + N, M, K, N, nO, r)
+    Wq, dW, W_O, wmax, s, Xq, xqo, dx, wq, dw = _oracle_state(O, X, Wt)
+    nOp = _pad32(nO)
+    oT = oracle.lora_down(X, A) if r else None
+    dXbuf = torch.full((M + 2, K + 8), -777.0, dtype=torch.bfloat16, device="cuda")
+    dX = dXbuf[:M, :K]
+    dA = torch.full((K, r), 1.0, dtype=torch.float32, device="cuda") if r else None
+    dB = torch.full((r, N), 1.0, dtype=torch.float32, device="cuda") if r else None
+    Gd = torch.full((M, r), float("nan"), dtype=torch.bfloat16, device="cuda") if r else None
+    acc = torch.full((M, K), -7, dtype=torch.int32, device="cuda")
+    st = torch.zeros(4, dtype=torch.int32, device="cuda")
+    ws = torch.empty(Q.workspace_bytes(Q.QUAFF_WS_BWD_INT8, M, K, N, nOp, r), dtype=torch.uint8, device="cuda")
+    Wq_d = torch.zeros((N, (K + 15) // 16 * 16), dtype=torch.int8, device="cuda")
+    Wq_d[:, :K] = dev(Wq)
+    Q.quaff_qlinear_bwd_int8(dev_bf16(dY), Wq_d[:, :K], dev(dW), dev(wq) if nOp else None, dev(dw), dev(O) if nO else None,
+                             dev(s) if nO else None, dev_bf16(X), dev_bf16(oT) if r else None, dev_bf16(A) if r else None,
+                             dev_bf16(B) if r else None, 0.5, dX, dA, dB, False, ws, st, Gd, acc)
+    torch.cuda.synchronize()
+    assert host(st)[0] == 0
+    Gg = host_bits(Gd) if r else None
+    odX, odA, odB, oG, oZq, odz, oacc = oracle.qlinear_bwd_int8(dY, Wq, dW, wq, dw, O, s, X, oT, A, B, 0.5, G_in=Gg)
+    assert np.array_equal(host(acc), oacc), "INT32 accumulator of the grad-input"
+    if r:
+        check_bf16_intermediate(Gg, oracle.qlinear_bwd(dY, Wq, dW, wq, dw, O, s, X, oT, A, B, 0.5, want_dX=False, want_dAB=False)[3], "G")
+    err = max_rel_err(host(dX), odX)
+    assert err <= TOL_BF16, f"dX max rel err {err:.3e}"
+    assert bool((dXbuf[M:, :] == -777.0).all()) and bool((dXbuf[:, K:] == -777.0).all()), "write outside dX"
+    if nO:
+        err_o = max_rel_err(host(dX)[:, O], odX[:, O], dx_floor(N))
+        assert err_o <= TOL_BF16, f"dX outlier columns max rel err {err_o:.3e}"
+    if r:
+        err_a, err_b = max_rel_err(host(dA), odA), max_rel_err(host(dB), odB)
+        assert err_a <= TOL_BF16 and err_b <= TOL_BF16, f"dA {err_a:.3e} dB {err_b:.3e}"
