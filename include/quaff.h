@@ -63,7 +63,8 @@ enum { /* `which` of quaff_workspace_bytes */
     QUAFF_WS_BWD = 3,
     QUAFF_WS_CALIBRATE = 4,  /* quaff_outlier_count and quaff_select_outliers (depends on K only) */
     QUAFF_WS_HITS = 5,       /* quaff_outlier_hits (depends on K only) */
-    QUAFF_WS_BWD_INT8 = 6    /* quaff_qlinear_bwd_int8 */
+    QUAFF_WS_BWD_INT8 = 6,   /* quaff_qlinear_bwd_int8 */
+    QUAFF_WS_BWD_LEAN = 7    /* quaff_qlinear_bwd without a transient bf16 copy of the weight (see there) */
 };
 
 const char* quaff_status_string(quaff_status_t s);
@@ -230,7 +231,14 @@ quaff_status_t quaff_qlinear_fwd(int M, int K, int N,
  *   dY [M][N] bf16, lddy (lddy % 8 == 0);  T [M][r] bf16 from the forward
  *   Wq, wq_O: 16-byte aligned, ldwq_main and ldwq multiples of 16 (as in the forward)
  *   G_out_opt [M][r] bf16 (dense, 16-byte aligned), optional: receives G (otherwise G lives in the workspace only)
- *   ws: QUAFF_WS_BWD bytes;  status_opt as in the forward.
+ *   dW, dw_O: 16-byte aligned;  with an outlier set, K <= 32768
+ *   status_opt as in the forward.
+ *   ws: QUAFF_WS_BWD bytes, or QUAFF_WS_BWD_LEAN bytes.  With QUAFF_WS_BWD bytes (2 N K bytes more) the call builds a
+ *   transient bf16 copy Wd of the weight in the workspace and the grad-input GEMM reads it by TMA: the faster way (the
+ *   copy lives only inside the call; nothing full-precision is kept between steps, Sec. 3.1).  With QUAFF_WS_BWD_LEAN
+ *   bytes no copy is made at all: the GEMM reads the codes Wq and wq_O in place and expands them to bf16 in shared
+ *   memory (about 1.4 times the GEMM time, bound by shared-memory bandwidth).  The products and their order are the same:
+ *   dX is bit-identical between the two off the outlier columns.
  * Independent parts of the backward are forked onto two library-owned side streams (lowest priority) and
  * joined back into `stream` before the call returns: for the caller everything is still ordered on
  * `stream`.  The weight dequantization runs beside G in front of the grad-input GEMM; dA and dB are enqueued behind the

@@ -22,7 +22,7 @@ QUAFF_ERR_WORKSPACE_TOO_SMALL = 4
 QUAFF_ERR_CUDA = 5
 QUAFF_ERR_TIMEOUT = 6
 QUAFF_BF16, QUAFF_F32 = 0, 1
-QUAFF_WS_PREPARE, QUAFF_WS_MOMENTUM, QUAFF_WS_FWD, QUAFF_WS_BWD, QUAFF_WS_CALIBRATE, QUAFF_WS_HITS, QUAFF_WS_BWD_INT8 = 0, 1, 2, 3, 4, 5, 6
+QUAFF_WS_PREPARE, QUAFF_WS_MOMENTUM, QUAFF_WS_FWD, QUAFF_WS_BWD, QUAFF_WS_CALIBRATE, QUAFF_WS_HITS, QUAFF_WS_BWD_INT8, QUAFF_WS_BWD_LEAN = 0, 1, 2, 3, 4, 5, 6, 7
 
 EXPORTS = ("quaff_status_string", "quaff_workspace_bytes", "quaff_debug_launch_count", "quaff_debug_force_fwd_tile", "quaff_debug_time_gemm", "quaff_prepare_weight", "quaff_momentum_update", "quaff_lora_down", "quaff_outlier_count", "quaff_select_outliers", "quaff_outlier_hits",
            "quaff_momentum_update_static", "quaff_outlier_colmax", "quaff_momentum_apply", "quaff_quant_act", "quaff_requant_weight_rows", "quaff_qlinear_fwd", "quaff_qlinear_bwd", "quaff_quant_grad", "quaff_qlinear_bwd_int8")

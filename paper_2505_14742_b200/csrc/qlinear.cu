@@ -7,6 +7,7 @@
 #include <atomic>
 #include <mutex>
 
+#include "bwd_expand.cuh"
 #include "fwd256.cuh"
 
 namespace quaff {
@@ -230,6 +231,60 @@ static quaff_status_t launch_fwd_wide(int which, const FwdWideParams& p, cudaStr
     return rc;
 }
 
+// The grad-input GEMM with in-kernel expansion of the INT8 weight (bwd_expand.cuh)
+static size_t bx_fixed_bytes(int mask_words) {     // alignment slack, B ring, barriers, outlier mask
+    return 1024 + (size_t)kBxBSlots * kBxBBytes + kBxBarrierBytes + round_up((size_t)2 * mask_words * 4, 16);
+}
+static size_t bx_smem_bytes(int nstages, int mask_words) {     // ... plus the IN ring with its row-scale ring
+    return bx_fixed_bytes(mask_words) + (size_t)nstages * (kBxInBytes + 256);
+}
+static int bx_stages(int mask_words) {
+    const int fit = (int)((kSmemLimit - bx_fixed_bytes(mask_words)) / (kBxInBytes + 256));
+    return max(2, min(fit, kMaxStages));
+}
+static quaff_status_t launch_bwd_expand(const BxParams& p, cudaStream_t st) {
+    static std::atomic<bool> configured[64];
+    static std::atomic<int> units_of[64];
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (dev < 0 || dev >= 64) return QUAFF_ERR_CUDA;
+    if (!configured[dev].load()) {
+        if (cudaFuncSetAttribute(bwd_expand_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit) != cudaSuccess) return QUAFF_ERR_CUDA;
+        int units = sm_count() / 2;
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(units * 2);
+        cfg.blockDim = dim3(kBxThreads);
+        cfg.dynamicSmemBytes = kSmemLimit;
+        cudaLaunchAttribute attr;
+        attr.id = cudaLaunchAttributeClusterDimension;
+        attr.val.clusterDim.x = 2; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
+        cfg.attrs = &attr;
+        cfg.numAttrs = 1;
+        int nclusters = 0;
+        if (cudaOccupancyMaxActiveClusters(&nclusters, bwd_expand_kernel, &cfg) == cudaSuccess && nclusters > 0) units = min(units, nclusters);
+        else cudaGetLastError();
+        units_of[dev].store(max(units, 1));
+        configured[dev].store(true);
+    }
+    const int ntiles = p.tiles_m * (p.tiles_main + p.tiles_p);
+    if (ntiles == 0) return QUAFF_OK;
+    const int units = min(ntiles, units_of[dev].load());
+    const bool timed = g_time_start[1] && g_time_stop[1];
+    unsigned int ev_flags = cudaEventRecordDefault;
+    if (timed) {
+        cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+        if (cudaStreamIsCapturing(st, &cap) == cudaSuccess && cap == cudaStreamCaptureStatusActive) ev_flags = cudaEventRecordExternal;
+        cudaEventRecordWithFlags(g_time_start[1], st, ev_flags);
+    }
+    launch_pdl(bwd_expand_kernel, dim3(units * 2), dim3(kBxThreads), bx_smem_bytes(p.nstages, p.mask_words), st, 2, p);
+    const quaff_status_t rc = launch_status();
+    if (timed) {
+        cudaEventRecordWithFlags(g_time_stop[1], st, ev_flags);
+        g_time_start[1] = g_time_stop[1] = nullptr;
+    }
+    return rc;
+}
+
 // ------------------------------------------------------------------ small kernels
 // dst[c][j] = src[j][c] for j < rows, 0 for rows <= j < rows_pad   (src is [rows][cols], dst is [cols][rows_pad])
 __global__ void transpose_pad_kernel(const uint16_t* __restrict__ src, int rows, int cols, uint16_t* __restrict__ dst, int rows_pad) {
@@ -342,19 +397,20 @@ __global__ void __launch_bounds__(256) dequant_weight_kernel(const int8_t* __res
     out[1] = make_uint4(pack_bf16x2(v[8], v[9]), pack_bf16x2(v[10], v[11]), pack_bf16x2(v[12], v[13]), pack_bf16x2(v[14], v[15]));
 }
 
-// dX[m][O_i] = bf16((P[m][i] + P[m][nOp+i]) / s_i + sum_j G[m][j] A[O_i][j]);  r is a multiple of 8:
-// the rows of G and A are read as 128-bit words of 8 bf16
+// Outlier columns of the grad-input (Eq. 5: Xhat = X s^-1, so dX[:, O_i] = dXhat[:, O_i] / s_i), tolerance class (plain fp32):
+//   dX[m][O_i] = bf16(((P1 - l) + P2) / s_i + l),   l = sum_j G[m][j] A[O_i][j]
+// with P2 = P[m][nOp + i] = (dY wd)[m][i] and P1 = P[m][i] = (dY Wd)[m][O_i] + (lora_in_p1 ? the tensor cores' G A^T : 0).
+// r is a multiple of 8: the rows of G and A are read as 128-bit words of 8 bf16
 __global__ void bwd_fixup_kernel(const float* __restrict__ P, int64_t ldp, int M, int nO, int nOp,
                                  const int32_t* __restrict__ O_idx, const float* __restrict__ s_O,
                                  const uint16_t* __restrict__ G, const uint16_t* __restrict__ A, int r,
-                                 uint16_t* __restrict__ dX, int64_t lddx) {
+                                 uint16_t* __restrict__ dX, int64_t lddx, int lora_in_p1) {
     pdl_launch_dependents();
     pdl_wait();
     const int idx = blockIdx.x * blockDim.x + threadIdx.x;
     if (idx >= M * nO) return;
     const int m = idx / nO, i = idx % nO;
     const int k = O_idx[i];
-    const float v = (P[(int64_t)m * ldp + i] + P[(int64_t)m * ldp + nOp + i]) / s_O[i];
     float l = 0.0f;
     const uint4* g = reinterpret_cast<const uint4*>(G + (int64_t)m * r);
     const uint4* a = reinterpret_cast<const uint4*>(A + (int64_t)k * r);
@@ -367,6 +423,8 @@ __global__ void bwd_fixup_kernel(const float* __restrict__ P, int64_t ldp, int M
             l = fmaf(bf16_hi(gw[e]), bf16_hi(aw[e]), l);
         }
     }
+    const float p1 = P[(int64_t)m * ldp + i] - (lora_in_p1 ? l : 0.0f);
+    const float v = (p1 + P[(int64_t)m * ldp + nOp + i]) / s_O[i];
     dX[(int64_t)m * lddx + k] = (uint16_t)f32_to_bf16_bits(v + l);
 }
 
@@ -479,13 +537,9 @@ static FwdWorkspace fwd_workspace(int M, int K, int N, int r) {
     return w;
 }
 
-// Output-column tile of the grad-input GEMM: 128, 192 or 256.  A tcgen05.mma of a CTA pair costs about 60 + N/2
-// clocks (measured: N = 128: 125, 192: 165, 256: 190), so wide tiles are cheaper per column, while the width also
-// decides how full the last wave is.  Cost model: waves on the CTA pairs x cost of one MMA of that width; among equals
-// the wider tile (fewer tiles, fewer epilogues).  (Widths that are not a multiple of 64 run far below this model -
-// measured: 176 columns 208 clocks per MMA, 240 columns 215 - so they are not candidates.)
+// ---- grad-input through a dequantized copy of the weight in the workspace (the faster of the two ways; see quaff.h)
 static int round_up32(int k) { return (k + 31) / 32 * 32; }
-static int bwd_tile_n(int M, int K, int nOp) {
+static int bwd_tile_n_wd(int M, int K, int nOp) {
     const int units = kPlanSMs / 2;
     const int tm = ceil_div(M, 2 * kTileM);
     const int kext = nOp > 0 ? round_up32(K) + 2 * nOp : K;
@@ -499,20 +553,60 @@ static int bwd_tile_n(int M, int K, int nOp) {
     return best;
 }
 
-struct BwdWorkspace {
+struct BwdWdWorkspace {
     size_t off_wd, off_g, off_p, off_part, off_part_a, off_part_b, total;
     int tile_n;       // output-column tile of the grad-input GEMM
     int Kpad;         // K rounded up to 32: where the outlier columns start
     int64_t ldwd;     // row pitch of Wd in elements
 };
 
-static BwdWorkspace bwd_workspace(int M, int K, int N, int nOp, int r) {
-    BwdWorkspace w;
-    w.tile_n = bwd_tile_n(M, K, nOp);
+static BwdWdWorkspace bwd_wd_workspace(int M, int K, int N, int nOp, int r) {
+    BwdWdWorkspace w;
+    w.tile_n = bwd_tile_n_wd(M, K, nOp);
     w.Kpad = round_up32(K);
     w.ldwd = (int64_t)w.Kpad + 2 * nOp;
     size_t off = 0;
     w.off_wd = off;   off += round_up((size_t)N * (size_t)w.ldwd * 2, 256);
+    w.off_g = off;    off += round_up((size_t)M * (size_t)max(r, 1) * 2, 256);
+    w.off_p = off;    off += round_up((size_t)M * (size_t)max(2 * nOp, 1) * 4, 256);
+    // split-K partials: one buffer per skinny GEMM (they run concurrently)
+    w.off_part = off;   off += round_up(split_part_bytes(M, N, r), 256);   // G = dY B^T
+    w.off_part_a = off; off += round_up(split_part_bytes(K, M, r), 256);   // dA = X^T G
+    w.off_part_b = off; off += round_up(split_part_bytes(N, M, r), 256);   // dB^T = dY^T T
+    w.total = off;
+    return w;
+}
+
+
+// ---- grad-input with the codes expanded inside the kernel (no copy of the weight)
+// Output-column tile of the grad-input GEMM: 128, 192 or 256.  A tcgen05.mma of a CTA pair costs about 60 + N/2
+// clocks (measured: N = 128: 125, 192: 165, 256: 190), so wide tiles are cheaper per column, while the width also
+// decides how full the last wave is.  Cost model: waves on the CTA pairs x cost of one MMA of that width; among equals
+// the wider tile (fewer tiles, fewer epilogues).  (Widths that are not a multiple of 64 run far below this model -
+// measured: 176 columns 208 clocks per MMA, 240 columns 215 - so they are not candidates.)
+static int bwd_tile_n(int M, int K, int nOp) {
+    const int units = kPlanSMs / 2;
+    const int tm = ceil_div(M, 2 * kTileM);
+    int best = 256;
+    double best_cost = 0.0;
+    for (int tn = 256; tn >= 128; tn -= 64) {
+        const int tiles = tm * (ceil_div(K, tn) + (nOp > 0 ? ceil_div(nOp, tn) : 0));      // main tiles + the tiles over the outlier rows
+        const double cost = (double)ceil_div(tiles, units) * (60.0 + 0.5 * tn);
+        if (tn == 256 || cost < best_cost) { best = tn; best_cost = cost; }
+    }
+    return best;
+}
+
+struct BwdLeanWorkspace {
+    size_t off_g, off_p, off_part, off_part_a, off_part_b, total;
+    int tile_n;       // output-column tile of the grad-input GEMM
+};
+
+static BwdLeanWorkspace bwd_lean_workspace(int M, int K, int N, int nOp, int r) {
+    BwdLeanWorkspace w;
+    w.tile_n = bwd_tile_n(M, K, nOp);
+    size_t off = 0;
+    // (no dequantized weight data: the grad-input GEMM expands the codes inside the kernel)
     w.off_g = off;    off += round_up((size_t)M * (size_t)max(r, 1) * 2, 256);
     w.off_p = off;    off += round_up((size_t)M * (size_t)max(2 * nOp, 1) * 4, 256);
     // split-K partials: one buffer per skinny GEMM (they run concurrently)
@@ -602,7 +696,8 @@ extern "C" size_t quaff_workspace_bytes(int which, int M, int K, int N, int nOp,
         case QUAFF_WS_PREPARE: return 0;
         case QUAFF_WS_MOMENTUM: return round_up((size_t)(nOp + 1) * 4, 256);
         case QUAFF_WS_FWD: return fwd_workspace(M, K, N, r).total;
-        case QUAFF_WS_BWD: return bwd_workspace(M, K, N, nOp, r).total;
+        case QUAFF_WS_BWD: return max(bwd_wd_workspace(M, K, N, nOp, r).total, bwd_lean_workspace(M, K, N, nOp, r).total);
+        case QUAFF_WS_BWD_LEAN: return bwd_lean_workspace(M, K, N, nOp, r).total;
         case QUAFF_WS_BWD_INT8: return bwd_int8_workspace(M, K, N, nOp, r).total;
         case QUAFF_WS_CALIBRATE: return round_up((size_t)max(K, 0) * 4, 256) + 256;   // column maxima / flags, sum, ticket
         case QUAFF_WS_HITS: return 2 * round_up((size_t)max(K, 0) * 4, 256) + 256;    // the same, then this batch's indicator
@@ -734,32 +829,15 @@ extern "C" quaff_status_t quaff_qlinear_fwd(int M, int K, int N, const int8_t* X
     return TN == 256 ? launch_gemm<EPI_FWD, CTAS, 256>(p, st) : launch_gemm<EPI_FWD, CTAS, 128>(p, st);
 }
 
-extern "C" quaff_status_t quaff_qlinear_bwd(int M, int K, int N, const quaff_bf16* dY, int64_t lddy, const int8_t* Wq,
-                                            int64_t ldwq_main, const float* dW, const int8_t* wq_O, int64_t ldwq,
-                                            const float* dw_O, int nOp, const int32_t* O_idx, int nO, const float* s_O,
-                                            const quaff_bf16* X, int64_t ldx, const quaff_bf16* T, const quaff_bf16* A,
-                                            const quaff_bf16* B, int r, float lora_scale, quaff_bf16* dX, int64_t lddx,
-                                            float* dA, float* dB, int accumulate, quaff_bf16* G_out_opt,
-                                            int32_t* status_opt, void* ws, size_t ws_bytes, quaff_stream_t stream) {
-    QUAFF_RETURN_IF(M < 0 || K <= 0 || N <= 0 || nOp < 0 || nO < 0 || nO > nOp || r < 0, QUAFF_ERR_INVALID_ARG);
-    QUAFF_RETURN_IF(!dY || lddy < N || !Wq || !dW || ldwq_main < K, QUAFF_ERR_INVALID_ARG);
-    QUAFF_RETURN_IF(nOp > 0 && (!wq_O || !dw_O || ldwq < nOp), QUAFF_ERR_INVALID_ARG);
-    QUAFF_RETURN_IF(nO > 0 && (!O_idx || !s_O), QUAFF_ERR_INVALID_ARG);
-    QUAFF_RETURN_IF(r > 0 && (!A || !B), QUAFF_ERR_INVALID_ARG);
-    QUAFF_RETURN_IF(r > 0 && (dA || dB) && (!dA || !dB || !X || !T || ldx < K), QUAFF_ERR_INVALID_ARG);
-    QUAFF_RETURN_IF(dX && lddx < K, QUAFF_ERR_INVALID_ARG);
-    QUAFF_RETURN_IF((nOp % 32) || (r % 8) || r > 64, QUAFF_ERR_UNSUPPORTED_SHAPE);
-    QUAFF_RETURN_IF(r > 0 && (N % 8), QUAFF_ERR_UNSUPPORTED_SHAPE);
-    QUAFF_RETURN_IF(!aligned16(dY) || (lddy % 8), QUAFF_ERR_ALIGNMENT);
-    QUAFF_RETURN_IF(!aligned16(Wq) || (ldwq_main % 16), QUAFF_ERR_ALIGNMENT);
-    QUAFF_RETURN_IF(nOp > 0 && (!aligned16(wq_O) || (ldwq % 16)), QUAFF_ERR_ALIGNMENT);
-    QUAFF_RETURN_IF(dX && (!aligned16(dX) || (lddx % 8)), QUAFF_ERR_ALIGNMENT);
-    QUAFF_RETURN_IF(r > 0 && (!aligned16(A) || !aligned16(B) || (G_out_opt && !aligned16(G_out_opt))), QUAFF_ERR_ALIGNMENT);
-    QUAFF_RETURN_IF(r > 0 && dA && (!aligned16(X) || !aligned16(T) || !aligned16(dA) || !aligned16(dB) || (ldx % 8)), QUAFF_ERR_ALIGNMENT);
-    const BwdWorkspace w = bwd_workspace(M, K, N, nOp, r);
-    QUAFF_RETURN_IF(!ws || !aligned16(ws) || ws_bytes < w.total, QUAFF_ERR_WORKSPACE_TOO_SMALL);
-    if (M == 0) return QUAFF_OK;
-    cudaStream_t st = (cudaStream_t)stream;
+// quaff_qlinear_bwd with a dequantized copy of the weight in the workspace (arguments validated by the caller)
+static quaff_status_t bwd_through_copy(int M, int K, int N, const quaff_bf16* dY, int64_t lddy, const int8_t* Wq,
+                                       int64_t ldwq_main, const float* dW, const int8_t* wq_O, int64_t ldwq,
+                                       const float* dw_O, int nOp, const int32_t* O_idx, int nO, const float* s_O,
+                                       const quaff_bf16* X, int64_t ldx, const quaff_bf16* T, const quaff_bf16* A,
+                                       const quaff_bf16* B, int r, float lora_scale, quaff_bf16* dX, int64_t lddx,
+                                       float* dA, float* dB, int accumulate, quaff_bf16* G_out_opt,
+                                       int32_t* status_opt, void* ws, cudaStream_t st) {
+    const BwdWdWorkspace w = bwd_wd_workspace(M, K, N, nOp, r);
     unsigned char* base = reinterpret_cast<unsigned char*>(ws);
     uint16_t* Wd = reinterpret_cast<uint16_t*>(base + w.off_wd);
     uint16_t* G = (r > 0 && G_out_opt) ? G_out_opt : reinterpret_cast<uint16_t*>(base + w.off_g);
@@ -881,7 +959,151 @@ extern "C" quaff_status_t quaff_qlinear_bwd(int M, int K, int N, const quaff_bf1
     }
     if (dX && nO > 0) {
         launch_pdl(bwd_fixup_kernel, dim3(ceil_div(M * nO, 256)), dim3(256), 0, st, 1, P, (int64_t)(2 * nOp), M, nO, nOp, O_idx, s_O, G, A, r,
-                   dX, lddx);
+                   dX, lddx, 0);
+        if ((rc = launch_status()) != QUAFF_OK) return leave(rc);
+    }
+    return leave(QUAFF_OK);
+}
+
+
+extern "C" quaff_status_t quaff_qlinear_bwd(int M, int K, int N, const quaff_bf16* dY, int64_t lddy, const int8_t* Wq,
+                                            int64_t ldwq_main, const float* dW, const int8_t* wq_O, int64_t ldwq,
+                                            const float* dw_O, int nOp, const int32_t* O_idx, int nO, const float* s_O,
+                                            const quaff_bf16* X, int64_t ldx, const quaff_bf16* T, const quaff_bf16* A,
+                                            const quaff_bf16* B, int r, float lora_scale, quaff_bf16* dX, int64_t lddx,
+                                            float* dA, float* dB, int accumulate, quaff_bf16* G_out_opt,
+                                            int32_t* status_opt, void* ws, size_t ws_bytes, quaff_stream_t stream) {
+    QUAFF_RETURN_IF(M < 0 || K <= 0 || N <= 0 || nOp < 0 || nO < 0 || nO > nOp || r < 0, QUAFF_ERR_INVALID_ARG);
+    QUAFF_RETURN_IF(!dY || lddy < N || !Wq || !dW || ldwq_main < K, QUAFF_ERR_INVALID_ARG);
+    QUAFF_RETURN_IF(nOp > 0 && (!wq_O || !dw_O || ldwq < nOp), QUAFF_ERR_INVALID_ARG);
+    QUAFF_RETURN_IF(nO > 0 && (!O_idx || !s_O), QUAFF_ERR_INVALID_ARG);
+    QUAFF_RETURN_IF(r > 0 && (!A || !B), QUAFF_ERR_INVALID_ARG);
+    QUAFF_RETURN_IF(r > 0 && (dA || dB) && (!dA || !dB || !X || !T || ldx < K), QUAFF_ERR_INVALID_ARG);
+    QUAFF_RETURN_IF(dX && lddx < K, QUAFF_ERR_INVALID_ARG);
+    QUAFF_RETURN_IF((nOp % 32) || (r % 8) || r > 64, QUAFF_ERR_UNSUPPORTED_SHAPE);
+    QUAFF_RETURN_IF(r > 0 && (N % 8), QUAFF_ERR_UNSUPPORTED_SHAPE);
+    QUAFF_RETURN_IF(!aligned16(dY) || (lddy % 8), QUAFF_ERR_ALIGNMENT);
+    QUAFF_RETURN_IF(!aligned16(Wq) || (ldwq_main % 16), QUAFF_ERR_ALIGNMENT);
+    QUAFF_RETURN_IF(nOp > 0 && (!aligned16(wq_O) || (ldwq % 16)), QUAFF_ERR_ALIGNMENT);
+    QUAFF_RETURN_IF(dX && (!aligned16(dX) || (lddx % 8)), QUAFF_ERR_ALIGNMENT);
+    QUAFF_RETURN_IF(r > 0 && (!aligned16(A) || !aligned16(B) || (G_out_opt && !aligned16(G_out_opt))), QUAFF_ERR_ALIGNMENT);
+    QUAFF_RETURN_IF(r > 0 && dA && (!aligned16(X) || !aligned16(T) || !aligned16(dA) || !aligned16(dB) || (ldx % 8)), QUAFF_ERR_ALIGNMENT);
+    QUAFF_RETURN_IF(nO > 0 && K > 32768, QUAFF_ERR_UNSUPPORTED_SHAPE);      // the per-column outlier mask lives in shared memory
+    QUAFF_RETURN_IF(!aligned16(dW) || (nOp > 0 && !aligned16(dw_O)), QUAFF_ERR_ALIGNMENT);
+    const BwdLeanWorkspace w = bwd_lean_workspace(M, K, N, nOp, r);
+    QUAFF_RETURN_IF(!ws || !aligned16(ws) || ws_bytes < w.total, QUAFF_ERR_WORKSPACE_TOO_SMALL);
+    if (M == 0) return QUAFF_OK;
+    cudaStream_t st = (cudaStream_t)stream;
+    // Two ways through the frozen INT8 weight, the same products in the same order either way (dX is bit-identical off the
+    // outlier columns): with room for a transient bf16 copy of the weight in the workspace (QUAFF_WS_BWD bytes) the copy is
+    // made and read by TMA, which is the faster way; with QUAFF_WS_BWD_LEAN bytes the codes are expanded inside the GEMM.
+    if (dX && ws_bytes >= bwd_wd_workspace(M, K, N, nOp, r).total)
+        return bwd_through_copy(M, K, N, dY, lddy, Wq, ldwq_main, dW, wq_O, ldwq, dw_O, nOp, O_idx, nO, s_O, X, ldx, T, A, B, r, lora_scale, dX,
+                                lddx, dA, dB, accumulate, G_out_opt, status_opt, ws, st);
+    unsigned char* base = reinterpret_cast<unsigned char*>(ws);
+    uint16_t* G = (r > 0 && G_out_opt) ? G_out_opt : reinterpret_cast<uint16_t*>(base + w.off_g);
+    float* P = reinterpret_cast<float*>(base + w.off_p);
+    float* part = reinterpret_cast<float*>(base + w.off_part);
+    float* part_a = reinterpret_cast<float*>(base + w.off_part_a);
+    float* part_b = reinterpret_cast<float*>(base + w.off_part_b);
+    quaff_status_t rc;
+    const bool want_dAB = r > 0 && dA && dB;
+    const int TN = w.tile_n;
+
+    // ---- every tensor map and launch parameter first: nothing has been enqueued when one of them fails
+    SkinnyGemm gemm_g, gemm_db, gemm_da;
+    BxParams p;
+    if (r > 0) {   // G = bf16(lora_scale * dY B^T): B [r][N] is already K-major for this contraction over N
+        if ((rc = skinny_prepare(gemm_g, 0, dY, lddy, B, N, M, N, r, part, status_opt)) != QUAFF_OK) return rc;
+    }
+    if (dX) {
+        memset(&p, 0, sizeof(p));
+        if ((rc = make_tmap_2d(&p.map_dy, dY, 2, M, N, lddy, kTileM, 64)) != QUAFF_OK) return rc;
+        // the codes in their stored orientation, the contraction index n as the row: boxes of 64 rows x 128 codes
+        if ((rc = make_tmap_2d(&p.map_wq, Wq, 1, N, K, ldwq_main, 64, 128)) != QUAFF_OK) return rc;
+        if (nO > 0) {   // the re-quantized outlier rows, likewise: wd = bf16(wq_O dw_O) is formed inside the kernel
+            if ((rc = make_tmap_2d(&p.map_wo, wq_O, 1, N, nOp, ldwq, 64, 128)) != QUAFF_OK) return rc;
+        }
+        if (r > 0) {
+            if ((rc = make_tmap_2d(&p.map_g, G, 2, M, r, r, kTileM, 64)) != QUAFF_OK) return rc;
+            if ((rc = make_tmap_2d(&p.map_a, A, 2, K, r, r, TN / 2, 64)) != QUAFF_OK) return rc;
+            p.nmma_l = pad16(r) / 16;
+        }
+        p.M = M; p.N = N; p.K = K;
+        p.nblk = ceil_div(N, 64);
+        p.nmma_last = ceil_div(N - (p.nblk - 1) * 64, 16);
+        p.tile_n = TN;
+        p.tile_np = (nO > 0 && nOp > 128) ? 256 : 128;    // each CTA supplies whole boxes of 64 columns
+        p.tiles_m = ceil_div(M, 2 * kTileM);
+        p.tiles_main = ceil_div(K, TN);
+        p.tiles_p = nO > 0 ? ceil_div(nOp, p.tile_np) : 0;
+        p.band_m = band_rows(p.tiles_m, p.tiles_main + p.tiles_p, 2 * kTileM, (size_t)N * 2);
+        p.nO = nO; p.nOp = nOp;
+        p.mask_words = nO > 0 ? ceil_div(K, 32) : 0;
+        p.nstages = bx_stages(p.mask_words);
+        p.dW = dW; p.dw_O = dw_O; p.O_idx = O_idx;
+        p.dX = dX; p.lddx = lddx; p.P = P;
+        p.status = status_opt;
+    }
+    if (want_dAB) {
+        // dB^T = dY^T T and dA = X^T G: the contraction runs over the tokens, the slow axis of all four matrices: MN-major operands
+        if ((rc = skinny_prepare(gemm_db, 1, dY, lddy, T, r, N, M, r, part_b, status_opt)) != QUAFF_OK) return rc;
+        if ((rc = skinny_prepare(gemm_da, 1, X, ldx, G, r, K, M, r, part_a, status_opt)) != QUAFF_OK) return rc;
+    }
+
+    // Dependencies:  G = dY B^T feeds the grad-input GEMM and dA = X^T G;  dB = T^T dY needs nothing computed here;
+    // the outlier fix-up follows the GEMM.
+    DeviceSide* ds = device_side();
+    std::unique_lock<std::mutex> lock;
+    SideSet* ss = nullptr;
+    if (ds) {
+        lock = std::unique_lock<std::mutex>(ds->mu);
+        ss = pick_side_set(ds, st);
+    }
+    bool forked0 = false, forked1 = false;
+    // From the first fork on, an error leaves through `leave`: whatever has been forked is joined back into the
+    // caller's stream, so that no branch stays open (a stream capture would otherwise be invalid, and a caller could
+    // reuse the workspace while a side stream still writes it).
+    auto leave = [&](quaff_status_t code) {
+        if (forked0 && !join_from(ss, 0, st) && code == QUAFF_OK) code = QUAFF_ERR_CUDA;
+        if (forked1 && !join_from(ss, 1, st) && code == QUAFF_OK) code = QUAFF_ERR_CUDA;
+        return code;
+    };
+
+    if (r > 0) {
+        if ((rc = skinny_launch(gemm_g, st)) != QUAFF_OK) return leave(rc);
+        launch_pdl(reduce_parts_bf16_kernel, dim3(ceil_div(M * r / 8, 256)), dim3(256), 0, st, 1, part, gemm_g.S, M, r, lora_scale, G);
+        if ((rc = launch_status()) != QUAFF_OK) return leave(rc);
+        if (ss && cudaEventRecord(ss->g_ready, st) != cudaSuccess) return leave(QUAFF_ERR_CUDA);
+    }
+    if (dX && (rc = launch_bwd_expand(p, st)) != QUAFF_OK) return leave(rc);
+    if (want_dAB) {
+        // dB and dA go to the side streams, behind G (dA needs it; dB needs nothing, but is held back as long, so that it does
+        // not compete with G for HBM in front of the GEMM).  Launch order = the order in which the block scheduler hands out
+        // SM slots: both are enqueued BEHIND the grad-input GEMM, which they do not depend on, so the persistent GEMM gets every
+        // SM first and the split-K CTAs of dB and dA (lowest priority) move in as the pairs that have no tile left in the last
+        // wave retire.
+        cudaStream_t s_db = st, s_da = st;
+        if (ss) {
+            if (cudaStreamWaitEvent(ss->s[1], ss->g_ready, 0) != cudaSuccess) return leave(QUAFF_ERR_CUDA);
+            forked1 = true;
+            s_db = ss->s[1];
+        }
+        if ((rc = skinny_launch(gemm_db, s_db)) != QUAFF_OK) return leave(rc);
+        launch_pdl(reduce_parts_kernel, dim3(ceil_div(N * r / 4, 256)), dim3(256), 0, s_db, 1, part_b, gemm_db.S, N, r, lora_scale, 1, accumulate, dB);
+        if ((rc = launch_status()) != QUAFF_OK) return leave(rc);
+        if (ss) {
+            if (cudaStreamWaitEvent(ss->s[0], ss->g_ready, 0) != cudaSuccess) return leave(QUAFF_ERR_CUDA);
+            forked0 = true;
+            s_da = ss->s[0];
+        }
+        if ((rc = skinny_launch(gemm_da, s_da)) != QUAFF_OK) return leave(rc);
+        launch_pdl(reduce_parts_kernel, dim3(ceil_div(K * r / 4, 256)), dim3(256), 0, s_da, 1, part_a, gemm_da.S, K, r, 1.0f, 0, accumulate, dA);
+        if ((rc = launch_status()) != QUAFF_OK) return leave(rc);
+    }
+    if (dX && nO > 0) {
+        launch_pdl(bwd_fixup_kernel, dim3(ceil_div(M * nO, 256)), dim3(256), 0, st, 1, P, (int64_t)(2 * nOp), M, nO, nOp, O_idx, s_O, G, A, r,
+                   dX, lddx, 1);     // P1 was copied out of the accumulator: it contains G A^T
         if ((rc = launch_status()) != QUAFF_OK) return leave(rc);
     }
     return leave(QUAFF_OK);
@@ -1030,7 +1252,7 @@ extern "C" quaff_status_t quaff_qlinear_bwd_int8(int M, int K, int N, const quaf
     }
     if (nO > 0) {
         launch_pdl(bwd_fixup_kernel, dim3(ceil_div(M * nO, 256)), dim3(256), 0, st, 1, P, (int64_t)(2 * nOp), M, nO, nOp, O_idx, s_O, G, A, r,
-                   dX, lddx);
+                   dX, lddx, 0);
         if ((rc = launch_status()) != QUAFF_OK) return leave(rc);
     }
     return leave(QUAFF_OK);

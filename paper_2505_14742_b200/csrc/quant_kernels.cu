@@ -101,8 +101,20 @@ __device__ __forceinline__ void load_row(uint4 (&raw)[J][2], const uint16_t* __r
 #ifndef QUAFF_QA_MIN_BLOCKS
 #define QUAFF_QA_MIN_BLOCKS 2
 #endif
+#ifndef QUAFF_QA_BLOCKS_J2
+#define QUAFF_QA_BLOCKS_J2 8
+#endif
+#ifndef QUAFF_QA_BLOCKS_J4
+#define QUAFF_QA_BLOCKS_J4 5
+#endif
+#ifndef QUAFF_QA_BLOCKS_J6
+#define QUAFF_QA_BLOCKS_J6 4
+#endif
+// CTA size and residency the compiler may assume: rows of up to 4096 columns (J <= 2) run in CTAs of at most 128
+// threads, eight of them per SM (64 registers per thread); wider rows keep more of the row per thread.
+template <int J> struct QaBounds { static constexpr int kThreads = J <= 6 ? 128 : 256, kBlocks = J <= 2 ? QUAFF_QA_BLOCKS_J2 : (J <= 4 ? QUAFF_QA_BLOCKS_J4 : (J <= 6 ? QUAFF_QA_BLOCKS_J6 : QUAFF_QA_MIN_BLOCKS)); };
 template <int J, bool TAIL>
-__global__ void __launch_bounds__(256, QUAFF_QA_MIN_BLOCKS) quant_act_kernel(const uint16_t* __restrict__ X, int64_t ldx, int M, int K,
+__global__ void __launch_bounds__(QaBounds<J>::kThreads, QaBounds<J>::kBlocks) quant_act_kernel(const uint16_t* __restrict__ X, int64_t ldx, int M, int K,
                                                         const int32_t* __restrict__ O_idx, int nO,
                                                         const float* __restrict__ s_O,
                                                         int8_t* __restrict__ Xq, int64_t ldxq,
@@ -120,6 +132,11 @@ __global__ void __launch_bounds__(256, QUAFF_QA_MIN_BLOCKS) quant_act_kernel(con
 
     const int lane = tid & 31, warp = tid >> 5, nwarps = T >> 5;
     const int nunits = (K + 15) >> 4;
+
+    // the CTA's first row is requested before anything else: its latency covers the staging of O below
+    uint4 raw[J][2];
+    int m = blockIdx.x;
+    if (m < M) load_row<J, TAIL>(raw, X + (int64_t)m * ldx, tid, T, K);
 
     for (int i = tid; i < nO; i += T) {
         O_s[i] = O_idx[i];
@@ -149,9 +166,6 @@ __global__ void __launch_bounds__(256, QUAFF_QA_MIN_BLOCKS) quant_act_kernel(con
         keep_s[(j * 2 + 1) * T + tid] = make_uint4(kw[4], kw[5], kw[6], kw[7]);
     }
 
-    uint4 raw[J][2];
-    int m = blockIdx.x;
-    if (m < M) load_row<J, TAIL>(raw, X + (int64_t)m * ldx, tid, T, K);
     int parity = 0;
     for (; m < M; m += gridDim.x, parity ^= 1) {
         const uint16_t* xrow = X + (int64_t)m * ldx;

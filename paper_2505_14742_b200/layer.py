@@ -25,7 +25,7 @@ class QuaffLinear:
     def __init__(self, Wt: torch.Tensor, O_idx: Optional[torch.Tensor], A: Optional[torch.Tensor],
                  B: Optional[torch.Tensor], lora_scale: float, gamma: float, max_tokens: int,
                  y_dtype: torch.dtype = torch.bfloat16, debug_acc: bool = False, keep_G: bool = False,
-                 int8_grad: bool = False):
+                 int8_grad: bool = False, lean_bwd: bool = False):
         dev = Wt.device
         self.N, self.K = Wt.shape
         self.nO = 0 if O_idx is None else int(O_idx.numel())
@@ -60,11 +60,13 @@ class QuaffLinear:
         # G = bf16(lora_scale dY B^T) of the last backward, kept on request (otherwise it lives in the workspace)
         self.G = torch.empty((M, r), dtype=bf, device=dev) if (keep_G and r) else None
         self.status = torch.zeros(4, dtype=torch.int32, device=dev)
+        # lean_bwd: a workspace without room for a bf16 copy of the weight: the grad-input GEMM expands the codes in-kernel
         # int8_grad: the backward runs the INT8 grad-input variant (quaff_qlinear_bwd_int8) - not the paper's method
         self.int8_grad = bool(int8_grad)
         ws_bytes = max(Q.workspace_bytes(Q.QUAFF_WS_MOMENTUM, M, K, N, nOp, r),
                        Q.workspace_bytes(Q.QUAFF_WS_FWD, M, K, N, nOp, r),
-                       Q.workspace_bytes(Q.QUAFF_WS_BWD_INT8 if int8_grad else Q.QUAFF_WS_BWD, M, K, N, nOp, r), 256)
+                       Q.workspace_bytes(Q.QUAFF_WS_BWD_INT8 if int8_grad else (Q.QUAFF_WS_BWD_LEAN if lean_bwd else Q.QUAFF_WS_BWD),
+                                         M, K, N, nOp, r), 256)
         self.ws = torch.empty(ws_bytes, dtype=torch.uint8, device=dev)
         # the LoRA down-projection runs beside the quantization chain, on its own stream and workspace
         self.ws_lora = torch.empty(max(Q.workspace_bytes(Q.QUAFF_WS_FWD, M, K, N, nOp, r), 256), dtype=torch.uint8, device=dev) if r else None

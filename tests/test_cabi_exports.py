@@ -47,13 +47,13 @@ def test_host_only_paths_from_two_threads():
     from paper_2505_14742_b200 import binding as Q
     L = Q.lib()
     shapes = [(256, 512, 512, 32, 8), (2048, 3072, 9216, 32, 16), (8192, 11008, 4096, 64, 64), (512, 2048, 4096, 128, 8)]
-    want = [[Q.workspace_bytes(w, *sh) for w in range(6)] for sh in shapes]
+    want = [[Q.workspace_bytes(w, *sh) for w in range(8)] for sh in shapes]
     bad = []
 
     def worker():
         for _ in range(300):
             for sh, ref in zip(shapes, want):
-                if [Q.workspace_bytes(w, *sh) for w in range(6)] != ref:
+                if [Q.workspace_bytes(w, *sh) for w in range(8)] != ref:
                     bad.append(sh)
             # null pointers / bad sizes: rejected on the host, no device needed
             if L.quaff_qlinear_bwd(16, 64, 64, None, 64, None, 64, None, None, 0, None, 0, None, 0, None, None, 0, None, None, None, 0,

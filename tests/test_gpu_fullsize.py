@@ -16,7 +16,7 @@ from util import TOL_BF16, check_bf16_intermediate, dev, dev_bf16, dx_floor, hos
 pytestmark = pytest.mark.gpu
 
 
-def _run_layer(wl, li, steps, nsample, check_acc, full_grads=True, int8_grad=False):
+def _run_layer(wl, li, steps, nsample, check_acc, full_grads=True, int8_grad=False, lean_bwd=False):
     import torch
     from paper_2505_14742_b200 import build
     from paper_2505_14742_b200.layer import QuaffLinear, StepGraph
@@ -28,7 +28,7 @@ def _run_layer(wl, li, steps, nsample, check_acc, full_grads=True, int8_grad=Fal
     nOp = synth.pad_to(sp.nO, 32)
     # keep_G: the backward writes G into a buffer of the layer instead of its workspace (same kernels, same launches)
     layer = QuaffLinear(dev_bf16(lin.W), dev(lin.O_idx), dev_bf16(lin.A), dev_bf16(lin.B), scale, wl.gamma, M, keep_G=True,
-                        int8_grad=int8_grad)
+                        int8_grad=int8_grad, lean_bwd=lean_bwd)
     Xd = torch.empty((M, K), dtype=torch.bfloat16, device="cuda")
     dYd = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
 
@@ -127,6 +127,12 @@ def test_llama7b_block_layers_full_size(li):
 @pytest.mark.parametrize("wl_name,li", [("llama7b_block", 4), ("phi3_attn", 0)], ids=["llama_gate_proj", "phi3_qkv"])
 def test_int8_grad_variant_full_size(wl_name, li):
     _run_layer(synth.WORKLOADS[wl_name], li, steps=1, nsample=24, check_acc=False, full_grads=False, int8_grad=True)
+
+
+# The backward without a bf16 copy of the weight (codes expanded inside the grad-input GEMM) at full size
+@pytest.mark.parametrize("wl_name,li", [("llama7b_block", 6), ("phi3_attn", 0)], ids=["llama_down_proj", "phi3_qkv"])
+def test_in_kernel_expansion_full_size(wl_name, li):
+    _run_layer(synth.WORKLOADS[wl_name], li, steps=1, nsample=24, check_acc=False, full_grads=False, lean_bwd=True)
 
 
 # Phi-3 MLP, 4096 tokens: fused gate_up 3072 -> 16384 and down 8192 -> 3072, one forward + backward step each

@@ -265,6 +265,24 @@ def test_qlinear_bwd(Q, M, K, N, nO, r):
     if r:
         err_a, err_b = max_rel_err(host(dA), odA), max_rel_err(host(dB), odB)
         assert err_a <= TOL_BF16 and err_b <= TOL_BF16, f"dA {err_a:.3e} dB {err_b:.3e}"
+    # The same call with a workspace that has no room for a bf16 copy of the weight: the grad-input GEMM then expands the
+    # INT8 codes inside the kernel.  Same products in the same order: bit-identical off the outlier columns (those differ
+    # in how the two partial products are separated), the same gradients, and within tolerance of the oracle everywhere.
+    lean = Q.workspace_bytes(Q.QUAFF_WS_BWD_LEAN, M, K, N, nOp, r)
+    assert lean < Q.workspace_bytes(Q.QUAFF_WS_BWD, M, K, N, nOp, r)
+    ws_lean = torch.empty(lean, dtype=torch.uint8, device="cuda")
+    dXl = torch.full((M + 2, K + 8), -777.0, dtype=torch.bfloat16, device="cuda")
+    dAl, dBl = (torch.full_like(dA, 3.0), torch.full_like(dB, 3.0)) if r else (None, None)
+    Q.quaff_qlinear_bwd(*args[:12], dXl[:M, :K], dAl, dBl, False, ws_lean, st)
+    torch.cuda.synchronize()
+    assert host(st)[0] == 0
+    assert bool((dXl[M:, :] == -777.0).all()) and bool((dXl[:, K:] == -777.0).all()), "write outside dX (in-kernel expansion)"
+    off_O = np.setdiff1d(np.arange(K), O)
+    assert np.array_equal(host_bits(dXl[:M, :K].contiguous())[:, off_O], host_bits(dX.contiguous())[:, off_O]), "in-kernel expansion: dX bits"
+    err = max_rel_err(host(dXl[:M, :K]), odX, dx_floor(N))
+    assert err <= TOL_BF16, f"dX (in-kernel expansion) max rel err {err:.3e}"
+    if r:
+        assert np.array_equal(host(dAl), host(dA)) and np.array_equal(host(dBl), host(dB))
     # the two halves of the call on their own (other stream layout inside the library): the same kernels, the same bits
     dX2 = torch.full((M, K), float("nan"), dtype=torch.bfloat16, device="cuda")
     Q.quaff_qlinear_bwd(*args[:12], dX2, None, None, False, ws, st)            # dX only
