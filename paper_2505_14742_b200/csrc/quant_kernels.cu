@@ -101,18 +101,16 @@ __device__ __forceinline__ void load_row(uint4 (&raw)[J][2], const uint16_t* __r
 #ifndef QUAFF_QA_MIN_BLOCKS
 #define QUAFF_QA_MIN_BLOCKS 2
 #endif
-#ifndef QUAFF_QA_BLOCKS_J2
-#define QUAFF_QA_BLOCKS_J2 8
-#endif
-#ifndef QUAFF_QA_BLOCKS_J4
-#define QUAFF_QA_BLOCKS_J4 5
-#endif
-#ifndef QUAFF_QA_BLOCKS_J6
-#define QUAFF_QA_BLOCKS_J6 4
+#ifndef QUAFF_QA_PERSM_J2
+#define QUAFF_QA_PERSM_J2 1024
 #endif
 // CTA size and residency the compiler may assume: rows of up to 4096 columns (J <= 2) run in CTAs of at most 128
 // threads, eight of them per SM (64 registers per thread); wider rows keep more of the row per thread.
-template <int J> struct QaBounds { static constexpr int kThreads = J <= 6 ? 128 : 256, kBlocks = J <= 2 ? QUAFF_QA_BLOCKS_J2 : (J <= 4 ? QUAFF_QA_BLOCKS_J4 : (J <= 6 ? QUAFF_QA_BLOCKS_J6 : QUAFF_QA_MIN_BLOCKS)); };
+template <int J> struct QaBounds {
+    static constexpr int kThreads = (J <= 6 && QUAFF_QA_MAX_THREADS <= 128) ? 128 : 256;
+    static constexpr int kPerSm = J <= 2 ? QUAFF_QA_PERSM_J2 : (J <= 4 ? 640 : (J <= 6 ? 512 : 512));      // threads per SM the registers must allow
+    static constexpr int kBlocks = kPerSm / kThreads;
+};
 template <int J, bool TAIL>
 __global__ void __launch_bounds__(QaBounds<J>::kThreads, QaBounds<J>::kBlocks) quant_act_kernel(const uint16_t* __restrict__ X, int64_t ldx, int M, int K,
                                                         const int32_t* __restrict__ O_idx, int nO,
@@ -169,7 +167,8 @@ __global__ void __launch_bounds__(QaBounds<J>::kThreads, QaBounds<J>::kBlocks) q
     int parity = 0;
     for (; m < M; m += gridDim.x, parity ^= 1) {
         const uint16_t* xrow = X + (int64_t)m * ldx;
-        // the CTA's next row is on its way while this one is processed
+        // the CTA's next row is on its way while this one is processed (measured: a second row in flight, in registers or
+        // as L2 prefetches, does not help - the kernel is not bound by the bytes in flight)
         uint4 nxt[J][2];
         const int mn = m + gridDim.x;
         if (mn < M) load_row<J, TAIL>(nxt, X + (int64_t)mn * ldx, tid, T, K);
