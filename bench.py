@@ -532,7 +532,7 @@ def run_micro(args):
     X[:, O.long()] *= 50.0
     s = 1.0 + 10.0 * torch.rand(nO, device="cuda", generator=g)
     flush = torch.empty(512 << 20, dtype=torch.uint8, device="cuda")
-    if args.micro in ("fwd", "bwd"):
+    if args.micro in ("fwd", "bwd", "bwd8"):
         # one layer's forward (or backward) call on random codes; the tensor-core GEMM inside it is timed by the
         # library's event pair (quaff_debug_time_gemm), everything else of the call runs untimed around it
         r = args.micro_rank
@@ -548,7 +548,8 @@ def run_micro(args):
         dA = torch.zeros((K, r), device="cuda"); dB = torch.zeros((r, N), device="cuda")
         st = torch.zeros(4, dtype=torch.int32, device="cuda")
         ws = torch.empty(max(Q.workspace_bytes(Q.QUAFF_WS_FWD, M, K, N, nOp, r),
-                             Q.workspace_bytes(Q.QUAFF_WS_BWD_LEAN if args.lean_bwd else Q.QUAFF_WS_BWD, M, K, N, nOp, r)),
+                             Q.workspace_bytes(Q.QUAFF_WS_BWD_INT8 if args.micro == "bwd8" else
+                                               (Q.QUAFF_WS_BWD_LEAN if args.lean_bwd else Q.QUAFF_WS_BWD), M, K, N, nOp, r)),
                          dtype=torch.uint8, device="cuda")
         Q.quaff_qlinear_fwd(Xq, xqo, dxv, Wq, dWv, wqo, dwOv, X, A, B, 1.0, T, Y, ws, None, None, st)
         which = 0 if args.micro == "fwd" else 1
@@ -560,6 +561,8 @@ def run_micro(args):
             Q.quaff_debug_time_gemm(which, e0, e1)
             if which == 0:
                 Q.quaff_qlinear_fwd(Xq, xqo, dxv, Wq, dWv, wqo, dwOv, X, A, B, 1.0, T, Y, ws, None, None, st)
+            elif args.micro == "bwd8":   # the INT8 grad-input variant (not the paper's method): its INT8 GEMM is the timed kernel
+                Q.quaff_qlinear_bwd_int8(dY, Wq, dWv, wqo, dwOv, O, s, X, T, A, B, 1.0, dX, None, None, False, ws, st)
             else:
                 # (dX only: with dA / dB the library schedules their split-K GEMMs into the SMs the grad-input GEMM leaves idle)
                 Q.quaff_qlinear_bwd(dY, Wq, dWv, wqo, dwOv, O, s, X, T, A, B, 1.0, dX, None, None, False, ws, st)
@@ -569,12 +572,13 @@ def run_micro(args):
         assert int(st[0].item()) == 0, "device-side wait timed out"
         ms = float(np.median(times))
         peaks = load_peaks()
-        work = 2.0 * M * N * (K + nOp + r) if which == 0 else 2.0 * M * N * (K + 2 * nOp) + 2.0 * M * K * r
-        peak = peaks["bf16_tflops"] * (2.0 if which == 0 else 1.0)
+        work = 2.0 * M * N * (K + nOp + r) if which == 0 else 2.0 * M * N * (K + nOp) + 2.0 * M * K * r
+        int8 = which == 0 or args.micro == "bwd8"
+        peak = peaks["bf16_tflops"] * (2.0 if int8 else 1.0)
         print(json.dumps({"micro": args.micro, "shape": {"M": M, "K": K, "N": N, "nO": nO, "r": r}, "ms_per_launch": ms, "launches": len(times),
                           "roofline": {"bound": "tensor", "achieved": work / (ms * 1e-3) / 1e12, "peak": peak,
-                                       "unit": "TOP/s" if which == 0 else "TFLOP/s", "frac": work / (ms * 1e-3) / 1e12 / peak,
-                                       "peak_source": f"{peaks['source']} cuBLAS bf16 burst" + (" x2 (nominal int8:bf16 ratio)" if which == 0 else "")}}),
+                                       "unit": "TOP/s" if int8 else "TFLOP/s", "frac": work / (ms * 1e-3) / 1e12 / peak,
+                                       "peak_source": f"{peaks['source']} cuBLAS bf16 burst" + (" x2 (nominal int8:bf16 ratio)" if int8 else "")}}),
               flush=True)
         return
     # R rotating buffer sets, together at least 2.5 times the 126 MB L2, so that back-to-back launches read HBM
@@ -743,7 +747,7 @@ def run_sweep(args):
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--micro", default=None, choices=["quant_act", "quant_grad", "momentum", "requant", "outlier_count", "lora_down", "fwd", "bwd"],
+    ap.add_argument("--micro", default=None, choices=["quant_act", "quant_grad", "momentum", "requant", "outlier_count", "lora_down", "fwd", "bwd", "bwd8"],
                     help="time one HBM-bound kernel alone instead of the step")
     ap.add_argument("--micro-shape", type=lambda v: tuple(int(x) for x in v.split(",")), default=(8192, 11008, 4096, 55),
                     help="M,K,N,nO of --micro (default: the LLaMA-2-7B down_proj rows)")
