@@ -524,3 +524,40 @@ def test_qlinear_bwd_int8(Q, M, K, N, nO, r):
     if r:
         err_a, err_b = max_rel_err(host(dA), odA), max_rel_err(host(dB), odB)
         assert err_a <= TOL_BF16 and err_b <= TOL_BF16, f"dA {err_a:.3e} dB {err_b:.3e}"
+
+
+# ----------------------------------------------------------------------------- state: determinism and checkpoint / resume
+def test_checkpoint_resume_and_determinism(Q):
+    """The only state a layer carries between steps is s_O (a caller-owned buffer).  Ten steps in one go, and five steps +
+    a copy of s_O into a fresh layer + five more steps, end in the same bits everywhere (s_O, codes, Y, dX, dA, dB); so does
+    a second run of the ten steps (no floating-point atomics, fixed split-K reduction order)."""
+    import torch
+    from paper_2505_14742_b200.layer import QuaffLinear
+    wl = synth.WORKLOADS["tiny"]
+    lin = synth.layer_inputs(wl, 0, b_std=0.02)
+    scale = wl.lora_alpha / lin.spec.r
+
+    def make():
+        return QuaffLinear(dev_bf16(lin.W), dev(lin.O_idx), dev_bf16(lin.A), dev_bf16(lin.B), scale, wl.gamma, wl.M)
+
+    def run(layer, steps):
+        out = None
+        for step in steps:
+            X, dY = synth.step_inputs(wl, 0, step, lin)
+            Y = layer.forward(dev_bf16(X))
+            dX, dA, dB = layer.backward(dev_bf16(dY))
+            torch.cuda.synchronize()
+            out = [host(layer.s_O), host(layer.Xq), host(layer.wq_O), host_bits(Y), host_bits(dX), host(dA), host(dB)]
+        return out
+
+    straight = run(make(), range(10))
+    again = run(make(), range(10))
+    first = make()
+    run(first, range(5))
+    saved = first.s_O.clone()                     # the checkpoint
+    resumed = make()
+    resumed.s_O.copy_(saved)
+    split = run(resumed, range(5, 10))
+    for a, b, c in zip(straight, again, split):
+        assert np.array_equal(a, b), "two runs of the same steps differ"
+        assert np.array_equal(a, c), "resuming from a saved s_O differs"
