@@ -269,7 +269,7 @@ quaff_status_t quaff_qlinear_bwd(int M, int K, int N,
  * for every k outside O; the nO outlier columns keep the floating-point path of quaff_qlinear_bwd,
  *   dXhat[m][O_i] = (sum_n dY[m][n] (Wd[n][O_i] + wd[n][i])) / s_O[i].
  * G, dX = dXhat + G A^T, dA, dB and all other arguments are those of quaff_qlinear_bwd; dX is required; N must be a
- * multiple of 16; dbg_acc_opt: optional dense [M][K] int32 dump of sum_n Zq Wq (parity checks);  ws: QUAFF_WS_BWD_INT8 bytes.
+ * multiple of 16, at most 16384 (more: QUAFF_ERR_UNSUPPORTED_SHAPE); dbg_acc_opt: optional dense [M][K] int32 dump of sum_n Zq Wq (parity checks);  ws: QUAFF_WS_BWD_INT8 bytes.
  * quaff_quant_grad is the quantization step on its own (Zq [M][N] int8 with ldz % 16 == 0, dz [M] f32).
  */
 quaff_status_t quaff_quant_grad(const quaff_bf16* dY, int64_t lddy, int M, int N, const float* dW, int8_t* Zq, int64_t ldz,

@@ -1127,7 +1127,7 @@ extern "C" quaff_status_t quaff_qlinear_bwd_int8(int M, int K, int N, const quaf
     QUAFF_RETURN_IF(nO > 0 && (!O_idx || !s_O), QUAFF_ERR_INVALID_ARG);
     QUAFF_RETURN_IF(r > 0 && (!A || !B), QUAFF_ERR_INVALID_ARG);
     QUAFF_RETURN_IF(r > 0 && (dA || dB) && (!dA || !dB || !X || !T || ldx < K), QUAFF_ERR_INVALID_ARG);
-    QUAFF_RETURN_IF((nOp % 32) || (r % 8) || r > 64 || (N % 16), QUAFF_ERR_UNSUPPORTED_SHAPE);
+    QUAFF_RETURN_IF((nOp % 32) || (r % 8) || r > 64 || (N % 16) || N > 16384, QUAFF_ERR_UNSUPPORTED_SHAPE);
     QUAFF_RETURN_IF(!aligned16(dY) || (lddy % 8) || !aligned16(dW), QUAFF_ERR_ALIGNMENT);
     QUAFF_RETURN_IF(!aligned16(Wq) || (ldwq_main % 16), QUAFF_ERR_ALIGNMENT);
     QUAFF_RETURN_IF(nOp > 0 && (!aligned16(wq_O) || (ldwq % 16)), QUAFF_ERR_ALIGNMENT);

@@ -294,6 +294,22 @@ __global__ void __launch_bounds__(256, 2) quant_grad_kernel(const uint16_t* __re
     __shared__ float red[2][8];
     const int tid = threadIdx.x, T = blockDim.x;
     const int lane = tid & 31, warp = tid >> 5, nwarps = T >> 5;
+    // this thread's column scales are the same for every row: with up to two units per thread they are read once and kept
+    // in registers (16 per unit); with more units they are re-read per row (L1 / L2 hits), the registers go to the products
+    constexpr bool kCacheScales = J <= 2;
+    float sc[kCacheScales ? J : 1][16];
+    auto load_scales = [&](int j, float (&dst)[16]) {
+        const int k0 = (tid + j * T) << 4;
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            const float4 v = k0 < N ? __ldg(reinterpret_cast<const float4*>(colscale + k0) + q) : make_float4(0.f, 0.f, 0.f, 0.f);
+            dst[4 * q] = v.x; dst[4 * q + 1] = v.y; dst[4 * q + 2] = v.z; dst[4 * q + 3] = v.w;
+        }
+    };
+    if (kCacheScales) {
+#pragma unroll
+        for (int j = 0; j < J; ++j) load_scales(j, sc[kCacheScales ? j : 0]);
+    }
     uint4 raw[J][2];
     int m = blockIdx.x;
     if (m < M) load_row<J, false>(raw, dY + (int64_t)m * lddy, tid, T, N);
@@ -302,18 +318,23 @@ __global__ void __launch_bounds__(256, 2) quant_grad_kernel(const uint16_t* __re
         uint4 nxt[J][2];
         const int mn = m + gridDim.x;
         if (mn < M) load_row<J, false>(nxt, dY + (int64_t)mn * lddy, tid, T, N);
+        // z = x * scale (one fp32 product), kept for the rounding pass; absmax over the row
+        float z[J][16];
         float amax = 0.0f;
 #pragma unroll
         for (int j = 0; j < J; ++j) {
-            const int k0 = (tid + j * T) << 4;
-            if (k0 >= N) continue;
-            const float4* sc = reinterpret_cast<const float4*>(colscale + k0);
+            float tmp[16];
+            if (!kCacheScales) load_scales(j, tmp);
+            const float (&scj)[16] = kCacheScales ? sc[kCacheScales ? j : 0] : tmp;
 #pragma unroll
             for (int h = 0; h < 2; ++h) {
-                float z[8];
-                scaled8(raw[j][h], __ldg(sc + 2 * h), __ldg(sc + 2 * h + 1), z);
+                const uint32_t w[4] = {raw[j][h].x, raw[j][h].y, raw[j][h].z, raw[j][h].w};
 #pragma unroll
-                for (int e = 0; e < 8; ++e) amax = fmaxf(amax, fabsf(z[e]));
+                for (int i = 0; i < 4; ++i) {
+                    z[j][8 * h + 2 * i] = __fmul_rn(bf16_lo(w[i]), scj[8 * h + 2 * i]);
+                    z[j][8 * h + 2 * i + 1] = __fmul_rn(bf16_hi(w[i]), scj[8 * h + 2 * i + 1]);
+                    amax = fmaxf(amax, fmaxf(fabsf(z[j][8 * h + 2 * i]), fabsf(z[j][8 * h + 2 * i + 1])));
+                }
             }
         }
 #pragma unroll
@@ -331,17 +352,12 @@ __global__ void __launch_bounds__(256, 2) quant_grad_kernel(const uint16_t* __re
         for (int j = 0; j < J; ++j) {
             const int k0 = (tid + j * T) << 4;
             if (k0 >= N) continue;
-            const float4* sc = reinterpret_cast<const float4*>(colscale + k0);
             uint32_t out[4];
 #pragma unroll
-            for (int h = 0; h < 2; ++h) {
-                float z[8];
-                scaled8(raw[j][h], __ldg(sc + 2 * h), __ldg(sc + 2 * h + 1), z);
-                uint32_t c[8];
-#pragma unroll
-                for (int e = 0; e < 8; ++e) c[e] = code_bits(z[e], rinv);
-                out[2 * h] = __byte_perm(__byte_perm(c[0], c[1], 0x0040), __byte_perm(c[2], c[3], 0x0040), 0x5410);
-                out[2 * h + 1] = __byte_perm(__byte_perm(c[4], c[5], 0x0040), __byte_perm(c[6], c[7], 0x0040), 0x5410);
+            for (int q = 0; q < 4; ++q) {
+                const uint32_t c0 = code_bits(z[j][4 * q], rinv), c1 = code_bits(z[j][4 * q + 1], rinv);
+                const uint32_t c2 = code_bits(z[j][4 * q + 2], rinv), c3 = code_bits(z[j][4 * q + 3], rinv);
+                out[q] = __byte_perm(__byte_perm(c0, c1, 0x0040), __byte_perm(c2, c3, 0x0040), 0x5410);
             }
             *reinterpret_cast<uint4*>(qrow + k0) = make_uint4(out[0], out[1], out[2], out[3]);
         }
@@ -366,18 +382,18 @@ static quaff_status_t launch_quant_grad(int T, const uint16_t* dY, int64_t lddy,
 quaff_status_t quant_grad_dispatch(const uint16_t* dY, int64_t lddy, int M, int N, const float* colscale, int8_t* Zq, int64_t ldz,
                                    float* dz, cudaStream_t st) {
     const int nunits = N / 16;
-    if ((N % 16) || nunits > 8 * 256) return QUAFF_ERR_UNSUPPORTED_SHAPE;
-    // units per thread: small CTAs (128 threads or fewer) up to 4 units; rows beyond 8192 columns take 256 threads
-    // rather than 8 units (the row and the prefetched next row would no longer fit the registers)
+    if ((N % 16) || nunits > 4 * 256) return QUAFF_ERR_UNSUPPORTED_SHAPE;
+    // units of 16 columns per thread: as few as keep the CTA at 256 threads or fewer (1..4); up to 4096 columns two units
+    // per thread in CTAs of 128 threads or fewer
     int J = 1;
-    while (J < 4 && ceil_div(nunits, J) > kQuantActMaxThreads) J *= 2;
-    if (ceil_div(nunits, J) > 256) J = 8;
+    while (J < 4 && ceil_div(nunits, J) > 256) ++J;
+    if (J == 1 && nunits > kQuantActMaxThreads) J = 2;
     const int T = min(256, ceil_div(ceil_div(nunits, J), 32) * 32);
     switch (J) {
         case 1: return launch_quant_grad<1>(T, dY, lddy, M, N, colscale, Zq, ldz, dz, st);
         case 2: return launch_quant_grad<2>(T, dY, lddy, M, N, colscale, Zq, ldz, dz, st);
-        case 4: return launch_quant_grad<4>(T, dY, lddy, M, N, colscale, Zq, ldz, dz, st);
-        default: return launch_quant_grad<8>(T, dY, lddy, M, N, colscale, Zq, ldz, dz, st);
+        case 3: return launch_quant_grad<3>(T, dY, lddy, M, N, colscale, Zq, ldz, dz, st);
+        default: return launch_quant_grad<4>(T, dY, lddy, M, N, colscale, Zq, ldz, dz, st);
     }
 }
 
@@ -676,7 +692,7 @@ extern "C" quaff_status_t quaff_momentum_update_static(const quaff_bf16* X, int6
 extern "C" quaff_status_t quaff_quant_grad(const quaff_bf16* dY, int64_t lddy, int M, int N, const float* dW, int8_t* Zq,
                                            int64_t ldz, float* dz, quaff_stream_t stream) {
     QUAFF_RETURN_IF(!dY || !dW || !Zq || !dz || M < 0 || N <= 0 || lddy < N || ldz < N, QUAFF_ERR_INVALID_ARG);
-    QUAFF_RETURN_IF(N % 16, QUAFF_ERR_UNSUPPORTED_SHAPE);
+    QUAFF_RETURN_IF((N % 16) || N > 16384, QUAFF_ERR_UNSUPPORTED_SHAPE);
     QUAFF_RETURN_IF(!aligned16(dY) || !aligned16(Zq) || !aligned16(dW) || (lddy % 8) || (ldz % 16), QUAFF_ERR_ALIGNMENT);
     if (M == 0) return QUAFF_OK;
     return quant_grad_dispatch(dY, lddy, M, N, dW, Zq, ldz, dz, (cudaStream_t)stream);
