@@ -32,8 +32,10 @@ def build(force: bool = False) -> str:
 def _load():
     global _lib
     if _lib is None:
-        build()
-        _lib = ctypes.CDLL(_LIB)
+        # QUAFF_ORACLE_LIB: load this shared object instead (the mutation test points the pins at copies of the
+        # oracle with one planted mistake each; nothing else sets it)
+        other = os.environ.get("QUAFF_ORACLE_LIB")
+        _lib = ctypes.CDLL(other) if other else ctypes.CDLL(build())
         _lib.qo_num_threads.restype = ctypes.c_int
         _lib.qo_int_gemm.restype = ctypes.c_int64
         _lib.qo_qlinear_fwd.restype = ctypes.c_int64

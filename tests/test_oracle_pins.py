@@ -387,6 +387,37 @@ def test_supplied_intermediates_T_and_G_are_used_as_given():
 
 
 # ----------------------------------------------------------------------------- backward
+def test_bf16_roundings_are_to_nearest_even_and_single():
+    """The three places where the oracle rounds to bf16, on values whose correct rounding is known by hand
+    (bf16 keeps 8 significant bits; 1 + 2^-8 lies exactly half way between 1 and 1 + 2^-7):
+    T = bf16(X A) and G = bf16(scale dY B^T) round the exact sum ONCE (1 + 2^-8 + 2^-30 is above the half-way point and
+    goes up, although it would first collapse onto the tie in fp32 and then go down), ties go to the even neighbour,
+    and Wd = bf16(code * Delta_W) rounds the fp32 product the same way."""
+    one, up = 0x3F80, 0x3F81                                  # 1.0 and 1 + 2^-7
+    ones = bf(np.ones((1, 3), np.float32))
+    col = bf(np.array([[1.0], [2.0 ** -8], [2.0 ** -30]], np.float32))
+    tie = bf(np.array([[1.0], [2.0 ** -8], [0.0]], np.float32))
+    odd = bf(np.array([[1.0 + 2.0 ** -7], [2.0 ** -8], [0.0]], np.float32))   # tie above an odd pattern: up to 1 + 2^-6
+    for a_col, want in ((col, up), (tie, one), (odd, 0x3F82)):
+        T = oracle.lora_down(ones, a_col)
+        assert T.shape == (1, 1) and int(T[0, 0]) == want
+        # G = bf16(1 * dY B^T) with dY = ones [1][3], B [1][3] = the same column as a row
+        z8 = np.zeros((3, 1), np.int8)
+        _, _, _, G = oracle.qlinear_bwd(ones, z8, np.zeros(3, np.float32), np.zeros((3, 0), np.int8), np.zeros(3, np.float32),
+                                        np.zeros(0, np.int32), np.zeros(0, np.float32), bf(np.zeros((1, 1), np.float32)),
+                                        bf(np.zeros((1, 1), np.float32)), bf(np.zeros((1, 1), np.float32)),
+                                        np.ascontiguousarray(a_col.reshape(1, 3)), 1.0, want_dX=False, want_dAB=False)
+        assert int(G[0, 0]) == want
+    # Wd: code 1 x step 1 + 2^-8 is the tie (down to 1); code 3 x the same step is 3 + 3 * 2^-8 = 1.1000000|11b x 2, above
+    # half way (up to 3 + 2^-6 = 3.015625); code -1 mirrors code 1.  dY = identity, so dX is Wd itself.
+    Wq = np.array([[1], [3], [-1]], np.int8)
+    dW = np.full(3, 1.0 + 2.0 ** -8, np.float32)
+    dX, _, _, _ = oracle.qlinear_bwd(bf(np.eye(3, dtype=np.float32)), Wq, dW, np.zeros((3, 0), np.int8), np.zeros(3, np.float32),
+                                     np.zeros(0, np.int32), np.zeros(0, np.float32), bf(np.zeros((3, 1), np.float32)),
+                                     None, None, None, 1.0, want_dAB=False)
+    assert dX[:, 0].tolist() == [1.0, 3.015625, -1.0]
+
+
 def _dequantized_map(O, Wq, dW, wq, dw, s, K):
     """The linear map of Eq. 9 with the codes held fixed: Y = X @ Weff, Weff[k,n]."""
     Wd = f32(bf(Wq.astype(np.float32) * dW[:, None])).astype(np.float64)          # [N,K]
@@ -596,6 +627,15 @@ def test_outlier_count_fixed_point_truncation_and_accumulation():
     assert xi.tolist() == [5, 8]
     xi = oracle.outlier_count(X, 2, xi)                                 # 64 * 2 > 2 * 64 is false (strict)
     assert xi.tolist() == [5, 8]
+
+
+def test_outlier_count_saturates_magnitudes_at_two_to_the_32():
+    # |x| in units of 2^-16 saturates at 2^32 - 1: 2^20 and 2^16 both count as 2^32 - 1 = S.
+    X = synth.f32_to_bf16_bits(np.array([[2.0 ** 20, 2.0 ** 16, 0.0, 0.0]], np.float32))
+    xi = oracle.outlier_count(X, 1, np.zeros(4, np.int32))              # S * 4 > 1 * 2S for both; 0 * 4 > 2S is false
+    assert xi.tolist() == [1, 1, 0, 0]
+    xi = oracle.outlier_count(X, 2, np.zeros(4, np.int32))              # S * 4 > 2 * 2S is false (unsaturated, 2^20 would count)
+    assert xi.tolist() == [0, 0, 0, 0]
 
 
 def test_outlier_count_matches_brute_force_and_finds_planted_channels():
