@@ -24,6 +24,8 @@
  *    A device-side wait that gave up (after about two seconds) is reported through the optional `status` word
  *    (QUAFF_ERR_TIMEOUT) after the stream has been synchronised; outputs are then undefined.
  *  - Inputs must be finite.  Results are deterministic (no floating-point atomics).
+ *  - An empty batch (M = 0) is valid wherever M is a token count (the calibration calls need M >= 1): nothing is
+ *    launched, and a backward call that does not accumulate stores the empty sums dA = 0 and dB = 0.
  *  - The outlier set: 0 <= nO <= K and nO <= 4096 in every entry point that takes one (more: QUAFF_ERR_UNSUPPORTED_SHAPE).
  *  - Threads: every entry point may be called from several host threads at once, on the same or on different
  *    devices and streams (lazily created per-device resources are guarded; quaff_qlinear_bwd calls on one device are

@@ -446,7 +446,7 @@ constexpr int kPlanSMs = 148;   // split-K plans (and so workspace sizes) are fi
 // than shorter splits save), at least two k-blocks per split.
 struct SplitPlan { int S, kblk; };
 static SplitPlan split_plan(int rows_out, int kc) {
-    const int tiles = ceil_div(rows_out, kTileM);
+    const int tiles = max(1, ceil_div(rows_out, kTileM));   // an empty batch still gets a (never launched) plan
     const int nblk = max(1, ceil_div(kc, 64));
     int S = max(1, min(max(1, kPlanSMs / tiles), ceil_div(nblk, 2)));
     SplitPlan p;
@@ -650,6 +650,15 @@ static quaff_status_t lora_down(const quaff_bf16* X, int64_t ldx, int M, int K, 
     if ((rc = skinny_launch(g, st)) != QUAFF_OK) return rc;
     launch_pdl(reduce_parts_bf16_kernel, dim3(ceil_div(M * r / 8, 256)), dim3(256), 0, st, 1, part, g.S, M, r, 1.0f, T_out);
     return launch_status();
+}
+
+// The backward of an empty batch: nothing to write to dX; the sums dA = X^T G and dB = T^T dY over no tokens are zero,
+// which a call that does not accumulate has to store.
+static quaff_status_t empty_batch_grads(int K, int N, int r, float* dA, float* dB, int accumulate, cudaStream_t st) {
+    if (r <= 0 || !dA || accumulate) return QUAFF_OK;
+    if (cudaMemsetAsync(dA, 0, (size_t)K * r * 4, st) != cudaSuccess) return QUAFF_ERR_CUDA;
+    if (cudaMemsetAsync(dB, 0, (size_t)r * N * 4, st) != cudaSuccess) return QUAFF_ERR_CUDA;
+    return QUAFF_OK;
 }
 
 }  // namespace quaff
@@ -992,7 +1001,7 @@ extern "C" quaff_status_t quaff_qlinear_bwd(int M, int K, int N, const quaff_bf1
     QUAFF_RETURN_IF(!aligned16(dW) || (nOp > 0 && !aligned16(dw_O)), QUAFF_ERR_ALIGNMENT);
     const BwdLeanWorkspace w = bwd_lean_workspace(M, K, N, nOp, r);
     QUAFF_RETURN_IF(!ws || !aligned16(ws) || ws_bytes < w.total, QUAFF_ERR_WORKSPACE_TOO_SMALL);
-    if (M == 0) return QUAFF_OK;
+    if (M == 0) return empty_batch_grads(K, N, r, dA, dB, accumulate, (cudaStream_t)stream);
     cudaStream_t st = (cudaStream_t)stream;
     // Two ways through the frozen INT8 weight, the same products in the same order either way (dX is bit-identical off the
     // outlier columns): with room for a transient bf16 copy of the weight in the workspace (QUAFF_WS_BWD bytes) the copy is
@@ -1136,7 +1145,7 @@ extern "C" quaff_status_t quaff_qlinear_bwd_int8(int M, int K, int N, const quaf
     QUAFF_RETURN_IF(r > 0 && dA && (!aligned16(X) || !aligned16(T) || !aligned16(dA) || !aligned16(dB) || (ldx % 8)), QUAFF_ERR_ALIGNMENT);
     const BwdInt8Workspace w = bwd_int8_workspace(M, K, N, nOp, r);
     QUAFF_RETURN_IF(!ws || !aligned16(ws) || ws_bytes < w.total, QUAFF_ERR_WORKSPACE_TOO_SMALL);
-    if (M == 0) return QUAFF_OK;
+    if (M == 0) return empty_batch_grads(K, N, r, dA, dB, accumulate, (cudaStream_t)stream);
     cudaStream_t st = (cudaStream_t)stream;
     unsigned char* base = reinterpret_cast<unsigned char*>(ws);
     int8_t* Zq = reinterpret_cast<int8_t*>(base + w.off_zq);

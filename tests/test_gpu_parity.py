@@ -488,6 +488,49 @@ def test_quant_grad_rejects_rows_wider_than_it_is_built_for(Q):
     assert e.value.code == Q.QUAFF_ERR_UNSUPPORTED_SHAPE
 
 
+def test_empty_batch_launches_nothing_and_stores_the_empty_sums(Q):
+    """M = 0 is a valid batch: sizes are defined, no output row is touched, and a backward call that does not
+    accumulate stores dA = 0 and dB = 0 (sums over no tokens); one that accumulates leaves them alone."""
+    import torch
+    K, N, nO, nOp, r = 256, 128, 5, 32, 16
+    for which in range(8):
+        assert 0 <= Q.workspace_bytes(which, 0, K, N, nOp, r) < (1 << 24)
+    dev = "cuda"
+    u8 = lambda *sh: torch.full(sh, 0x5A, dtype=torch.uint8, device=dev)
+    Xq, xqo, Wq, wqo = u8(1, K), u8(1, nOp), u8(N, K), u8(N, nOp)
+    dx, dW, dwo, s = (torch.ones(n, device=dev) for n in (1, N, N, nO))
+    O = torch.arange(nO, dtype=torch.int32, device=dev)
+    bfz = lambda *sh: torch.full(sh, 7.0, dtype=torch.bfloat16, device=dev)
+    X, A, B, T, Y, dY, dX = bfz(1, K), bfz(K, r), bfz(r, N), bfz(1, r), bfz(1, N), bfz(1, N), bfz(1, K)
+    dA, dB = torch.full((K, r), 3.0, device=dev), torch.full((r, N), 3.0, device=dev)
+    ws = torch.empty(max(Q.workspace_bytes(w, 1, K, N, nOp, r) for w in range(8)) + 256, dtype=torch.uint8, device=dev)
+    L, p, st = Q.lib(), (lambda t: t.data_ptr()), torch.cuda.current_stream().cuda_stream
+    n0 = Q.quaff_debug_launch_count()
+    assert L.quaff_quant_act(p(X), K, 0, K, p(O), nO, p(s), p(Xq), K, p(xqo), nOp, nOp, p(dx), st) == 0
+    assert L.quaff_lora_down(p(X), K, 0, K, p(A), r, p(T), None, p(ws), ws.numel(), st) == 0
+    assert L.quaff_qlinear_fwd(0, K, N, p(Xq), K, p(xqo), nOp, nOp, p(dx), p(Wq), K, p(dW), p(wqo), nOp, p(dwo), p(X), K, p(A), p(B),
+                               r, 2.0, p(T), p(Y), Q.QUAFF_BF16, N, None, None, None, p(ws), ws.numel(), st) == 0
+    bwd_args = lambda acc: (0, K, N, p(dY), N, p(Wq), K, p(dW), p(wqo), nOp, p(dwo), nOp, p(O), nO, p(s), p(X), K, p(T), p(A), p(B), r,
+                            2.0, p(dX), K, p(dA), p(dB), acc, None)
+    assert L.quaff_qlinear_bwd(*bwd_args(1), None, p(ws), ws.numel(), st) == 0
+    assert L.quaff_qlinear_bwd_int8(*bwd_args(1), None, None, p(ws), ws.numel(), st) == 0
+    assert Q.quaff_debug_launch_count() == n0                 # nothing launched so far
+    torch.cuda.synchronize()
+    assert float(dA.min()) == 3.0 and float(dB.max()) == 3.0  # accumulate: untouched
+    for t in (Xq, xqo):
+        assert int(t.min()) == 0x5A
+    for t in (T, Y, dX):
+        assert float(t.float().min()) == 7.0
+    assert L.quaff_qlinear_bwd(*bwd_args(0), None, p(ws), ws.numel(), st) == 0
+    torch.cuda.synchronize()
+    assert float(dA.abs().max()) == 0.0 and float(dB.abs().max()) == 0.0
+    dA.fill_(3.0); dB.fill_(3.0)
+    assert L.quaff_qlinear_bwd_int8(*bwd_args(0), None, None, p(ws), ws.numel(), st) == 0
+    torch.cuda.synchronize()
+    assert float(dA.abs().max()) == 0.0 and float(dB.abs().max()) == 0.0
+    assert float(dX.float().min()) == 7.0
+
+
 BWD8_SHAPES = [(1, 128, 64, 0, 0), (128, 128, 128, 32, 16), (200, 320, 144, 5, 8), (256, 512, 512, 8, 8),
                (384, 640, 1024, 40, 16), (130, 304, 2048, 33, 64), (100, 256, 256, 3, 0), (520, 1032, 3072, 32, 16),
                (300, 2056, 528, 70, 32), (200, 11008, 528, 1100, 16), (2048, 1000, 1536, 20, 64)]
