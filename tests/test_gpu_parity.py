@@ -529,6 +529,15 @@ def test_empty_batch_launches_nothing_and_stores_the_empty_sums(Q):
     torch.cuda.synchronize()
     assert float(dA.abs().max()) == 0.0 and float(dB.abs().max()) == 0.0
     assert float(dX.float().min()) == 7.0
+    # Eq. 8 over no tokens: the column maxima are 0, beta = 1, and Eq. 7 moves s towards 1 (s = 2, gamma = 0.5: 1.5)
+    s2, wmax = torch.full((nO,), 2.0, device=dev), torch.ones(nO, device=dev)
+    cm, be = torch.full((nO,), -1.0, device=dev), torch.full((nO,), -1.0, device=dev)
+    assert L.quaff_momentum_update(p(X), K, 0, K, p(O), nO, p(wmax), 0.5, p(s2), p(cm), p(be), p(ws), ws.numel(), st) == 0
+    torch.cuda.synchronize()
+    assert s2.tolist() == [1.5] * nO and cm.tolist() == [0.0] * nO and be.tolist() == [1.0] * nO
+    os_, ocm, obe = oracle.momentum_update(np.zeros((0, K), np.uint16), np.arange(nO, dtype=np.int32), np.ones(nO, np.float32), 0.5,
+                                           np.full(nO, 2.0, np.float32))
+    assert os_.tolist() == [1.5] * nO and ocm.tolist() == [0.0] * nO and obe.tolist() == [1.0] * nO
 
 
 BWD8_SHAPES = [(1, 128, 64, 0, 0), (128, 128, 128, 32, 16), (200, 320, 144, 5, 8), (256, 512, 512, 8, 8),
