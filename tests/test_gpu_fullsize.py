@@ -186,20 +186,29 @@ def test_phi3_mlp_late_outliers_momentum_adaptation():
             assert np.all(s[-sp.late:] > 25.0), "the late outlier channels (20-100x) have been picked up by the momentum update"
 
 
-# Twelve points of the shape sweep (tokens x K x N x rank x outlier fraction): together they take every value of every
-# axis - M in {512, 2048, 8192, 32768}, K and N in {2048, 4096, 8192}, rank in {8, 32, 64}, 0.5 / 1 / 5 % outlier
+# Sixteen points of the shape sweep (tokens x K x N x rank x outlier fraction): together they take every value of every
+# axis, and every pair of values of two axes - M in {512, 2048, 8192, 32768}, K and N in {2048, 4096, 8192}, rank in {8, 32, 64}, 0.5 / 1 / 5 % outlier
 # channels.  5 % of 8192 is nO = 410 (nOp = 416 > 128: the forward with all three accumulators resident), 5 % of
 # 2048 is nO = 102 (nOp = 128).
 SWEEP_POINTS = [(512, 2048, 4096, 8, 0.05), (2048, 8192, 2048, 32, 0.01), (32768, 2048, 2048, 64, 0.005),
                 (8192, 8192, 4096, 8, 0.05), (512, 4096, 8192, 64, 0.01), (2048, 4096, 4096, 32, 0.005),
                 (8192, 2048, 8192, 32, 0.05), (32768, 4096, 2048, 8, 0.01), (512, 8192, 8192, 32, 0.005),
-                (2048, 2048, 2048, 64, 0.05), (8192, 4096, 2048, 64, 0.005), (32768, 8192, 4096, 32, 0.01)]
+                (2048, 2048, 2048, 64, 0.05), (8192, 4096, 2048, 64, 0.005), (32768, 8192, 4096, 32, 0.01),
+                (2048, 2048, 8192, 8, 0.005), (8192, 2048, 4096, 64, 0.01), (32768, 4096, 8192, 8, 0.05),
+                (512, 8192, 2048, 64, 0.005)]
 
 
 def test_sweep_points_cover_every_axis_value():
     for axis, want in ((0, {512, 2048, 8192, 32768}), (1, {2048, 4096, 8192}), (2, {2048, 4096, 8192}), (3, {8, 32, 64}),
                        (4, {0.005, 0.01, 0.05})):
         assert {p[axis] for p in SWEEP_POINTS} == want
+    # ... and every PAIR of values of two different axes occurs together in some point
+    import itertools
+    axes = ((512, 2048, 8192, 32768), (2048, 4096, 8192), (2048, 4096, 8192), (8, 32, 64), (0.005, 0.01, 0.05))
+    for a, b in itertools.combinations(range(5), 2):
+        for va in axes[a]:
+            for vb in axes[b]:
+                assert any(p[a] == va and p[b] == vb for p in SWEEP_POINTS), (a, va, b, vb)
 
 
 @pytest.mark.parametrize("M,K,N,r,frac", SWEEP_POINTS)
