@@ -228,6 +228,31 @@ BWD_SHAPES = [(1, 128, 64, 0, 0), (128, 128, 128, 32, 16), (200, 320, 136, 5, 8)
 
 @pytest.mark.parametrize("M,K,N,nO,r", BWD_SHAPES)
 def test_qlinear_bwd(Q, M, K, N, nO, r):
+    _check_bwd(Q, M, K, N, nO, r)
+
+
+# Shapes nobody picked by hand: seeded draws over the supported ranges (ragged everything; K a multiple of 16 and N of 8,
+# which the row pitches of the contiguous test buffers need), each through the forward and through both backward paths.
+def _random_shape(seed):
+    rng = np.random.default_rng(9000 + seed)
+    M = int(rng.integers(1, 601))
+    K = 16 * int(rng.integers(1, 121))
+    N = 8 * int(rng.integers(1, 241))
+    nO = int(rng.integers(0, min(K, 140) + 1)) if seed % 4 else 0
+    r = 8 * int(rng.integers(0, 9)) if seed % 5 else 0
+    return M, K, N, nO, r
+
+
+@pytest.mark.parametrize("seed", range(24))
+def test_random_shapes_forward_and_backward(Q, seed):
+    M, K, N, nO, r = _random_shape(seed)
+    _check_fwd(Q, M, K, N, nO, r, seed % 2 == 0)
+    _check_bwd(Q, M, K, N, nO, r)
+    if N % 16 == 0:                       # the INT8 grad-input variant takes rows of whole 16-column units
+        test_qlinear_bwd_int8(Q, M, K, N, nO, r)
+
+
+def _check_bwd(Q, M, K, N, nO, r):
     import torch
     K = (K + 7) // 8 * 8
     O, X, Wt, A, B, dY = _mk_inputs(600 + M + N, M, K, N, nO, r)
