@@ -505,6 +505,22 @@ def test_quant_grad_bit_exact(Q, M, N):
     assert np.array_equal(host(dz), odz)
 
 
+@pytest.mark.parametrize("seed", range(16))
+def test_random_shapes_of_the_bit_exact_kernels(Q, seed):
+    """Seeded draws over the supported sizes for the integer-exact steps: the row width decides how many 16-column units a
+    thread holds and whether the ragged-tail variant runs, so widths nobody picked by hand are the point."""
+    rng = np.random.default_rng(7000 + seed)
+    M = int(rng.integers(1, 301))
+    K = int(rng.integers(1, 32769)) if seed % 2 else int(rng.integers(1, 4097))
+    nO = int(rng.integers(0, min(K, 300) + 1))
+    test_quant_act_bit_exact(Q, M, K, nO)
+    test_momentum_update_bit_exact(Q, M, K, max(1, nO), float(rng.integers(0, 11)) / 10.0)
+    test_requant_weight_rows_bit_exact(Q, max(1, nO), int(rng.integers(1, 5001)))
+    Kw = max(8, min(K, 4096) // 8 * 8)            # the contiguous bf16 weight of that test needs a row pitch of 16 bytes
+    test_prepare_weight_bit_exact(Q, int(rng.integers(1, 1201)), Kw, min(nO, Kw))
+    test_quant_grad_bit_exact(Q, M, 16 * int(rng.integers(1, 1025)))
+
+
 def test_quant_grad_rejects_rows_wider_than_it_is_built_for(Q):
     import torch
     dY = torch.zeros((2, 16400), dtype=torch.bfloat16, device="cuda")
