@@ -16,7 +16,7 @@ from util import TOL_BF16, check_bf16_intermediate, dev, dev_bf16, dx_floor, hos
 pytestmark = pytest.mark.gpu
 
 
-def _run_layer(wl, li, steps, nsample, check_acc, full_grads=True, int8_grad=False, lean_bwd=False):
+def _run_layer(wl, li, steps, nsample, check_acc, full_grads=True, int8_grad=False, lean_bwd=False, step_inputs=None, extra_rows=()):
     import torch
     from paper_2505_14742_b200 import build
     from paper_2505_14742_b200.layer import QuaffLinear, StepGraph
@@ -43,7 +43,7 @@ def _run_layer(wl, li, steps, nsample, check_acc, full_grads=True, int8_grad=Fal
     rng = np.random.default_rng(wl.seed + li)
     none_O, none_s, none_wq = np.zeros(0, np.int32), np.zeros(0, np.float32), np.zeros((1, 0), np.int8)
     for step in range(steps):
-        X, dY = synth.step_inputs(wl, li, step, lin)
+        X, dY = (step_inputs or synth.step_inputs)(wl, li, step, lin)
         Xd.copy_(dev_bf16(X)); dYd.copy_(dev_bf16(dY))
         if graph is None:
             body()                      # first call eagerly (function attributes), then everything through the graph
@@ -62,6 +62,7 @@ def _run_layer(wl, li, steps, nsample, check_acc, full_grads=True, int8_grad=Fal
         assert np.array_equal(host(layer.wq_O), wq) and np.array_equal(host(layer.dw_O), dw)
         rows = np.sort(rng.choice(M, nsample, replace=False))
         rows[0], rows[-1] = 0, M - 1                       # first and last row of the first and last tile
+        rows = np.unique(np.concatenate([rows, np.asarray(extra_rows, dtype=rows.dtype)]))
         Xs, dYs = np.ascontiguousarray(X[rows]), np.ascontiguousarray(dY[rows])
         Tg, Gg = host_bits(layer.T), host_bits(layer.G)
         # the bf16 intermediates of the sampled rows: at most one ulp from the oracle's; everything downstream is
@@ -98,10 +99,10 @@ def _run_layer(wl, li, steps, nsample, check_acc, full_grads=True, int8_grad=Fal
             # INT32 accumulators of the same rows through the C ABI's debug dumps (a separate call: the dumps are
             # not on the timed path)
             from paper_2505_14742_b200 import binding as Q
-            a1 = torch.empty((nsample, N), dtype=torch.int32, device="cuda")
-            a2 = torch.empty((nsample, N), dtype=torch.int32, device="cuda")
-            Ys = torch.empty((nsample, N), dtype=torch.bfloat16, device="cuda")
-            Ts = torch.empty((nsample, r), dtype=torch.bfloat16, device="cuda")
+            a1 = torch.empty((len(rows), N), dtype=torch.int32, device="cuda")
+            a2 = torch.empty((len(rows), N), dtype=torch.int32, device="cuda")
+            Ys = torch.empty((len(rows), N), dtype=torch.bfloat16, device="cuda")
+            Ts = torch.empty((len(rows), r), dtype=torch.bfloat16, device="cuda")
             Q.quaff_qlinear_fwd(dev(Xq[rows]), dev(xqo[rows]), dev(dx[rows]), layer.Wq, layer.dW, layer.wq_O, layer.dw_O,
                                 dev_bf16(Xs), layer.A, layer.B, scale, Ts, Ys, layer.ws, a1, a2, layer.status)
             torch.cuda.synchronize()
@@ -216,3 +217,32 @@ def test_shape_sweep_points(M, K, N, r, frac):
     """One forward + backward step of a sweep point through the graph-replayed layer, against the oracle."""
     wl = synth.sweep_point(M, K, N, r, frac)
     _run_layer(wl, 0, steps=1, nsample=16, check_acc=True, full_grads=False)
+
+
+def test_tensors_larger_than_two_gib():
+    """540672 tokens x 2048 channels: X, Y, dY and dX are 2.2 GB each and the INT8 codes 1.1 GB, so byte offsets of the
+    later rows do not fit 32 bits (row 524288 starts at exactly 2^31 bytes).  The batch is a block of 8192 synthetic
+    tokens repeated 66 times, each repetition scaled by another power of two (exact in bf16), so that a row fetched from
+    or stored to a wrapped address would carry the wrong magnitude.  All codes and step sizes are compared, Y / dX on
+    sampled rows on both sides of the 2^31-byte line, dA / dB on sampled columns over all tokens."""
+    import dataclasses
+    reps, block = 66, 8192
+    wl = synth.sweep_point(reps * block, 2048, 2048, 8, 0.005)
+    small = dataclasses.replace(wl, M=block)
+
+    def tiled(wl_, li, step, lin):
+        Xb, dYb = synth.step_inputs(small, li, step, lin)
+        def rep(bits):
+            expo = (bits >> 7) & 0xFF
+            ok = (expo > 8) & (expo < 240)
+            # x 1/4 .. x 4: the exponent field moves, nothing rounds
+            scaled = [np.where(ok, (bits.astype(np.int32) + (shift << 7)).astype(np.uint16), bits) for shift in range(-2, 3)]
+            out = np.empty((reps, block, bits.shape[1]), np.uint16)
+            for t in range(reps):
+                out[t] = scaled[t % 5]
+            return out.reshape(reps * block, bits.shape[1])
+        return rep(Xb), rep(dYb)
+
+    line = (1 << 31) // (2 * 2048)                                   # first row whose byte offset needs 32 bits
+    _run_layer(wl, 0, steps=1, nsample=24, check_acc=True, full_grads=False, step_inputs=tiled,
+               extra_rows=(line - 1, line, line + 1, 2 * block + 5, reps * block - 2))
