@@ -128,7 +128,9 @@ class StepGraph:
         side = torch.cuda.Stream()
         side.wait_stream(torch.cuda.current_stream())
         with torch.cuda.stream(side):
-            with torch.cuda.graph(self.graph, stream=side):
+            # thread-local capture mode: CUDA calls of OTHER host threads (a process group's watchdog, a data loader)
+            # do not invalidate the capture; what this thread enqueues is checked as strictly as before
+            with torch.cuda.graph(self.graph, stream=side, capture_error_mode="thread_local"):
                 body()
         torch.cuda.current_stream().wait_stream(side)
 
