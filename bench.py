@@ -509,7 +509,8 @@ def run_gpu(args, wl):
                              "note": "the same kernel without the LoRA-gradient GEMMs beside it (backward for dX only, L2 flushed), "
                                      "against the burst peak"}
 
-    cpu = cpu_baseline(wl, min(wl.M, 8 * args.sample_tokens), reps=2) if not args.no_cpu_baseline else None
+    # the oracle on the host cores: a single-GPU run only (with more ranks every GPU of the job would be held meanwhile)
+    cpu = cpu_baseline(wl, min(wl.M, 8 * args.sample_tokens), reps=2) if (world == 1 and not args.no_cpu_baseline) else None
     line = {"metric": METRIC, "value": qdist.whole_job_rate(M, world, ms_per_step), "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
             "repeats": {"n": args.repeats, "ms_per_step_min": float(np.min(region_ms)) / args.steps,
