@@ -139,9 +139,10 @@ struct GemmCfg {
     static constexpr int kStageBytes = kABytes + kBBytes;
     static constexpr int kScaleBytes = (EPI == EPI_FWD) ? 2 * 2 * TN * 4 : 0;   // [2 buffers][dW | dw_O][TN]
     static constexpr int kFixed = 1024 + (int)sizeof(GemmSmem) + kScaleBytes;
-    // The skinny split-K GEMMs run a handful of k-blocks per CTA: a short ring and half of TMEM leave room
-    // for a second such CTA (or other kernels) on the same SM, so that independent ones overlap.
-    static constexpr int kStageCap = (EPI == EPI_PART) ? 4 : kMaxStages;
+    // The skinny split-K GEMMs stream one operand from HBM and are bound by the latency of those loads: six stages
+    // (measured: 4 -> 6 stages takes T = X A at 8192 x 11008 from 50 to 46 us, more gives nothing); half of TMEM, so that
+    // a kernel that follows can allocate its own while this one drains.
+    static constexpr int kStageCap = (EPI == EPI_PART) ? 6 : kMaxStages;
     static constexpr int kTmemCols = (EPI == EPI_PART) ? 2 * TN : 512;
     static constexpr int kStagesFit = (kSmemLimit - kFixed) / kStageBytes;
     static constexpr int kStages = kStagesFit < kStageCap ? kStagesFit : kStageCap;
